@@ -1,0 +1,144 @@
+/*
+ * snn_conv.h -- C ABI of the sub-bit binary 3x3 convolution library (sm_100a).
+ *
+ * One layer of a Sub-bit Neural Network is stored as (Sec. 4.4 "Compression"):
+ * a layer-specific set of 2^tau binary 3x3 kernels (the codebook), one tau-bit
+ * index per (c_out, c_in) kernel, and channel-wise scales (Sec. 3).  Its
+ * forward pass is  Y = alpha * (w_bar o a_bar)  (Sec. 3; Algorithm 1, forward
+ * step), a 3x3 cross-correlation of +/-1 weights with +/-1 activations, or
+ * with fp16 activations in the weights-only setting (Sec. 5.3 deployment test,
+ * Table 2 ".../32" rows).
+ *
+ * Conventions fixed by this library:
+ *   - code of a kernel: 9-bit integer, bit (8 - (3*ky + kx)) set <=> K[ky][kx] = +1.
+ *     Code 0 is the all -1 kernel (the paper's kernel no. 1), code 511 the
+ *     all +1 kernel (no. 512) (Sec. 4.1).  Everything is 0-based here.
+ *   - index stream: element e = co*c_in + ci occupies bits [e*tau, (e+1)*tau) of
+ *     an LSB-first byte stream (tau*c_in*c_out bits in total, Sec. 4.4).
+ *   - binary activations: uint32 [N][H][W][ceil(c_in/32)], channel ci = bit ci%32
+ *     of word ci/32, bit 1 = +1, bit 0 = -1, unused high bits MUST be 0.
+ *   - fp16 activations: IEEE binary16 [N][H][W][c_in].
+ *   - output: [N][Ho][Wo][c_out], Ho = floor((H + 2*pad - 3)/stride) + 1,
+ *     int32 pre-scale sums S or fp32 Y = (float)S * alpha[co] (one multiply).
+ *   - zero padding contributes 0 to the sum (it is not a -1).
+ *
+ * All entry points return a status; on failure snn_last_error() gives a text.
+ * Nothing throws, aborts or traps.  There is no CPU fallback: every step runs
+ * in CUDA kernels, and a path that does not support a shape says so.
+ */
+#ifndef SNN_CONV_H_
+#define SNN_CONV_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SNN_API __attribute__((visibility("default")))
+#else
+#define SNN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct snn_conv snn_conv_t; /* opaque; owned by the library */
+
+typedef enum {
+  SNN_OK = 0,
+  SNN_ERR_INVALID_ARG = 1,
+  SNN_ERR_UNSUPPORTED = 2, /* path cannot run this shape; nothing was launched */
+  SNN_ERR_CUDA = 3,
+  SNN_ERR_OOM = 4,
+  SNN_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out */
+} snn_status_t;
+
+enum { SNN_ACT_BIN = 0, SNN_ACT_F16 = 1 };
+enum { SNN_OUT_F32 = 0, SNN_OUT_I32 = 1 }; /* I32 only with SNN_ACT_BIN */
+enum {
+  SNN_PATH_AUTO = 0,       /* tuned choice if snn_conv_tune ran for the shape, else a heuristic */
+  SNN_PATH_REUSE = 1,      /* codebook-reuse: per-channel partial maps + index-driven accumulate (Sec. 4.5) */
+  SNN_PATH_DECODED = 2,    /* decoded weights, XOR + popcount implicit GEMM (Sec. 3) */
+  SNN_PATH_DECODED_TC = 3  /* decoded weights on the tcgen05 tensor cores */
+};
+
+typedef struct {
+  int32_t c_in, c_out;        /* >= 1; need not be multiples of 32 */
+  int32_t tau;                /* 1..9; 9 = full 512-kernel codebook = a standard 1-bit layer (Sec. 4.1) */
+  int32_t stride, pad;        /* stride in {1,2}; pad in {0,1}; kernel is 3x3 */
+  int32_t act_type;           /* SNN_ACT_* */
+  int32_t device;             /* CUDA ordinal */
+  const uint16_t* codebook;   /* HOST, 2^tau codes, each < 512; duplicates allowed */
+  const uint8_t* idx_packed;  /* HOST, ceil(c_out*c_in*tau/8) bytes, see above */
+  const float* alpha;         /* HOST, c_out finite fp32 scales */
+} snn_conv_desc_t;
+
+/*
+ * Sec. 4.4 storage -> device form.  Copies the host arrays (the caller may free
+ * them on return), unpacks the index stream and decodes the weights on the
+ * device.  *out receives a handle that owns its device buffers.
+ * Errors: INVALID_ARG (null pointer, tau/stride/pad out of range, code >= 512,
+ * non-finite alpha, c_in/c_out < 1), CUDA, OOM.
+ */
+SNN_API snn_status_t snn_conv_create(const snn_conv_desc_t* desc, snn_conv_t** out);
+
+/*
+ * Sec. 3 / Algorithm 1 forward step for one batch.  act_dev and out_dev are
+ * DEVICE pointers owned by the caller (layouts above), act_dev 16-byte aligned,
+ * out_dev 16-byte aligned; they are neither kept nor freed.  The call is
+ * asynchronous on cuda_stream (a cudaStream_t, NULL = default stream) and does
+ * not allocate.  N may be 0 (nothing is launched).
+ * Errors: INVALID_ARG (null, H/W giving no output, I32 output with fp16
+ * activations, unknown path), UNSUPPORTED (the named path cannot run this
+ * layer; AUTO never returns it), CUDA.
+ */
+SNN_API snn_status_t snn_conv_forward(snn_conv_t* h, const void* act_dev, int32_t N, int32_t H, int32_t W,
+                              void* out_dev, int32_t out_type, int32_t path, void* cuda_stream);
+
+/*
+ * Same operation with HOST buffers: copies act_host to the device, runs the
+ * forward pass, copies the result back and waits for it.  Staging buffers live
+ * in the handle and grow on demand (the only call besides create/tune that may
+ * allocate).  Pinned host memory makes the copies asynchronous.
+ */
+SNN_API snn_status_t snn_conv_forward_host(snn_conv_t* h, const void* act_host, int32_t N, int32_t H, int32_t W,
+                                   void* out_host, int32_t out_type, int32_t path);
+
+/*
+ * Path selection from measured time (Sec. 4.5: the gain of sharing depends on
+ * 2^tau / c_out, so the choice is per layer shape).  Times every supported
+ * path on zero-filled scratch inputs of the given shape and remembers the
+ * fastest for (N, H, W).  Synchronous.  *best_path / ms[4] (indexed by
+ * SNN_PATH_*, negative = unsupported) may be NULL.
+ */
+SNN_API snn_status_t snn_conv_tune(snn_conv_t* h, int32_t N, int32_t H, int32_t W, int32_t* best_path, float* ms);
+
+/* Path SNN_PATH_AUTO would take for this shape (never AUTO itself). */
+SNN_API int32_t snn_conv_chosen_path(const snn_conv_t* h, int32_t N, int32_t H, int32_t W);
+
+/* SNN_OK if `path` can run this layer at this shape, else SNN_ERR_UNSUPPORTED. */
+SNN_API snn_status_t snn_conv_path_supported(const snn_conv_t* h, int32_t path, int32_t N, int32_t H, int32_t W);
+
+/* Frees the handle and its device buffers.  NULL is a no-op returning SNN_OK. */
+SNN_API snn_status_t snn_conv_destroy(snn_conv_t* h);
+
+/* Text of the calling thread's last failure; never NULL. */
+SNN_API const char* snn_last_error(void);
+
+SNN_API const char* snn_version(void);
+
+/* Number of kernels this library has launched in this process (all handles). */
+SNN_API int64_t snn_kernel_launches(void);
+
+/*
+ * Measured instruction-rate ceilings used as roofline denominators for the
+ * ALU paths: runs a short saturating loop of one instruction kind on `device`
+ * and returns results per second in *rate (per-lane results: a warp
+ * instruction counts 32).  kind: 0 = POPC, 1 = LOP3 (xor), 2 = IADD3,
+ * 3 = LDS.32 (conflict-free), 4 = XOR+POPC+IADD chain as the decoded loop issues it.
+ */
+SNN_API snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SNN_CONV_H_ */

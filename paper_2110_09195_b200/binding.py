@@ -1,0 +1,220 @@
+"""ctypes binding of include/snn_conv.h: argument marshalling only.
+
+The names mirror the C entry points (snn_conv_create -> SnnConv(...),
+snn_conv_forward -> SnnConv.forward, ...).  Tensors are torch CUDA tensors
+used purely as device memory; streams come from torch.  There is no fallback:
+if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import numpy as np
+
+ACT_BIN, ACT_F16 = 0, 1
+OUT_F32, OUT_I32 = 0, 1
+PATH_AUTO, PATH_REUSE, PATH_DECODED, PATH_DECODED_TC = 0, 1, 2, 3
+PATH_NAMES = {PATH_AUTO: "auto", PATH_REUSE: "reuse", PATH_DECODED: "decoded", PATH_DECODED_TC: "decoded_tc"}
+_STATUS = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "CUDA", 4: "OOM", 5: "TIMEOUT"}
+
+_LIB_PATH = Path(__file__).resolve().parent / "libsnnconv.so"
+_lib = None
+
+# every symbol include/snn_conv.h declares
+EXPORTED_SYMBOLS = (
+    "snn_conv_create", "snn_conv_forward", "snn_conv_forward_host", "snn_conv_tune", "snn_conv_chosen_path",
+    "snn_conv_path_supported", "snn_conv_destroy", "snn_last_error", "snn_version", "snn_kernel_launches",
+    "snn_microbench",
+)
+
+
+class SnnError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"snnconv {_STATUS.get(status, status)}: {message}")
+        self.status = status
+        self.status_name = _STATUS.get(status, str(status))
+
+
+class _Desc(ctypes.Structure):
+    _fields_ = [
+        ("c_in", ctypes.c_int32), ("c_out", ctypes.c_int32), ("tau", ctypes.c_int32),
+        ("stride", ctypes.c_int32), ("pad", ctypes.c_int32), ("act_type", ctypes.c_int32),
+        ("device", ctypes.c_int32),
+        ("codebook", ctypes.c_void_p), ("idx_packed", ctypes.c_void_p), ("alpha", ctypes.c_void_p),
+    ]
+
+
+def library_path() -> Path:
+    return _LIB_PATH
+
+
+def load_library():
+    """Loads libsnnconv.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise ImportError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2110_09195_b200.build` "
+            "(nvcc, sm_100a).  This package has no CPU or PyTorch fallback.")
+    lib = ctypes.CDLL(str(_LIB_PATH))
+    i32, vp = ctypes.c_int32, ctypes.c_void_p
+    lib.snn_conv_create.restype = i32
+    lib.snn_conv_create.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(vp)]
+    lib.snn_conv_forward.restype = i32
+    lib.snn_conv_forward.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, vp]
+    lib.snn_conv_forward_host.restype = i32
+    lib.snn_conv_forward_host.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32]
+    lib.snn_conv_tune.restype = i32
+    lib.snn_conv_tune.argtypes = [vp, i32, i32, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_float)]
+    lib.snn_conv_chosen_path.restype = i32
+    lib.snn_conv_chosen_path.argtypes = [vp, i32, i32, i32]
+    lib.snn_conv_path_supported.restype = i32
+    lib.snn_conv_path_supported.argtypes = [vp, i32, i32, i32, i32]
+    lib.snn_conv_destroy.restype = i32
+    lib.snn_conv_destroy.argtypes = [vp]
+    lib.snn_last_error.restype = ctypes.c_char_p
+    lib.snn_last_error.argtypes = []
+    lib.snn_version.restype = ctypes.c_char_p
+    lib.snn_version.argtypes = []
+    lib.snn_kernel_launches.restype = ctypes.c_int64
+    lib.snn_kernel_launches.argtypes = []
+    lib.snn_microbench.restype = i32
+    lib.snn_microbench.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double)]
+    _lib = lib
+    return lib
+
+
+def _check(status: int):
+    if status != 0:
+        raise SnnError(status, load_library().snn_last_error().decode("utf-8", "replace"))
+
+
+def version() -> str:
+    return load_library().snn_version().decode()
+
+
+def kernel_launches() -> int:
+    return int(load_library().snn_kernel_launches())
+
+
+def microbench(kind: int, device: int = 0) -> float:
+    rate = ctypes.c_double(0.0)
+    _check(load_library().snn_microbench(kind, device, ctypes.byref(rate)))
+    return float(rate.value)
+
+
+class SnnConv:
+    """One sub-bit 3x3 layer on one GPU (wraps a snn_conv_t handle)."""
+
+    def __init__(self, c_in, c_out, tau, codebook, idx_packed, alpha, stride=1, pad=1, act_type=ACT_BIN, device=0):
+        lib = load_library()
+        cb = np.ascontiguousarray(codebook, dtype=np.uint16)
+        ip = np.ascontiguousarray(idx_packed, dtype=np.uint8)
+        al = np.ascontiguousarray(alpha, dtype=np.float32)
+        if not 1 <= int(tau) <= 9:
+            raise SnnError(1, f"tau={tau} outside 1..9")
+        if cb.size != (1 << int(tau)):
+            raise SnnError(1, f"codebook has {cb.size} entries, expected {1 << int(tau)}")
+        if ip.size < (int(c_out) * int(c_in) * int(tau) + 7) // 8:
+            raise SnnError(1, "index stream shorter than c_out*c_in*tau bits")
+        if al.size != int(c_out):
+            raise SnnError(1, f"alpha has {al.size} entries, expected {c_out}")
+        d = _Desc(int(c_in), int(c_out), int(tau), int(stride), int(pad), int(act_type), int(device),
+                  cb.ctypes.data, ip.ctypes.data, al.ctypes.data)
+        h = ctypes.c_void_p()
+        self._h = None
+        _check(lib.snn_conv_create(ctypes.byref(d), ctypes.byref(h)))
+        self._h = h
+        self.c_in, self.c_out, self.tau = int(c_in), int(c_out), int(tau)
+        self.stride, self.pad, self.act_type, self.device = int(stride), int(pad), int(act_type), int(device)
+
+    # -- helpers ------------------------------------------------------------
+    def out_hw(self, h, w):
+        return (h + 2 * self.pad - 3) // self.stride + 1, (w + 2 * self.pad - 3) // self.stride + 1
+
+    def _check_act(self, act):
+        import torch
+        if self.act_type == ACT_BIN:
+            if act.dtype not in (torch.int32, torch.uint32) or act.dim() != 4 or act.shape[3] != (self.c_in + 31) // 32:
+                raise SnnError(1, "binary activations must be int32/uint32 (N, H, W, ceil(c_in/32))")
+        else:
+            if act.dtype != torch.float16 or act.dim() != 4 or act.shape[3] != self.c_in:
+                raise SnnError(1, "fp16 activations must be float16 (N, H, W, c_in)")
+        if not act.is_contiguous():
+            raise SnnError(1, "activations must be contiguous")
+
+    def alloc_out(self, n, h, w, out_type=OUT_F32, device=None, pin=False):
+        import torch
+        ho, wo = self.out_hw(h, w)
+        dt = torch.float32 if out_type == OUT_F32 else torch.int32
+        if device is None:
+            device = f"cuda:{self.device}"
+        if pin:
+            return torch.empty((n, ho, wo, self.c_out), dtype=dt, pin_memory=True)
+        return torch.empty((n, ho, wo, self.c_out), dtype=dt, device=device)
+
+    # -- the C entry points -------------------------------------------------
+    def forward(self, act, out=None, out_type=OUT_F32, path=PATH_AUTO, stream=None):
+        """snn_conv_forward: act / out are CUDA tensors; asynchronous on `stream`
+        (default: torch's current stream)."""
+        import torch
+        if not act.is_cuda or act.device.index != self.device:
+            raise SnnError(1, f"activations must live on cuda:{self.device}")
+        self._check_act(act)
+        n, h, w = int(act.shape[0]), int(act.shape[1]), int(act.shape[2])
+        if out is None:
+            out = self.alloc_out(n, h, w, out_type)
+        else:
+            ho, wo = self.out_hw(h, w)
+            want = torch.float32 if out_type == OUT_F32 else torch.int32
+            if (not out.is_cuda or out.device.index != self.device or out.dtype != want or not out.is_contiguous()
+                    or tuple(out.shape) != (n, ho, wo, self.c_out)):
+                raise SnnError(1, "output tensor has the wrong device, dtype, shape or layout")
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        _check(load_library().snn_conv_forward(self._h, act.data_ptr(), n, h, w, out.data_ptr(), int(out_type),
+                                               int(path), ctypes.c_void_p(stream.cuda_stream)))
+        return out
+
+    def forward_host(self, act, out=None, out_type=OUT_F32, path=PATH_AUTO):
+        """snn_conv_forward_host: act / out are CPU tensors (pinned for speed);
+        synchronous, copies included."""
+        import torch
+        if act.is_cuda:
+            raise SnnError(1, "forward_host takes CPU tensors")
+        self._check_act(act)
+        n, h, w = int(act.shape[0]), int(act.shape[1]), int(act.shape[2])
+        if out is None:
+            out = self.alloc_out(n, h, w, out_type, pin=True)
+        _check(load_library().snn_conv_forward_host(self._h, act.data_ptr(), n, h, w, out.data_ptr(), int(out_type),
+                                                    int(path)))
+        return out
+
+    def tune(self, n, h, w):
+        """snn_conv_tune: returns (best_path, [ms per path], negative = unsupported)."""
+        best = ctypes.c_int32(0)
+        ms = (ctypes.c_float * 4)()
+        _check(load_library().snn_conv_tune(self._h, int(n), int(h), int(w), ctypes.byref(best), ms))
+        return int(best.value), [float(v) for v in ms]
+
+    def chosen_path(self, n, h, w) -> int:
+        return int(load_library().snn_conv_chosen_path(self._h, int(n), int(h), int(w)))
+
+    def path_supported(self, path, n, h, w) -> bool:
+        st = load_library().snn_conv_path_supported(self._h, int(path), int(n), int(h), int(w))
+        if st not in (0, 2):
+            _check(st)
+        return st == 0
+
+    def destroy(self):
+        if getattr(self, "_h", None) is not None:
+            load_library().snn_conv_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

@@ -1,0 +1,416 @@
+// Host side of the C ABI declared in include/snn_conv.h: argument checks,
+// the layer handle, path selection and the launches.  No arithmetic of the
+// method happens on the host.
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <new>
+#include <tuple>
+
+#include "snn_internal.h"
+
+using namespace snn;
+
+namespace {
+
+thread_local char g_err[512] = "";
+std::atomic<long long> g_launches{0};
+
+snn_status_t fail(snn_status_t st, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  if (getenv("SNN_LOG")) fprintf(stderr, "[snnconv] error %d: %s\n", (int)st, g_err);
+  return st;
+}
+
+snn_status_t cuda_fail(cudaError_t e, const char* what) {
+  snn_status_t st = (e == cudaErrorMemoryAllocation) ? SNN_ERR_OOM : SNN_ERR_CUDA;
+  return fail(st, "%s: %s", what, cudaGetErrorString(e));
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) return;
+    ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+}  // namespace
+
+struct snn_conv {
+  int C, K, tau, stride, pad, act_type, device;
+  LayerDev L;
+  std::mutex mu;
+  std::map<std::tuple<int, int, int>, int> tuned;  // (N,H,W) -> path
+  // staging for snn_conv_forward_host
+  void* stage_in = nullptr;
+  void* stage_out = nullptr;
+  size_t stage_in_bytes = 0, stage_out_bytes = 0;
+  cudaStream_t host_stream = nullptr;
+  int* tc_status_host = nullptr;  // pinned, written by the tensor-core kernel on a bounded-wait timeout
+};
+
+namespace {
+
+bool make_geom(const snn_conv* h, int N, int H, int W, Geom* g) {
+  if (N < 0 || H < 1 || W < 1) return false;
+  if (H + 2 * h->pad < 3 || W + 2 * h->pad < 3) return false;
+  g->N = N; g->H = H; g->W = W;
+  g->C = h->C; g->K = h->K; g->Cw = (h->C + 31) / 32;
+  g->stride = h->stride; g->pad = h->pad;
+  g->Ho = (H + 2 * h->pad - 3) / h->stride + 1;
+  g->Wo = (W + 2 * h->pad - 3) / h->stride + 1;
+  g->tau = h->tau; g->T = 1 << h->tau;
+  // index arithmetic in the kernels is 32-bit for pixel counts
+  long long in_px = (long long)N * H * W, out_px = (long long)N * g->Ho * g->Wo;
+  if (in_px >= (1ll << 31) || out_px >= (1ll << 31)) return false;
+  return true;
+}
+
+bool path_ok(const snn_conv* h, int path, const Geom& g) {
+  switch (path) {
+    case SNN_PATH_REUSE: return reuse_supported(g, h->act_type);
+    case SNN_PATH_DECODED: return popc_supported(g, h->act_type);
+    case SNN_PATH_DECODED_TC: return tc_supported(g, h->act_type);
+    default: return false;
+  }
+}
+
+// Untuned default: tensor cores when they apply, else the popcount path for
+// small c_out relative to the codebook and the reuse path for large (Sec. 4.5:
+// sharing pays in proportion to c_out / 2^tau).
+int heuristic_path(const snn_conv* h, const Geom& g) {
+  if (path_ok(h, SNN_PATH_DECODED_TC, g)) return SNN_PATH_DECODED_TC;
+  if (h->act_type == SNN_ACT_BIN) {
+    if (g.K >= 4 * g.T && path_ok(h, SNN_PATH_REUSE, g)) return SNN_PATH_REUSE;
+    if (path_ok(h, SNN_PATH_DECODED, g)) return SNN_PATH_DECODED;
+  }
+  if (path_ok(h, SNN_PATH_REUSE, g)) return SNN_PATH_REUSE;
+  return SNN_PATH_DECODED;
+}
+
+int auto_path(snn_conv* h, const Geom& g) {
+  if (const char* f = getenv("SNN_FORCE_PATH")) {
+    int v = atoi(f);
+    if (v >= 1 && v <= 3 && path_ok(h, v, g)) return v;
+  }
+  {
+    std::lock_guard<std::mutex> lk(h->mu);
+    auto it = h->tuned.find(std::make_tuple(g.N, g.H, g.W));
+    if (it != h->tuned.end()) return it->second;
+  }
+  return heuristic_path(h, g);
+}
+
+snn_status_t run_path(snn_conv* h, int path, const Geom& g, const Launch& l) {
+  int launched = 0;
+  cudaError_t e = cudaSuccess;
+  switch (path) {
+    case SNN_PATH_REUSE: e = reuse_forward(h->L, g, h->act_type, l, &launched); break;
+    case SNN_PATH_DECODED: e = popc_forward(h->L, g, l, &launched); break;
+    case SNN_PATH_DECODED_TC: e = tc_forward(h->L, g, h->act_type, l, &launched, h->tc_status_host); break;
+    default: return fail(SNN_ERR_INVALID_ARG, "unknown path %d", path);
+  }
+  g_launches += launched;
+  if (e != cudaSuccess) return cuda_fail(e, "kernel launch");
+  return SNN_OK;
+}
+
+snn_status_t check_forward_args(snn_conv* h, const void* act, int N, int H, int W, void* out, int out_type, int path,
+                                Geom* g, int* chosen) {
+  if (!h) return fail(SNN_ERR_INVALID_ARG, "null handle");
+  if (out_type != SNN_OUT_F32 && out_type != SNN_OUT_I32) return fail(SNN_ERR_INVALID_ARG, "bad out_type %d", out_type);
+  if (out_type == SNN_OUT_I32 && h->act_type != SNN_ACT_BIN)
+    return fail(SNN_ERR_INVALID_ARG, "int32 output needs binary activations");
+  if (path < SNN_PATH_AUTO || path > SNN_PATH_DECODED_TC) return fail(SNN_ERR_INVALID_ARG, "unknown path %d", path);
+  if (!make_geom(h, N, H, W, g))
+    return fail(SNN_ERR_INVALID_ARG, "shape N=%d H=%d W=%d gives no output (pad %d) or is too large", N, H, W, h->pad);
+  if (N > 0 && (!act || !out)) return fail(SNN_ERR_INVALID_ARG, "null activation / output pointer");
+  if (((uintptr_t)act & 15) || ((uintptr_t)out & 15))
+    return fail(SNN_ERR_INVALID_ARG, "activation / output pointers must be 16-byte aligned");
+  int pth = path;
+  if (pth == SNN_PATH_AUTO) pth = auto_path(h, *g);
+  else if (!path_ok(h, pth, *g))
+    return fail(SNN_ERR_UNSUPPORTED, "path %d does not support this layer (act_type %d, C=%d K=%d)", pth, h->act_type,
+                h->C, h->K);
+  *chosen = pth;
+  return SNN_OK;
+}
+
+size_t act_bytes(const snn_conv* h, const Geom& g) {
+  size_t px = (size_t)g.N * g.H * g.W;
+  return h->act_type == SNN_ACT_BIN ? px * g.Cw * 4 : px * g.C * 2;
+}
+size_t out_bytes(const Geom& g) { return (size_t)g.N * g.Ho * g.Wo * g.K * 4; }
+
+}  // namespace
+
+extern "C" {
+
+const char* snn_last_error(void) { return g_err; }
+const char* snn_version(void) { return "snnconv 0.1 (sm_100a)"; }
+int64_t snn_kernel_launches(void) { return (int64_t)g_launches.load(); }
+
+snn_status_t snn_conv_create(const snn_conv_desc_t* d, snn_conv_t** out) {
+  if (!out) return fail(SNN_ERR_INVALID_ARG, "null out pointer");
+  *out = nullptr;
+  if (!d) return fail(SNN_ERR_INVALID_ARG, "null descriptor");
+  if (!d->codebook || !d->idx_packed || !d->alpha) return fail(SNN_ERR_INVALID_ARG, "null codebook / index / alpha");
+  if (d->c_in < 1 || d->c_out < 1) return fail(SNN_ERR_INVALID_ARG, "c_in=%d c_out=%d", d->c_in, d->c_out);
+  if (d->c_in > (1 << 16) || d->c_out > (1 << 16)) return fail(SNN_ERR_INVALID_ARG, "channel count above 65536");
+  if (d->tau < 1 || d->tau > 9) return fail(SNN_ERR_INVALID_ARG, "tau=%d outside 1..9", d->tau);
+  if (d->stride < 1 || d->stride > 2) return fail(SNN_ERR_INVALID_ARG, "stride=%d outside {1,2}", d->stride);
+  if (d->pad < 0 || d->pad > 1) return fail(SNN_ERR_INVALID_ARG, "pad=%d outside {0,1}", d->pad);
+  if (d->act_type != SNN_ACT_BIN && d->act_type != SNN_ACT_F16)
+    return fail(SNN_ERR_INVALID_ARG, "act_type=%d", d->act_type);
+  const int T = 1 << d->tau;
+  for (int j = 0; j < T; ++j)
+    if (d->codebook[j] >= 512) return fail(SNN_ERR_INVALID_ARG, "codebook[%d]=%u is not a 9-bit code", j, d->codebook[j]);
+  for (int k = 0; k < d->c_out; ++k)
+    if (!std::isfinite(d->alpha[k])) return fail(SNN_ERR_INVALID_ARG, "alpha[%d] is not finite", k);
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+    cudaGetLastError();
+    return fail(SNN_ERR_CUDA, "no CUDA device available (this library has no CPU path)");
+  }
+  if (d->device < 0 || d->device >= ndev) return fail(SNN_ERR_INVALID_ARG, "device %d of %d", d->device, ndev);
+  DeviceGuard guard(d->device);
+  if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", d->device);
+
+  snn_conv* h = new (std::nothrow) snn_conv();
+  if (!h) return fail(SNN_ERR_OOM, "host allocation failed");
+  h->C = d->c_in; h->K = d->c_out; h->tau = d->tau; h->stride = d->stride; h->pad = d->pad;
+  h->act_type = d->act_type; h->device = d->device;
+  Geom g;
+  make_geom(h, 0, 3, 3, &g);
+  const size_t n_elem = (size_t)h->K * h->C;
+  const size_t idx_bytes = (n_elem * h->tau + 7) / 8;
+  const int Tp = (T + 15) / 16 * 16;
+  uint8_t* d_stream = nullptr;
+  cudaError_t e = cudaSuccess;
+  auto alloc = [&](void** p, size_t bytes) {
+    if (e == cudaSuccess) e = cudaMalloc(p, bytes ? bytes : 16);
+  };
+  alloc((void**)&d_stream, idx_bytes + 4);
+  alloc((void**)&h->L.idx, n_elem * 2);
+  alloc((void**)&h->L.codebook, (size_t)T * 2);
+  alloc((void**)&h->L.alpha, (size_t)h->K * 4);
+  alloc((void**)&h->L.wplanes, (size_t)9 * g.Cw * h->K * 4);
+  alloc((void**)&h->L.corr, (size_t)16 * h->K * 4);
+  alloc((void**)&h->L.match9, (size_t)Tp * 512);
+  size_t tcw = tc_weight_bytes(g, h->act_type, &h->L.Kpad, &h->L.Cpad);
+  if (tcw) {
+    if (h->act_type == SNN_ACT_BIN) alloc((void**)&h->L.w8, tcw);
+    else alloc((void**)&h->L.w16, tcw);
+  }
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->host_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaHostAlloc((void**)&h->tc_status_host, sizeof(int), cudaHostAllocMapped);
+  if (e == cudaSuccess) *h->tc_status_host = 0;
+  cudaStream_t s = h->host_stream;
+  if (e == cudaSuccess) e = cudaMemcpyAsync(d_stream, d->idx_packed, idx_bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(h->L.codebook, d->codebook, (size_t)T * 2, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(h->L.alpha, d->alpha, (size_t)h->K * 4, cudaMemcpyHostToDevice, s);
+  int launched = 0;
+  if (e == cudaSuccess) e = decode_layer(h->L, d_stream, g, h->act_type, s, &launched);
+  g_launches += launched;
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (d_stream) cudaFree(d_stream);
+  if (e != cudaSuccess) {
+    snn_status_t st = cuda_fail(e, "snn_conv_create");
+    snn_conv_destroy(h);
+    cudaGetLastError();
+    return st;
+  }
+  *out = h;
+  return SNN_OK;
+}
+
+snn_status_t snn_conv_destroy(snn_conv_t* h) {
+  if (!h) return SNN_OK;
+  DeviceGuard guard(h->device);
+  cudaFree(h->L.idx);
+  cudaFree(h->L.codebook);
+  cudaFree(h->L.alpha);
+  cudaFree(h->L.wplanes);
+  cudaFree(h->L.corr);
+  cudaFree(h->L.match9);
+  cudaFree(h->L.w8);
+  cudaFree(h->L.w16);
+  cudaFree(h->stage_in);
+  cudaFree(h->stage_out);
+  if (h->tc_status_host) cudaFreeHost(h->tc_status_host);
+  if (h->host_stream) cudaStreamDestroy(h->host_stream);
+  delete h;
+  return SNN_OK;
+}
+
+snn_status_t snn_conv_forward(snn_conv_t* h, const void* act_dev, int32_t N, int32_t H, int32_t W, void* out_dev,
+                              int32_t out_type, int32_t path, void* cuda_stream) {
+  Geom g;
+  int chosen = 0;
+  snn_status_t st = check_forward_args(h, act_dev, N, H, W, out_dev, out_type, path, &g, &chosen);
+  if (st != SNN_OK) return st;
+  if (N == 0) return SNN_OK;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", h->device);
+  if (h->tc_status_host && *h->tc_status_host) {
+    int code = *h->tc_status_host;
+    *h->tc_status_host = 0;
+    return fail(SNN_ERR_TIMEOUT, "an earlier tensor-core launch gave up a bounded wait (code %d)", code);
+  }
+  Launch l{act_dev, out_dev, out_type == SNN_OUT_I32, (cudaStream_t)cuda_stream};
+  return run_path(h, chosen, g, l);
+}
+
+snn_status_t snn_conv_forward_host(snn_conv_t* h, const void* act_host, int32_t N, int32_t H, int32_t W,
+                                   void* out_host, int32_t out_type, int32_t path) {
+  if (!h) return fail(SNN_ERR_INVALID_ARG, "null handle");
+  Geom g;
+  if (!make_geom(h, N, H, W, &g)) return fail(SNN_ERR_INVALID_ARG, "shape N=%d H=%d W=%d gives no output", N, H, W);
+  if (N == 0) return SNN_OK;
+  if (!act_host || !out_host) return fail(SNN_ERR_INVALID_ARG, "null host pointer");
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", h->device);
+  const size_t ib = act_bytes(h, g), ob = out_bytes(g);
+  cudaError_t e = cudaSuccess;
+  if (ib > h->stage_in_bytes) {
+    cudaFree(h->stage_in);
+    h->stage_in = nullptr; h->stage_in_bytes = 0;
+    e = cudaMalloc(&h->stage_in, ib);
+    if (e != cudaSuccess) return cuda_fail(e, "staging input");
+    h->stage_in_bytes = ib;
+  }
+  if (ob > h->stage_out_bytes) {
+    cudaFree(h->stage_out);
+    h->stage_out = nullptr; h->stage_out_bytes = 0;
+    e = cudaMalloc(&h->stage_out, ob);
+    if (e != cudaSuccess) return cuda_fail(e, "staging output");
+    h->stage_out_bytes = ob;
+  }
+  cudaStream_t s = h->host_stream;
+  e = cudaMemcpyAsync(h->stage_in, act_host, ib, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return cuda_fail(e, "host to device copy");
+  snn_status_t st = snn_conv_forward(h, h->stage_in, N, H, W, h->stage_out, out_type, path, (void*)s);
+  if (st != SNN_OK) return st;
+  e = cudaMemcpyAsync(out_host, h->stage_out, ob, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(e, "device to host copy");
+  if (h->tc_status_host && *h->tc_status_host) {
+    int code = *h->tc_status_host;
+    *h->tc_status_host = 0;
+    return fail(SNN_ERR_TIMEOUT, "tensor-core kernel gave up a bounded wait (code %d)", code);
+  }
+  return SNN_OK;
+}
+
+snn_status_t snn_conv_path_supported(const snn_conv_t* h, int32_t path, int32_t N, int32_t H, int32_t W) {
+  if (!h) return fail(SNN_ERR_INVALID_ARG, "null handle");
+  Geom g;
+  if (!make_geom(h, N, H, W, &g)) return fail(SNN_ERR_INVALID_ARG, "shape gives no output");
+  if (path == SNN_PATH_AUTO) return SNN_OK;
+  return path_ok(h, path, g) ? SNN_OK : SNN_ERR_UNSUPPORTED;
+}
+
+int32_t snn_conv_chosen_path(const snn_conv_t* h, int32_t N, int32_t H, int32_t W) {
+  if (!h) return SNN_PATH_AUTO;
+  Geom g;
+  if (!make_geom(h, N, H, W, &g)) return SNN_PATH_AUTO;
+  return auto_path(const_cast<snn_conv*>(h), g);
+}
+
+snn_status_t snn_conv_tune(snn_conv_t* h, int32_t N, int32_t H, int32_t W, int32_t* best_path, float* ms) {
+  if (!h) return fail(SNN_ERR_INVALID_ARG, "null handle");
+  Geom g;
+  if (!make_geom(h, N, H, W, &g) || N < 1) return fail(SNN_ERR_INVALID_ARG, "shape gives no output");
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", h->device);
+  void *a = nullptr, *o = nullptr;
+  cudaError_t e = cudaMalloc(&a, act_bytes(h, g));
+  if (e == cudaSuccess) e = cudaMalloc(&o, out_bytes(g));
+  if (e == cudaSuccess) e = cudaMemset(a, 0x5a, act_bytes(h, g));
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  if (e == cudaSuccess) e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  if (e != cudaSuccess) {
+    cudaFree(a); cudaFree(o);
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    return cuda_fail(e, "snn_conv_tune setup");
+  }
+  if (h->act_type == SNN_ACT_BIN && (h->C & 31)) {
+    // keep the unused high bits of the last word zero, as the layout requires
+    // (0x5a5a5a5a has bits above C set): clear and use an all -1 input instead
+    cudaMemset(a, 0, act_bytes(h, g));
+  }
+  if (h->act_type == SNN_ACT_F16) cudaMemset(a, 0x3c, act_bytes(h, g));  // 0x3c3c = 1.0586 in fp16
+  cudaStream_t s = h->host_stream;
+  float best = -1.f;
+  int best_p = 0;
+  snn_status_t st = SNN_OK;
+  for (int pth = 1; pth <= 3; ++pth) {
+    if (ms) ms[pth] = -1.f;
+    if (!path_ok(h, pth, g)) continue;
+    Launch l{a, o, 0, s};
+    const int reps = 5;
+    for (int w = 0; w < 2 && st == SNN_OK; ++w) st = run_path(h, pth, g, l);
+    if (st != SNN_OK) break;
+    cudaEventRecord(e0, s);
+    for (int r = 0; r < reps && st == SNN_OK; ++r) st = run_path(h, pth, g, l);
+    cudaEventRecord(e1, s);
+    e = cudaEventSynchronize(e1);
+    if (st != SNN_OK) break;
+    if (e != cudaSuccess) { st = cuda_fail(e, "snn_conv_tune timing"); break; }
+    float t = 0.f;
+    cudaEventElapsedTime(&t, e0, e1);
+    t /= reps;
+    if (ms) ms[pth] = t;
+    if (best < 0.f || t < best) { best = t; best_p = pth; }
+  }
+  if (ms) ms[0] = best;
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  cudaFree(a);
+  cudaFree(o);
+  if (st != SNN_OK) return st;
+  if (!best_p) return fail(SNN_ERR_UNSUPPORTED, "no path supports this layer");
+  {
+    std::lock_guard<std::mutex> lk(h->mu);
+    h->tuned[std::make_tuple(N, H, W)] = best_p;
+  }
+  if (best_path) *best_path = best_p;
+  if (getenv("SNN_LOG"))
+    fprintf(stderr, "[snnconv] tuned C=%d K=%d tau=%d N=%d %dx%d -> path %d (%.4f ms)\n", h->C, h->K, h->tau, N, H, W,
+            best_p, best);
+  return SNN_OK;
+}
+
+snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate) {
+  if (!rate) return fail(SNN_ERR_INVALID_ARG, "null rate pointer");
+  if (kind < 0 || kind > 4) return fail(SNN_ERR_INVALID_ARG, "unknown microbenchmark %d", kind);
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
+    cudaGetLastError();
+    return fail(SNN_ERR_CUDA, "device %d not available", device);
+  }
+  DeviceGuard guard(device);
+  if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", device);
+  cudaError_t e = microbench(kind, rate);
+  g_launches += 2;
+  if (e != cudaSuccess) return cuda_fail(e, "snn_microbench");
+  return SNN_OK;
+}
+
+}  // extern "C"
