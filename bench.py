@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the sub-bit binary 3x3 convolution library on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+One "step" is one pass of the whole hot path over one batch: the 16 binary 3x3
+layers of the ImageNet ResNet-18-shaped stack (batch 64 per GPU, tau = 5,
+bit-packed +/-1 activations), each layer on its own seeded synthetic input,
+launched back to back on one stream through the C ABI.  Prints ONE JSON line.
+
+With N > 1 (torchrun) every rank runs its own batch of 64 on its own GPU: the
+images are independent, there is no exchange step, so the scaling is weak and
+no collective is on the data path (only the timing reduction uses one).
+
+`--impl reference` times the CPU oracle (oracle/, the plain nested-loop
+definition) on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "ResNet-18 binary conv-stack img/s (dense-equivalent binary-conv TOPS in effective_tops)"
+UNIT = "img/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs."""
+
+    def __init__(self, device_index: int, period_s: float = 0.05):
+        self.idx, self.period = device_index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = device_index
+            if visible:
+                ids = [v for v in visible.split(",") if v.strip()]
+                if device_index < len(ids) and ids[device_index].strip().isdigit():
+                    phys = int(ids[device_index])
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join(timeout=2)
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------
+# reference arm: the CPU oracle on the host cores
+# --------------------------------------------------------------------------
+def time_oracle_stack(workload, n_images: int, max_layers=None):
+    """Runs n_images through every layer of the stack with the oracle; returns seconds."""
+    import oracle
+    t_total = 0.0
+    for i, shape in enumerate(workload.layers[:max_layers]):
+        seed = wl.layer_seed(workload.config, i)
+        p = wl.draw_layer_params(shape, workload.tau, seed)
+        if workload.act == "bin":
+            act = wl.pack_activation_bits(wl.draw_activation_bits(shape, n_images, seed))
+            t0 = time.perf_counter()
+            oracle.conv_bin(p.codebook, workload.tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out, shape.stride,
+                            shape.pad, act)
+            t_total += time.perf_counter() - t0
+        else:
+            act = wl.draw_activation_f16(shape, n_images, seed)
+            t0 = time.perf_counter()
+            oracle.conv_f16(p.codebook, workload.tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out, shape.stride,
+                            shape.pad, act)
+            t_total += time.perf_counter() - t0
+    return t_total
+
+
+def oracle_sample_images(workload, budget_s: float = 15.0) -> int:
+    """Images per step so that one oracle pass over the stack takes about budget_s."""
+    import oracle
+    oracle.build()
+    t1 = time_oracle_stack(workload, 1)
+    n = int(max(1, min(workload.batch, budget_s / max(t1, 1e-6))))
+    return n
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    workload = wl.get_workload(args.workload)
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    # bound the whole run to a few minutes: at most ~120 s of oracle time in total
+    per_step_budget = max(1.0, min(15.0, 120.0 / (steps + warmup)))
+    n_img = oracle_sample_images(workload, per_step_budget)
+    for _ in range(warmup):
+        time_oracle_stack(workload, n_img)
+    t = 0.0
+    for _ in range(steps):
+        t += time_oracle_stack(workload, n_img)
+    ms = t / steps * 1e3
+    value = n_img / (ms * 1e-3)
+    cores = oracle.threads()
+    sample = f"{n_img} of {workload.batch} images through all {len(workload.layers)} layers per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32" if workload.act == "bin" else "f64", "data": "synthetic",
+        "config": {"workload": _workload_name(workload), "images_per_step": n_img},
+        "effective_tops": 2 * workload.with_batch(n_img).dense_macs() / (ms * 1e-3) / 1e12,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def _workload_name(workload):
+    return f"{workload.name}_stack_n{workload.batch}_tau{workload.tau}_{workload.act}"
+
+
+# --------------------------------------------------------------------------
+# own arm
+# --------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2110_09195_b200 as snn
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    snn.load_library()
+    peaks = _peaks()
+    workload = wl.get_workload(args.workload, tau=args.tau, batch=args.batch)
+    first_layer = 0
+    if args.layers:
+        lo, hi = (int(v) for v in args.layers.split(":"))
+        first_layer = lo
+        workload = wl.Workload(workload.name + f"[{lo}:{hi}]", workload.config, workload.batch, workload.tau,
+                               workload.act, workload.layers[lo:hi])
+    nb = workload.batch
+    act_code = snn.ACT_BIN if workload.act == "bin" else snn.ACT_F16
+    forced = {"auto": snn.PATH_AUTO, "reuse": snn.PATH_REUSE, "decoded": snn.PATH_DECODED,
+              "decoded_tc": snn.PATH_DECODED_TC}[args.path]
+
+    layers, acts, outs, host_acts, host_outs, paths = [], [], [], [], [], []
+    for i, shape in enumerate(workload.layers, start=first_layer):
+        seed = wl.layer_seed(workload.config, i) + 7919 * rank
+        p = wl.draw_layer_params(shape, workload.tau, wl.layer_seed(workload.config, i))
+        layer = snn.SnnConv(shape.c_in, shape.c_out, workload.tau, p.codebook, p.idx_packed, p.alpha, shape.stride,
+                            shape.pad, act_code, device=local_rank)
+        if workload.act == "bin":
+            a = torch.from_numpy(wl.pack_activation_bits(wl.draw_activation_bits(shape, nb, seed)).view(np.int32))
+        else:
+            a = torch.from_numpy(wl.draw_activation_f16(shape, nb, seed))
+        host_acts.append(a.pin_memory())
+        acts.append(a.to(dev))
+        outs.append(layer.alloc_out(nb, shape.h, shape.w))
+        host_outs.append(layer.alloc_out(nb, shape.h, shape.w, pin=True))
+        if forced == snn.PATH_AUTO:
+            layer.tune(nb, shape.h, shape.w)
+        paths.append(layer.chosen_path(nb, shape.h, shape.w) if forced == snn.PATH_AUTO else forced)
+        layers.append(layer)
+
+    stream = torch.cuda.current_stream(dev)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)  # > 126 MB L2
+
+    def step():
+        for layer, a, o, pth in zip(layers, acts, outs, paths):
+            layer.forward(a, o, snn.OUT_F32, pth, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(max(3, args.warmup)):
+        flush.zero_()
+        step()
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = snn.kernel_launches()
+    barrier()
+    wall0 = time.perf_counter()
+    for e0, e1 in ev:
+        flush.zero_()          # L2 flush between timed iterations (outside the event pair)
+        e0.record(stream)
+        step()
+        e1.record(stream)
+    barrier()
+    wall = time.perf_counter() - wall0
+    launches = snn.kernel_launches() - launches0
+    step_ms = [e0.elapsed_time(e1) for e0, e1 in ev]
+    total_ms = float(sum(step_ms))
+
+    # per-layer device time (same launch configuration, L2 flushed before every layer)
+    reps = max(3, min(20, args.steps))
+    layer_ms = [0.0] * len(layers)
+    for _ in range(reps):
+        for j, (layer, a, o, pth) in enumerate(zip(layers, acts, outs, paths)):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            layer.forward(a, o, snn.OUT_F32, pth, stream)
+            e1.record(stream)
+            e1.synchronize()
+            layer_ms[j] += e0.elapsed_time(e1) / reps
+    clocks = sampler.stop()
+
+    # end to end through the host-buffer entry point: H2D of the inputs and D2H of the results inside the timing
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    for j, layer in enumerate(layers):
+        layer.forward_host(host_acts[j], host_outs[j], snn.OUT_F32, paths[j])
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        for j, layer in enumerate(layers):
+            layer.forward_host(host_acts[j], host_outs[j], snn.OUT_F32, paths[j])
+    torch.cuda.synchronize(dev)
+    e2e_ms = (time.perf_counter() - t0) / e2e_steps * 1e3
+    h2d = sum(a.numel() * a.element_size() for a in host_acts)
+    d2h = sum(o.numel() * o.element_size() for o in host_outs)
+
+    # max over ranks (device-timed)
+    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step = total_ms / args.steps
+    value = nb * world / (ms_per_step * 1e-3)
+    e2e_value = nb * world / (e2e_ms * 1e-3)
+
+    # ---- roofline of the dominant kernel (the path whose launches take the largest share of the step)
+    by_path = {}
+    for j, (shape, pth) in enumerate(zip(workload.layers, paths)):
+        d = by_path.setdefault(pth, {"ms": 0.0, "macs": 0, "bytes": 0, "launches": 0})
+        d["ms"] += layer_ms[j]
+        d["macs"] += shape.dense_macs(nb)
+        d["bytes"] += (shape.in_bytes_bin(nb) if workload.act == "bin" else shape.in_bytes_f16(nb)) + shape.out_bytes(nb)
+        d["launches"] += 1
+    dom = max(by_path, key=lambda k: by_path[k]["ms"])
+    d = by_path[dom]
+    sec = d["ms"] * 1e-3
+    hbm_frac = d["bytes"] / sec / 1e9 / peaks["hbm_gbs"]
+    alu_rates = {}
+    if dom == snn.PATH_DECODED_TC:
+        # dense contraction: int8 (binary activations) at twice the measured bf16 rate, fp16 at the bf16 rate
+        ratio = 2.0 if workload.act == "bin" else 1.0
+        peak = peaks["bf16_tflops_sustained"] * ratio
+        achieved = 2 * d["macs"] / sec / 1e12
+        pipe = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak}
+    elif dom == snn.PATH_DECODED:
+        # one POPC per 32 MACs; 16 POPC lanes per SM per clock on 148 SMs at the maximum SM clock
+        peak = 148 * 16 * peaks["sm_max_mhz"] * 1e6 / 1e12
+        achieved = d["macs"] / 32 / sec / 1e12
+        pipe = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Tpopc/s", "frac": achieved / peak}
+        alu_rates["popc_measured_per_s"] = snn.microbench(0, local_rank)
+    else:
+        # one 4-pixel shared-memory word per (c_out, c_in, 4 pixels); 32 words per SM per clock
+        peak = 148 * 32 * peaks["sm_max_mhz"] * 1e6 / 1e12
+        achieved = d["macs"] / 9 / 4 / sec / 1e12
+        pipe = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Tlds/s", "frac": achieved / peak}
+        alu_rates["lds_measured_per_s"] = snn.microbench(3, local_rank)
+    if hbm_frac >= pipe["frac"]:
+        roofline = {"bound": "hbm", "achieved": d["bytes"] / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": hbm_frac}
+    else:
+        roofline = pipe
+    roofline.update({"traffic": None, "kernel": snn.PATH_NAMES[dom], "launches_per_step": d["launches"],
+                     "share_of_step": d["ms"] / max(sum(layer_ms), 1e-9), "peak_source": peaks["source"],
+                     "hbm_frac": hbm_frac, "pipe_frac": pipe["frac"], **alu_rates})
+    # whole-step roofline: sum over layers of max(HBM floor, pipe floor at the path's peak)
+    step_floor_hbm_ms = workload.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e3
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32" if workload.act == "bin" else "f16", "data": "synthetic",
+        "config": {"workload": _workload_name(workload), "layers": len(layers), "batch_per_gpu": nb,
+                   "tau": workload.tau, "l2": "flushed between timed steps (256 MB write)",
+                   "paths": [snn.PATH_NAMES[p] for p in paths]},
+        "effective_tops": 2 * workload.dense_macs() * world / (ms_per_step * 1e-3) / 1e12,
+        "hbm_floor_ms_per_step": step_floor_hbm_ms,
+        "step_frac_of_hbm_floor": step_floor_hbm_ms / ms_per_step,
+        "layer_ms": [round(v, 5) for v in layer_ms],
+        "roofline": roofline,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "wall_s_timed_region": wall,
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        n_img = oracle_sample_images(workload, 15.0)
+        t_or = time_oracle_stack(workload, n_img)
+        line["cpu_baseline"] = {
+            "value": n_img / t_or, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"{n_img} of {nb} images through all {len(layers)} layers, {t_or:.1f} s",
+        }
+    elif rank == 0:
+        line["cpu_baseline"] = None
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    for layer in layers:
+        layer.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet18", choices=list(wl.WORKLOAD_NAMES))
+    ap.add_argument("--tau", type=int, default=None)
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--path", default="auto", choices=["auto", "reuse", "decoded", "decoded_tc"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", default=None, help="a:b restricts the stack to layers [a, b) (profiling aid)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
