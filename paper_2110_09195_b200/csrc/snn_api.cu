@@ -225,6 +225,7 @@ snn_status_t snn_conv_create(const snn_conv_desc_t* d, snn_conv_t** out) {
   if (e == cudaSuccess) e = cudaMemcpyAsync(h->L.alpha, d->alpha, (size_t)h->K * 4, cudaMemcpyHostToDevice, s);
   int launched = 0;
   if (e == cudaSuccess) e = decode_layer(h->L, d_stream, g, h->act_type, s, &launched);
+  if (e == cudaSuccess && tcw) e = tc_expand_weights(h->L, g, h->act_type, s, &launched);
   g_launches += launched;
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (d_stream) cudaFree(d_stream);

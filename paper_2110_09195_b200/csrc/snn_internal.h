@@ -54,6 +54,7 @@ bool tc_supported(const Geom& g, int act_type);
 cudaError_t tc_forward(const LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched,
                        int* dev_status_host);
 size_t tc_weight_bytes(const Geom& g, int act_type, int* Kpad, int* Cpad);
+cudaError_t tc_expand_weights(const LayerDev& L, const Geom& g, int act_type, cudaStream_t s, int* launched);
 
 cudaError_t microbench(int kind, double* rate);
 

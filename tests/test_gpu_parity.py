@@ -155,3 +155,53 @@ def test_deterministic_and_host_entry(snn, oracle_mod):
     assert layer.chosen_path(4, 14, 14) == best and ms[best] > 0
     assert (layer.forward(act).cpu().numpy() == y_ref).all()
     layer.destroy()
+
+
+def check_f16_layer(snn, oracle_mod, shape, tau, n, seed):
+    p = wl.draw_layer_params(shape, tau, seed)
+    act_np = wl.draw_activation_f16(shape, n, seed)
+    y_ref = oracle_mod.conv_f16(p.codebook, tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out, shape.stride,
+                                shape.pad, act_np)
+    layer = snn.SnnConv(shape.c_in, shape.c_out, tau, p.codebook, p.idx_packed, p.alpha, shape.stride, shape.pad,
+                        snn.ACT_F16)
+    act = torch.from_numpy(act_np).cuda()
+    ran = []
+    for path in _paths(layer, n, shape.h, shape.w):
+        flat_y, out_y = _guarded(y_ref.shape, torch.float32)
+        layer.forward(act, out_y, snn.OUT_F32, path)
+        torch.cuda.synchronize()
+        y = out_y.cpu().numpy()
+        assert _canaries_intact(flat_y, y_ref.size)
+        sigma = p.alpha.astype(np.float64) * np.sqrt(9.0 * shape.c_in)
+        bound = REL_F16 * np.maximum(np.abs(y_ref.astype(np.float64)), sigma[None, None, None, :])
+        err = np.abs(y.astype(np.float64) - y_ref.astype(np.float64))
+        assert (err <= bound).all(), f"path {snn.PATH_NAMES[path]}: max err/bound {np.max(err / bound)}"
+        # the accumulation is fp32 over exact products: the norm-wise error is far inside the bound
+        assert np.linalg.norm(err) <= 1e-4 * np.linalg.norm(y_ref)
+        ran.append(path)
+    layer.destroy()
+    return ran
+
+
+@pytest.mark.parametrize("c_in,c_out,h,w,stride,pad,tau,n", [
+    (16, 16, 32, 32, 1, 1, 5, 1),
+    (64, 64, 14, 14, 1, 1, 5, 2),
+    (64, 128, 14, 14, 2, 1, 5, 2),
+    (40, 24, 9, 7, 1, 0, 4, 2),
+    (33, 7, 6, 5, 2, 1, 3, 2),       # c_in not a multiple of 8: scalar staging
+    (256, 256, 7, 7, 1, 1, 5, 1),
+])
+def test_f16_activation_variant(snn, oracle_mod, c_in, c_out, h, w, stride, pad, tau, n):
+    shape = wl.LayerShape(c_in, c_out, h, w, stride, pad)
+    ran = check_f16_layer(snn, oracle_mod, shape, tau, n, 2000 + c_in + c_out)
+    assert len(ran) >= 2  # at least one named path plus AUTO
+
+
+def test_tensor_core_path_runs_the_stack_shapes(snn):
+    """The tcgen05 path must cover every ResNet-18/34 layer shape at the benchmark batch."""
+    wk = wl.get_workload("resnet18")
+    for shape in set(wk.layers):
+        p = wl.draw_layer_params(shape, 5, 1)
+        layer = snn.SnnConv(shape.c_in, shape.c_out, 5, p.codebook, p.idx_packed, p.alpha, shape.stride, shape.pad)
+        assert layer.path_supported(snn.PATH_DECODED_TC, wk.batch, shape.h, shape.w)
+        layer.destroy()
