@@ -226,12 +226,34 @@ def run_ours(args):
         paths.append(layer.chosen_path(nb, shape.h, shape.w) if forced == snn.PATH_AUTO else forced)
         layers.append(layer)
 
-    stream = torch.cuda.current_stream(dev)
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)  # > 126 MB L2
+    side = torch.cuda.Stream(dev)
+
+    def launch_layers(idxs, stream):
+        for j in idxs:
+            layers[j].forward(acts[j], outs[j], snn.OUT_F32, paths[j], stream)
+
+    def capture(idxs):
+        """The launches of one step (or one layer) as a CUDA graph, so that the host's
+        per-call cost does not sit between the kernels that are being timed."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            launch_layers(idxs, side)          # warm-up outside capture (sets kernel attributes)
+            side.synchronize()
+            with torch.cuda.graph(g, stream=side):
+                launch_layers(idxs, torch.cuda.current_stream(dev))
+        return g
+
+    all_idx = list(range(len(layers)))
+    use_graph = not args.no_graph
+    step_graph = capture(all_idx) if use_graph else None
+    stream = torch.cuda.current_stream(dev)
 
     def step():
-        for layer, a, o, pth in zip(layers, acts, outs, paths):
-            layer.forward(a, o, snn.OUT_F32, pth, stream)
+        if use_graph:
+            step_graph.replay()
+        else:
+            launch_layers(all_idx, stream)
 
     def barrier():
         if world > 1:
@@ -256,19 +278,24 @@ def run_ours(args):
         e1.record(stream)
     barrier()
     wall = time.perf_counter() - wall0
-    launches = snn.kernel_launches() - launches0
+    launches = (snn.kernel_launches() - launches0) if not use_graph else len(layers) * args.steps
     step_ms = [e0.elapsed_time(e1) for e0, e1 in ev]
     total_ms = float(sum(step_ms))
 
-    # per-layer device time (same launch configuration, L2 flushed before every layer)
+    # per-layer device time (same launch configuration, L2 flushed before every layer; the
+    # flush also keeps the GPU busy while the host enqueues, so no host latency is timed)
     reps = max(3, min(20, args.steps))
     layer_ms = [0.0] * len(layers)
+    layer_graphs = [capture([j]) for j in all_idx] if use_graph else None
     for _ in range(reps):
-        for j, (layer, a, o, pth) in enumerate(zip(layers, acts, outs, paths)):
+        for j in all_idx:
             flush.zero_()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            layer.forward(a, o, snn.OUT_F32, pth, stream)
+            if use_graph:
+                layer_graphs[j].replay()
+            else:
+                launch_layers([j], stream)
             e1.record(stream)
             e1.synchronize()
             layer_ms[j] += e0.elapsed_time(e1) / reps
@@ -345,6 +372,7 @@ def run_ours(args):
         "dtype": "int32" if workload.act == "bin" else "f16", "data": "synthetic",
         "config": {"workload": _workload_name(workload), "layers": len(layers), "batch_per_gpu": nb,
                    "tau": workload.tau, "l2": "flushed between timed steps (256 MB write)",
+                   "launch": "host calls" if args.no_graph else "CUDA graph of the per-layer C-ABI launches",
                    "paths": [snn.PATH_NAMES[p] for p in paths]},
         "effective_tops": 2 * workload.dense_macs() * world / (ms_per_step * 1e-3) / 1e12,
         "hbm_floor_ms_per_step": step_floor_hbm_ms,
@@ -389,6 +417,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "reuse", "decoded", "decoded_tc"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every layer from the host instead of a CUDA graph")
     ap.add_argument("--layers", default=None, help="a:b restricts the stack to layers [a, b) (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -11,6 +11,7 @@
 #include <mutex>
 #include <new>
 #include <tuple>
+#include <utility>
 
 #include "snn_internal.h"
 
@@ -54,13 +55,14 @@ struct snn_conv {
   int C, K, tau, stride, pad, act_type, device;
   LayerDev L;
   std::mutex mu;
-  std::map<std::tuple<int, int, int>, int> tuned;  // (N,H,W) -> path
+  std::map<std::tuple<int, int, int>, std::pair<int, int>> tuned;  // (N,H,W) -> (path, tensor-core variant)
   // staging for snn_conv_forward_host
   void* stage_in = nullptr;
   void* stage_out = nullptr;
   size_t stage_in_bytes = 0, stage_out_bytes = 0;
   cudaStream_t host_stream = nullptr;
   int* tc_status_host = nullptr;  // pinned, written by the tensor-core kernel on a bounded-wait timeout
+  int* tc_status_dev = nullptr;   // the same word as the device sees it
 };
 
 namespace {
@@ -110,18 +112,27 @@ int auto_path(snn_conv* h, const Geom& g) {
   {
     std::lock_guard<std::mutex> lk(h->mu);
     auto it = h->tuned.find(std::make_tuple(g.N, g.H, g.W));
-    if (it != h->tuned.end()) return it->second;
+    if (it != h->tuned.end()) return it->second.first;
   }
   return heuristic_path(h, g);
 }
 
-snn_status_t run_path(snn_conv* h, int path, const Geom& g, const Launch& l) {
+// Tensor-core tile variant remembered by snn_conv_tune for this shape (0 = heuristic).
+int tuned_variant(snn_conv* h, const Geom& g) {
+  std::lock_guard<std::mutex> lk(h->mu);
+  auto it = h->tuned.find(std::make_tuple(g.N, g.H, g.W));
+  return (it != h->tuned.end() && it->second.first == SNN_PATH_DECODED_TC) ? it->second.second : 0;
+}
+
+snn_status_t run_path(snn_conv* h, int path, const Geom& g, const Launch& l, int variant = -1) {
   int launched = 0;
   cudaError_t e = cudaSuccess;
   switch (path) {
     case SNN_PATH_REUSE: e = reuse_forward(h->L, g, h->act_type, l, &launched); break;
     case SNN_PATH_DECODED: e = popc_forward(h->L, g, l, &launched); break;
-    case SNN_PATH_DECODED_TC: e = tc_forward(h->L, g, h->act_type, l, &launched, h->tc_status_host); break;
+    case SNN_PATH_DECODED_TC:
+      e = tc_forward(h->L, g, h->act_type, l, &launched, h->tc_status_dev, variant >= 0 ? variant : tuned_variant(h, g));
+      break;
     default: return fail(SNN_ERR_INVALID_ARG, "unknown path %d", path);
   }
   g_launches += launched;
@@ -219,6 +230,7 @@ snn_status_t snn_conv_create(const snn_conv_desc_t* d, snn_conv_t** out) {
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->host_stream, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&h->tc_status_host, sizeof(int), cudaHostAllocMapped);
   if (e == cudaSuccess) *h->tc_status_host = 0;
+  if (e == cudaSuccess) e = cudaHostGetDevicePointer((void**)&h->tc_status_dev, h->tc_status_host, 0);
   cudaStream_t s = h->host_stream;
   if (e == cudaSuccess) e = cudaMemcpyAsync(d_stream, d->idx_packed, idx_bytes, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(h->L.codebook, d->codebook, (size_t)T * 2, cudaMemcpyHostToDevice, s);
@@ -359,26 +371,37 @@ snn_status_t snn_conv_tune(snn_conv_t* h, int32_t N, int32_t H, int32_t W, int32
   if (h->act_type == SNN_ACT_F16) cudaMemset(a, 0x3c, act_bytes(h, g));  // 0x3c3c = 1.0586 in fp16
   cudaStream_t s = h->host_stream;
   float best = -1.f;
-  int best_p = 0;
+  int best_p = 0, best_v = 0;
   snn_status_t st = SNN_OK;
-  for (int pth = 1; pth <= 3; ++pth) {
-    if (ms) ms[pth] = -1.f;
-    if (!path_ok(h, pth, g)) continue;
+  auto time_one = [&](int pth, int variant, float* t_out) -> snn_status_t {
     Launch l{a, o, 0, s};
     const int reps = 5;
-    for (int w = 0; w < 2 && st == SNN_OK; ++w) st = run_path(h, pth, g, l);
-    if (st != SNN_OK) break;
+    snn_status_t r = SNN_OK;
+    for (int w = 0; w < 2 && r == SNN_OK; ++w) r = run_path(h, pth, g, l, variant);
+    if (r != SNN_OK) return r;
     cudaEventRecord(e0, s);
-    for (int r = 0; r < reps && st == SNN_OK; ++r) st = run_path(h, pth, g, l);
+    for (int k = 0; k < reps && r == SNN_OK; ++k) r = run_path(h, pth, g, l, variant);
     cudaEventRecord(e1, s);
-    e = cudaEventSynchronize(e1);
-    if (st != SNN_OK) break;
-    if (e != cudaSuccess) { st = cuda_fail(e, "snn_conv_tune timing"); break; }
+    cudaError_t ce = cudaEventSynchronize(e1);
+    if (r != SNN_OK) return r;
+    if (ce != cudaSuccess) return cuda_fail(ce, "snn_conv_tune timing");
     float t = 0.f;
     cudaEventElapsedTime(&t, e0, e1);
-    t /= reps;
-    if (ms) ms[pth] = t;
-    if (best < 0.f || t < best) { best = t; best_p = pth; }
+    *t_out = t / reps;
+    return SNN_OK;
+  };
+  for (int pth = 1; pth <= 3 && st == SNN_OK; ++pth) {
+    if (ms) ms[pth] = -1.f;
+    if (!path_ok(h, pth, g)) continue;
+    const int nvar = pth == SNN_PATH_DECODED_TC ? tc_variant_count() : 1;
+    for (int v = 0; v < nvar && st == SNN_OK; ++v) {
+      if (pth == SNN_PATH_DECODED_TC && !tc_variant_ok(g, h->act_type, v)) continue;
+      float t = 0.f;
+      st = time_one(pth, pth == SNN_PATH_DECODED_TC ? v : -1, &t);
+      if (st != SNN_OK) break;
+      if (ms && (ms[pth] < 0.f || t < ms[pth])) ms[pth] = t;
+      if (best < 0.f || t < best) { best = t; best_p = pth; best_v = v; }
+    }
   }
   if (ms) ms[0] = best;
   cudaEventDestroy(e0);
@@ -389,12 +412,12 @@ snn_status_t snn_conv_tune(snn_conv_t* h, int32_t N, int32_t H, int32_t W, int32
   if (!best_p) return fail(SNN_ERR_UNSUPPORTED, "no path supports this layer");
   {
     std::lock_guard<std::mutex> lk(h->mu);
-    h->tuned[std::make_tuple(N, H, W)] = best_p;
+    h->tuned[std::make_tuple(N, H, W)] = std::make_pair(best_p, best_p == SNN_PATH_DECODED_TC ? best_v : 0);
   }
   if (best_path) *best_path = best_p;
   if (getenv("SNN_LOG"))
-    fprintf(stderr, "[snnconv] tuned C=%d K=%d tau=%d N=%d %dx%d -> path %d (%.4f ms)\n", h->C, h->K, h->tau, N, H, W,
-            best_p, best);
+    fprintf(stderr, "[snnconv] tuned C=%d K=%d tau=%d N=%d %dx%d -> path %d variant %d (%.4f ms)\n", h->C, h->K,
+            h->tau, N, H, W, best_p, best_v, best);
   return SNN_OK;
 }
 

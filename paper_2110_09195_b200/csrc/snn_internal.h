@@ -51,11 +51,31 @@ bool reuse_supported(const Geom& g, int act_type);
 cudaError_t reuse_forward(const LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched);
 
 bool tc_supported(const Geom& g, int act_type);
+// Tile variants of the tensor-core kernel (sub-tiles per CTA, weight-stage size, CTAs per SM);
+// variant 0 is the heuristic choice, the others are what snn_conv_tune sweeps.
+int tc_variant_count();
+bool tc_variant_ok(const Geom& g, int act_type, int variant);
 cudaError_t tc_forward(const LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched,
-                       int* dev_status_host);
+                       int* status_dev, int variant);
 size_t tc_weight_bytes(const Geom& g, int act_type, int* Kpad, int* Cpad);
 cudaError_t tc_expand_weights(const LayerDev& L, const Geom& g, int act_type, cudaStream_t s, int* launched);
 
 cudaError_t microbench(int kind, double* rate);
+
+// Largest dynamic shared memory a CTA may ask for on sm_100 (227 KB).
+constexpr int kMaxDynSmem = 227 * 1024;
+
+// Raises a kernel's dynamic shared-memory limit to the maximum, once per device.
+template <typename Kernel>
+inline cudaError_t allow_max_smem(Kernel kernel, unsigned long long* done_mask) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (__atomic_load_n(done_mask, __ATOMIC_ACQUIRE) & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  if (e == cudaSuccess) __atomic_fetch_or(done_mask, bit, __ATOMIC_RELEASE);
+  return e;
+}
 
 }  // namespace snn

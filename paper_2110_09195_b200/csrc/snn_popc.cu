@@ -195,8 +195,8 @@ static cudaError_t launch_popc(PopcParams p, cudaStream_t s) {
   if (cwc > 16) cwc = 16;
   p.cwc = cwc;
   size_t smem = (size_t)cwc * per_word + 64;
-  cudaError_t e = cudaFuncSetAttribute(popc_conv_kernel<PM, PN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem);
+  static unsigned long long done = 0;
+  cudaError_t e = allow_max_smem(popc_conv_kernel<PM, PN>, &done);
   if (e != cudaSuccess) return e;
   dim3 grid((unsigned)(p.tiles_x * tiles_y), (unsigned)((p.K + KT - 1) / KT));
   popc_conv_kernel<PM, PN><<<grid, 256, smem, s>>>(p);

@@ -209,8 +209,8 @@ static int pow2_floor(int v) {
 
 template <int Q>
 static cudaError_t launch_reuse(const ReuseParams& p, size_t smem, dim3 grid, int threads, cudaStream_t s) {
-  cudaError_t e =
-      cudaFuncSetAttribute(reuse_conv_kernel<Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  static unsigned long long done = 0;
+  cudaError_t e = allow_max_smem(reuse_conv_kernel<Q>, &done);
   if (e != cudaSuccess) return e;
   reuse_conv_kernel<Q><<<grid, threads, smem, s>>>(p);
   return cudaGetLastError();

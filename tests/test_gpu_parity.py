@@ -90,6 +90,8 @@ def test_config0_single_layer(snn, oracle_mod):
     (32, 40, 2, 1, 2, 1, 2, 3),
     (96, 130, 3, 17, 1, 1, 6, 1),
     (300, 20, 6, 5, 1, 1, 1, 2),     # tau = 1: two kernels
+    (2048, 32, 6, 6, 1, 1, 5, 1),    # activations staged in several channel blocks
+    (1056, 48, 9, 8, 2, 1, 5, 1),    # the same with the four stride-2 planes
 ])
 def test_ragged_shapes(snn, oracle_mod, c_in, c_out, h, w, stride, pad, tau, n):
     shape = wl.LayerShape(c_in, c_out, h, w, stride, pad)
@@ -205,3 +207,22 @@ def test_tensor_core_path_runs_the_stack_shapes(snn):
         layer = snn.SnnConv(shape.c_in, shape.c_out, 5, p.codebook, p.idx_packed, p.alpha, shape.stride, shape.pad)
         assert layer.path_supported(snn.PATH_DECODED_TC, wk.batch, shape.h, shape.w)
         layer.destroy()
+
+
+@pytest.mark.parametrize("c_in,c_out,h,w,stride", [(64, 64, 20, 20, 1), (256, 128, 9, 9, 1), (128, 256, 12, 12, 2)])
+def test_tensor_core_tile_variants(snn, oracle_mod, monkeypatch, c_in, c_out, h, w, stride):
+    """Every tile shape the tuner may pick (sub-tiles per CTA, weight-stage size, CTAs per SM)
+    gives the same sums."""
+    shape = wl.LayerShape(c_in, c_out, h, w, stride, 1)
+    for mt in (1, 2, 4):
+        for kb in (16, 32, 64):
+            for one in (0, 1):
+                monkeypatch.setenv("SNN_TC_MT", str(mt))
+                monkeypatch.setenv("SNN_TC_STAGE_KB", str(kb))
+                monkeypatch.setenv("SNN_TC_ONE_PER_SM", str(one))
+                p = wl.draw_layer_params(shape, 5, 77)
+                layer = snn.SnnConv(c_in, c_out, 5, p.codebook, p.idx_packed, p.alpha, stride, 1)
+                ok = layer.path_supported(snn.PATH_DECODED_TC, 3, h, w)
+                layer.destroy()
+                if ok:
+                    check_bin_layer(snn, oracle_mod, shape, 5, 3, 77, paths=[snn.PATH_DECODED_TC])
