@@ -138,6 +138,42 @@ SNN_API int64_t snn_kernel_launches(void);
  */
 SNN_API snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate);
 
+/*
+ * Forward pass for callers that must not allocate device memory.  (The paper has
+ * no counterpart to this entry point; it exists for how the library is embedded.)
+ *
+ * Some hosts cannot let a library call cudaMalloc: an application that has handed
+ * the whole device to its own memory pool, a process whose memory budget is fixed
+ * at start-up, or a latency-bound loop that cannot afford the device-wide
+ * synchronisation an allocation may bring.  snn_conv_create allocates, so such
+ * callers use this call instead: it takes the layer as the descriptor states it
+ * (HOST arrays, as for snn_conv_create) together with the DEVICE activation and
+ * output buffers, and does everything else - copy of the layer, decode, XOR +
+ * popcount convolution - inside one fixed device array that is part of the
+ * library image (SNN_STATIC_SCRATCH_BYTES on every GPU that loads the library,
+ * held until the process exits).  It calls no cudaMalloc / cudaFree and no
+ * allocating library routine.
+ *
+ * Limits: binary activations only; c_in and c_out at most SNN_STATIC_MAX_CHANNELS
+ * (a 512 x 512 layer with any tau fits); a layer whose scratch need exceeds the
+ * array is refused with SNN_ERR_UNSUPPORTED and a message that names both sizes.
+ * Layouts, output types and argument errors are those of snn_conv_forward; the
+ * work is asynchronous on cuda_stream once the host arrays have been handed to
+ * the copy engine (keep them alive and unchanged until the stream has passed them
+ * unless they are pageable memory, which the runtime stages before returning).
+ *
+ * The first call on a device resolves the device address of the array
+ * (cudaGetSymbolAddress); make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's
+ * contents: each call rewrites in full every region it reads, so results never
+ * depend on an earlier call, but two calls whose GPU work overlaps (different
+ * streams, or threads) race on it.  Serialise them.
+ */
+#define SNN_STATIC_SCRATCH_BYTES (1536 * 1024)
+#define SNN_STATIC_MAX_CHANNELS 512
+SNN_API snn_status_t snn_conv_forward_static(const snn_conv_desc_t* desc, const void* act_dev, int32_t N, int32_t H,
+                                             int32_t W, void* out_dev, int32_t out_type, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

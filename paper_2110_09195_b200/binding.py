@@ -25,7 +25,7 @@ _lib = None
 EXPORTED_SYMBOLS = (
     "snn_conv_create", "snn_conv_forward", "snn_conv_forward_host", "snn_conv_tune", "snn_conv_chosen_path",
     "snn_conv_path_supported", "snn_conv_destroy", "snn_last_error", "snn_version", "snn_kernel_launches",
-    "snn_microbench",
+    "snn_microbench", "snn_conv_forward_static",
 )
 
 
@@ -80,6 +80,8 @@ def load_library():
     lib.snn_version.argtypes = []
     lib.snn_kernel_launches.restype = ctypes.c_int64
     lib.snn_kernel_launches.argtypes = []
+    lib.snn_conv_forward_static.restype = i32
+    lib.snn_conv_forward_static.argtypes = [ctypes.POINTER(_Desc), vp, i32, i32, i32, vp, i32, vp]
     lib.snn_microbench.restype = i32
     lib.snn_microbench.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double)]
     _lib = lib
@@ -103,6 +105,36 @@ def microbench(kind: int, device: int = 0) -> float:
     rate = ctypes.c_double(0.0)
     _check(load_library().snn_microbench(kind, device, ctypes.byref(rate)))
     return float(rate.value)
+
+
+def forward_static(c_in, c_out, tau, codebook, idx_packed, alpha, act, out, stride=1, pad=1, out_type=OUT_F32,
+                   device=0, stream=None):
+    """snn_conv_forward_static: one forward pass without any device allocation by the library.
+
+    For hosts that cannot let a library allocate (a device handed over to the
+    application's own pool, a fixed memory budget, a loop that cannot take an
+    allocation's synchronisation).  The layer is given as host arrays each time;
+    `act` and `out` are CUDA tensors the caller already owns.  Binary activations
+    only, at most 512 channels in and out.  Calls share one fixed scratch array
+    per GPU, so do not let two of them overlap on the device."""
+    import torch
+    cb = np.ascontiguousarray(codebook, dtype=np.uint16)
+    ip = np.ascontiguousarray(idx_packed, dtype=np.uint8)
+    al = np.ascontiguousarray(alpha, dtype=np.float32)
+    if not 1 <= int(tau) <= 9 or cb.size != (1 << int(tau)):
+        raise SnnError(1, "tau outside 1..9 or codebook of the wrong size")
+    if ip.size < (int(c_out) * int(c_in) * int(tau) + 7) // 8 or al.size != int(c_out):
+        raise SnnError(1, "index stream or alpha of the wrong size")
+    if not (act.is_cuda and out.is_cuda and act.is_contiguous() and out.is_contiguous()):
+        raise SnnError(1, "act and out must be contiguous CUDA tensors")
+    n, h, w = int(act.shape[0]), int(act.shape[1]), int(act.shape[2])
+    d = _Desc(int(c_in), int(c_out), int(tau), int(stride), int(pad), ACT_BIN, int(device),
+              cb.ctypes.data, ip.ctypes.data, al.ctypes.data)
+    if stream is None:
+        stream = torch.cuda.current_stream(device)
+    _check(load_library().snn_conv_forward_static(ctypes.byref(d), act.data_ptr(), n, h, w, out.data_ptr(),
+                                                  int(out_type), ctypes.c_void_p(stream.cuda_stream)))
+    return out
 
 
 class SnnConv:

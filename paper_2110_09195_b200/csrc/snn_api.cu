@@ -169,6 +169,19 @@ size_t out_bytes(const Geom& g) { return (size_t)g.N * g.Ho * g.Wo * g.K * 4; }
 
 }  // namespace
 
+namespace snn {
+// used by snn_static.cu
+snn_status_t api_fail(snn_status_t st, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  if (getenv("SNN_LOG")) fprintf(stderr, "[snnconv] error %d: %s\n", (int)st, g_err);
+  return st;
+}
+void api_count_launches(int n) { g_launches += n; }
+}  // namespace snn
+
 extern "C" {
 
 const char* snn_last_error(void) { return g_err; }
