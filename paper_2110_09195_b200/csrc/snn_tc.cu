@@ -314,6 +314,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
     mbar_init(bar_afree, 1);
     mbar_init(bar_accum, 1);
     *abort_flag = 0;
+    wait_flags[0] = wait_flags[1] = wait_flags[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
