@@ -336,8 +336,6 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
                (uint32_t)((ky >> 1) * p.Wq + (kx >> 1));
       seg_units[e] = u + (uint32_t)(seg * p.st_k * 2) * (uint32_t)p.Rr;
     }
-    for (int c = tid; c < 256; c += TC_THREADS)
-      alpha_s[c] = (c < p.Nt && n0 + c < p.K) ? __ldg(p.alpha + n0 + c) : 0.f;
   }
   tc_fence_before();
   __syncthreads();
@@ -461,6 +459,9 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
     accum_release();  // lets the workers into the epilogue
   } else {
     // ------------------------------------------------ workers: expand activations, then epilogue
+    // this CTA's scales: requested now, parked in shared memory after the expansion (the
+    // epilogue reads them behind the accumulator barrier), so their latency is hidden
+    const float my_alpha = (tid < p.Nt && n0 + tid < p.K) ? __ldg(p.alpha + n0 + tid) : 0.f;
     for (int cb = 0; cb < p.n_cb; ++cb) {
       if (cb > 0) {
         // one elected thread polls; the rest wait on a hardware barrier instead of spinning
@@ -475,10 +476,10 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
         for (int pl = 0; pl < p.n_planes; ++pl) {
           const int pa = pl >> 1, pb = pl & 1;
           uint8_t* a_plane = a_smem + (size_t)pl * plane_bytes;
+          if (F16) {
 #pragma unroll 2
-          for (int r = tid; r < p.Rr; r += TC_WORKERS) {
-            const int pix = position_to_pixel(p, Q0 + (uint32_t)r, pa, pb);
-            if (F16) {
+            for (int r = tid; r < p.Rr; r += TC_WORKERS) {
+              const int pix = position_to_pixel(p, Q0 + (uint32_t)r, pa, pb);
               const int ch0 = cb * p.cb_chunks * 8;
               const __half* src = (const __half*)p.act + (size_t)(pix < 0 ? 0 : pix) * p.C + ch0;
               const bool vec = pix >= 0 && ((p.C & 7) == 0);
@@ -496,28 +497,56 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
                 }
                 *reinterpret_cast<uint4*>(a_plane + ((size_t)c * p.Rr + r) * 16) = v;
               }
-            } else {
-              const int w0 = cb * (p.cb_chunks / 2), nw = p.cb_chunks / 2;
-              const uint32_t* src = (const uint32_t*)p.act + (size_t)(pix < 0 ? 0 : pix) * p.Cw + w0;
-              const bool present = pix >= 0;
-              const bool vec4 = present && ((p.Cw & 3) == 0);
-              for (int w = 0; w < nw; w += 4) {
-                uint32_t bits[4] = {0, 0, 0, 0};
-                if (vec4 && ((w0 + w) & 3) == 0 && w0 + w + 4 <= p.Cw) {
-                  const uint4 b4 = __ldg(reinterpret_cast<const uint4*>(src + w));
-                  bits[0] = b4.x; bits[1] = b4.y; bits[2] = b4.z; bits[3] = b4.w;
-                } else if (present) {
+            }
+          } else {
+            // two rows and up to eight 32-channel words per row are requested before any is
+            // expanded, so a thread has its global loads in flight together
+            const int nw = p.cb_chunks / 2, w0 = cb * nw;
+            const bool vec_ok = (p.Cw & 3) == 0 && (w0 & 3) == 0;
+            for (int rb = tid; rb < p.Rr; rb += 2 * TC_WORKERS) {
+              const int r1 = rb + TC_WORKERS;
+              const bool has1 = r1 < p.Rr;
+              const int pix0 = position_to_pixel(p, Q0 + (uint32_t)rb, pa, pb);
+              const int pix1 = has1 ? position_to_pixel(p, Q0 + (uint32_t)r1, pa, pb) : -1;
+              const uint32_t* s0 = (const uint32_t*)p.act + (size_t)(pix0 < 0 ? 0 : pix0) * p.Cw + w0;
+              const uint32_t* s1 = (const uint32_t*)p.act + (size_t)(pix1 < 0 ? 0 : pix1) * p.Cw + w0;
+              for (int wb = 0; wb < nw; wb += 8) {
+                uint32_t b0[8], b1[8];
 #pragma unroll
-                  for (int k = 0; k < 4; ++k)
-                    if (w0 + w + k < p.Cw && w + k < nw) bits[k] = __ldg(src + w + k);
+                for (int k = 0; k < 8; ++k) b0[k] = b1[k] = 0;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                  const int wq = wb + 4 * h;
+                  if (vec_ok && w0 + wq + 4 <= p.Cw && wq + 4 <= nw) {
+                    if (pix0 >= 0) {
+                      const uint4 t = __ldg(reinterpret_cast<const uint4*>(s0 + wq));
+                      b0[4 * h] = t.x; b0[4 * h + 1] = t.y; b0[4 * h + 2] = t.z; b0[4 * h + 3] = t.w;
+                    }
+                    if (pix1 >= 0) {
+                      const uint4 t = __ldg(reinterpret_cast<const uint4*>(s1 + wq));
+                      b1[4 * h] = t.x; b1[4 * h + 1] = t.y; b1[4 * h + 2] = t.z; b1[4 * h + 3] = t.w;
+                    }
+                  } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                      if (wq + k < nw && w0 + wq + k < p.Cw) {
+                        if (pix0 >= 0) b0[4 * h + k] = __ldg(s0 + wq + k);
+                        if (pix1 >= 0) b1[4 * h + k] = __ldg(s1 + wq + k);
+                      }
+                    }
+                  }
                 }
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  if (w + k < nw) {
-                    const int wg = w0 + w + k;
-                    expand_word(bits[k], p.C - wg * 32, present && wg < p.Cw,
-                                a_plane + ((size_t)(2 * (w + k)) * p.Rr + r) * 16,
-                                a_plane + ((size_t)(2 * (w + k) + 1) * p.Rr + r) * 16);
+                for (int k = 0; k < 8; ++k) {
+                  if (wb + k < nw) {
+                    const int wg = w0 + wb + k;
+                    expand_word(b0[k], p.C - wg * 32, pix0 >= 0 && wg < p.Cw,
+                                a_plane + ((size_t)(2 * (wb + k)) * p.Rr + rb) * 16,
+                                a_plane + ((size_t)(2 * (wb + k) + 1) * p.Rr + rb) * 16);
+                    if (has1)
+                      expand_word(b1[k], p.C - wg * 32, pix1 >= 0 && wg < p.Cw,
+                                  a_plane + ((size_t)(2 * (wb + k)) * p.Rr + r1) * 16,
+                                  a_plane + ((size_t)(2 * (wb + k) + 1) * p.Rr + r1) * 16);
                   }
                 }
               }
@@ -529,6 +558,7 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
       mbar_arrive(bar_aready);
     }
 
+    alpha_s[tid] = my_alpha;
     // ---- epilogue: row m of sub-tile mt lives in TMEM lane m, columns mt*Nt ..
     accum_wait();               // released by the MMA warp when the accumulators are complete
     tc_fence_after();
