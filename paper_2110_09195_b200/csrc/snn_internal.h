@@ -28,6 +28,8 @@ struct LayerDev {
   uint8_t* match9 = nullptr;     // [T/16 or 1][512][16] matching-tap counts per (window, codebook kernel)
   int8_t* w8 = nullptr;          // tensor-core operand: +/-1 int8 weights, tiled (snn_tc.cu)
   uint16_t* w16 = nullptr;       // tensor-core operand: +/-1 fp16 weights, tiled (fp16 activations)
+  void* tc_scratch = nullptr;    // expanded activations of the tensor-core path (grows on demand)
+  size_t tc_scratch_bytes = 0;
   int Kpad = 0;                  // K rounded up for the tensor-core tiling
   int Cpad = 0;                  // C rounded up for the tensor-core tiling
 };
@@ -55,8 +57,8 @@ bool tc_supported(const Geom& g, int act_type);
 // variant 0 is the heuristic choice, the others are what snn_conv_tune sweeps.
 int tc_variant_count();
 bool tc_variant_ok(const Geom& g, int act_type, int variant);
-cudaError_t tc_forward(const LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched,
-                       int* status_dev, int variant);
+cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched, int* status_dev,
+                       int variant);
 size_t tc_weight_bytes(const Geom& g, int act_type, int* Kpad, int* Cpad);
 cudaError_t tc_expand_weights(const LayerDev& L, const Geom& g, int act_type, cudaStream_t s, int* launched);
 

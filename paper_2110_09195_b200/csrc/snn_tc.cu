@@ -6,28 +6,37 @@
 //   M = 128 consecutive positions of a padded, flattened copy of the input,
 //   N = a tile of output channels, K = (tap, input channel).
 //
-// Implicit im2col without copies.  The input tile is expanded once into shared
-// memory as [16-byte channel chunk][position][16 B], the K-major layout without
-// swizzle in which consecutive rows are 16 bytes apart.  The A operand of tap
-// (ky, kx) is then the same buffer read from a start address shifted by
-// ky*pitch + kx rows, so the nine taps reuse one staged tile.  The flattened
-// space keeps one zero column per row and one zero row per image (shared by
-// neighbours), which makes zero padding literal zeros (a zero byte contributes
-// 0, as the definition requires; no border correction is needed here).
-// Stride 2 splits the padded input into its four row/column parity planes, in
-// each of which the taps are again plain shifts.
+// Two kernels per forward call.
 //
-// Per CTA (320 threads): warps 0-7 expand activations and later run the
-// epilogue (TMEM -> registers -> shared-memory transposition -> alpha scale ->
-// 128-byte row stores), one thread of warp 8 issues the MMAs, one thread of
-// warp 9 streams weight stages with bulk async copies through an mbarrier ring.
-// Measured on B200 and shaping this code: a thread alone on its warp retires
-// roughly one instruction per 5-8 cycles and pays ~200 cycles per mbarrier
-// wait, so the issuing thread runs straight-line code over large stages from
-// offsets tabulated by the other threads; threads that wait do so on hardware
-// barriers, not by polling, because pollers crowd the issuing threads.
-// Every wait is bounded; a wait that runs out raises a status word the host
-// reads, and the CTA still frees its TMEM and returns.
+// 1. tc_expand_act_kernel writes the activations once, as tensor-core operands,
+//    into a scratch buffer the layer handle owns:  xa[plane][16-byte channel
+//    chunk][position][16 B]  (bits -> +1/-1 bytes, or fp16 copied), over a
+//    padded, flattened position space that keeps one zero column per row and
+//    one zero row per image (shared by neighbours), so that zero padding is a
+//    literal zero operand (a zero contributes 0, as the definition requires).
+//    Stride 2 splits the padded input into its four row/column parity planes.
+//
+// 2. tc_conv_kernel is a persistent, warp-specialised GEMM.  Because a chunk's
+//    positions are contiguous in xa, the A operand of a tile is a handful of
+//    plain bulk copies into shared memory in the K-major, no-swizzle layout
+//    (rows 16 bytes apart), and the A operand of tap (ky, kx) is the same
+//    shared-memory block read from a start address shifted by ky*pitch + kx
+//    rows: the nine taps reuse one staged tile, there is no im2col copy.
+//      warp 0      one thread streams A units and weight stages (cp.async.bulk
+//                  onto mbarriers; rings of NA units and NS stages)
+//      warp 1      one thread issues tcgen05.mma into one of two TMEM
+//                  accumulator buffers and commits barriers
+//      warps 2-9   epilogue: TMEM -> registers -> per-warp shared-memory
+//                  transposition -> alpha scale -> 128-byte row stores, for
+//                  tile i while the MMAs of tile i+1 run
+//    Measured on B200 and shaping this code: a thread alone on its warp retires
+//    about one instruction per 5-8 cycles (more when other warps compete) and
+//    an mbarrier wait costs ~200 cycles even when it is ready, so the issuing
+//    thread runs straight code over large stages from tabulated offsets; warps
+//    that wait elect one poller that sleeps between attempts, because many
+//    pollers crowd the issuing threads.  Every wait is bounded; one that runs
+//    out raises a status word the host reads, and the CTA still frees its
+//    TMEM and returns.
 #include <cuda_fp16.h>
 
 #include <cstdlib>
@@ -38,14 +47,15 @@ namespace snn {
 
 namespace {
 
-constexpr int TC_WORKERS = 256;               // warps 0-7
-constexpr int TC_THREADS = TC_WORKERS + 64;   // + warp 8 (MMA issue) + warp 9 (weight producer)
+constexpr int TC_THREADS = 320;               // warp 0 producer, warp 1 MMA issue, warps 2-9 epilogue
+constexpr int EPI_WARPS = 8;
 constexpr int NS_MAX = 8;                     // most weight stages in flight
+constexpr int NA_MAX = 4;                     // most activation units in flight
 constexpr uint32_t WAIT_LIMIT = 1u << 20;     // try_wait attempts before a wait gives up
-constexpr int EPI_PITCH = 144;                // bytes per staged output row (32 words + 16 B pad: conflict-free)
-constexpr int EPI_BYTES = 8 * 32 * EPI_PITCH; // per-warp transposition tiles
+constexpr int EPI_PITCH = 128;                // bytes per staged output row; 16-byte columns are XOR-swizzled by row
+constexpr int EPI_BYTES = EPI_WARPS * 32 * EPI_PITCH;
 constexpr int kMaxSegs = 192;                 // entries of the A-offset table
-constexpr size_t kSmemTail = 1024 + 1024;     // alpha table + (barriers, flags, A-offset table)
+constexpr size_t kSmemTail = 1280;            // barriers, flags, A-offset table
 
 // Division by a run-time constant as multiply-high + shifts (round-up method,
 // exact for every 32-bit numerator).
@@ -68,7 +78,8 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t q, const FastDiv& f) {
 }
 
 struct TcParams {
-  const void* act;        // uint32 [N][H][W][Cw] or half [N][H][W][C]
+  const void* act;        // uint32 [N][H][W][Cw] or half [N][H][W][C]      (expansion kernel)
+  uint8_t* xa;            // expanded activations [plane][chunk][Qpad][16 B]  (scratch)
   const uint8_t* wt;      // tiled weights: [layout tile][tap][chunk][NtL][16 B]
   const float* alpha;
   void* out;
@@ -82,17 +93,22 @@ struct TcParams {
   int n_planes;           // 1 (stride 1) or 4 (stride 2)
   int halo;               // largest tap shift in rows
   int Rr;                 // staged rows per plane = 128*MT + halo
-  int MT, Nt;             // M sub-tiles per CTA, channels per CTA
-  int cb_chunks, n_cb;    // chunks per channel block (activations are staged per block), blocks
-  int kpt;                // MMAs per sub-tile and tap within a channel block (= cb_chunks / 2)
-  int st_taps;            // taps per weight stage (1, 3 or 9; more than 1 only with one channel block)
+  uint32_t Qpad;          // positions per (plane, chunk) row of xa
+  int MT, Nt;             // M sub-tiles per tile, channels per tile
+  int cb_chunks, n_cb;    // chunks per activation unit (a channel block of one tile), units per tile
+  int kpt;                // MMAs per sub-tile and tap within a unit (= cb_chunks / 2)
+  int st_taps;            // taps per weight stage (1, 3 or 9; more than 1 only with one unit per tile)
   int st_k;               // MMAs per sub-tile, tap and stage (= kpt when a stage holds whole taps)
-  int NS;                 // weight stages in flight
+  int NS, NA;             // weight stages / activation units in flight
+  int n_acc;              // TMEM accumulator buffers (1 or 2)
+  int b_resident;         // the whole weight set of the CTA's channel tile stays in the ring
+  int n_ntiles;           // channel tiles
+  int total_tiles;        // position groups * channel tiles
   long long Qtot;         // flattened positions to cover
-  uint32_t tmem_cols;     // power of two >= MT*Nt
-  uint32_t a_bytes;       // bytes of the staged activation block
+  uint32_t tmem_cols;     // power of two >= n_acc*MT*Nt
+  uint32_t a_unit_bytes;  // bytes of one staged activation unit
   uint32_t stage_bytes;   // bytes of one weight stage
-  uint32_t tail_off;      // offset of the alpha table and barriers behind both regions
+  uint32_t off_b, off_epi, off_tail;  // shared-memory offsets
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -142,17 +158,11 @@ __device__ __forceinline__ void raise_status(int* status, int code) {
   *reinterpret_cast<volatile int*>(status) = code;
   __threadfence_system();
 }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// Hardware barriers: 1 = the 256 workers among themselves; 2 = workers wait, the
-// MMA warp arrives (288 threads in all) once the accumulators are complete.
-__device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-__device__ __forceinline__ void accum_wait() { asm volatile("bar.sync 2, 288;" ::: "memory"); }
-__device__ __forceinline__ void accum_release() { asm volatile("bar.arrive 2, 288;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, K-major, no swizzle: rows 16 B apart inside an
 // 8-row group, groups `sbo` bytes apart, the two 16-byte K chunks `lbo` bytes apart.
@@ -216,10 +226,10 @@ __device__ __forceinline__ uint32_t nibble_to_mask(uint32_t nib) {
   return t * 0xffu;
 }
 
-// 32 activation bits -> 32 bytes of +1 / -1 (zero where the channel does not exist) -> two 16-byte chunks
-__device__ __forceinline__ void expand_word(uint32_t bits, int channels_left, bool present, uint8_t* dst_lo,
-                                            uint8_t* dst_hi) {
-  uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
+// 32 activation bits -> 32 bytes of +1 / -1 (zero where the channel does not exist)
+__device__ __forceinline__ void expand_word(uint32_t bits, int channels_left, bool present, uint4& lo, uint4& hi) {
+  lo = make_uint4(0, 0, 0, 0);
+  hi = make_uint4(0, 0, 0, 0);
   if (present && channels_left > 0) {
     lo.x = nibble_to_pm1(bits & 15u);
     lo.y = nibble_to_pm1((bits >> 4) & 15u);
@@ -241,12 +251,11 @@ __device__ __forceinline__ void expand_word(uint32_t bits, int channels_left, bo
       hi.w &= nibble_to_mask(vm >> 28);
     }
   }
-  *reinterpret_cast<uint4*>(dst_lo) = lo;
-  *reinterpret_cast<uint4*>(dst_hi) = hi;
 }
 
 // Flattened position of plane (pa, pb) -> input pixel index, or -1 when it is padding.
 __device__ __forceinline__ int position_to_pixel(const TcParams& p, uint32_t q, int pa, int pb) {
+  if ((long long)q >= p.Qtot) return -1;
   const uint32_t rg = fdiv(q, p.dWq);
   const int j = (int)(q - rg * (uint32_t)p.Wq);
   const uint32_t n = fdiv(rg, p.dHq);
@@ -260,8 +269,8 @@ __device__ __forceinline__ int position_to_pixel(const TcParams& p, uint32_t q, 
 // One 16/32-column slice of an accumulator row straight from registers (used
 // when c_out is not a multiple of 4 or the channel tile not a multiple of 32).
 template <bool F16, int NC>
-__device__ __forceinline__ void epilogue_slice(const TcParams& p, uint32_t taddr, const float* alpha_s, int c0, int n0,
-                                               bool valid, size_t obase) {
+__device__ __forceinline__ void epilogue_slice(const TcParams& p, uint32_t taddr, int c0, int n0, bool valid,
+                                               size_t obase) {
   uint32_t v[NC];
   if (NC == 32) tmem_ld32(taddr, reinterpret_cast<uint32_t(&)[32]>(v));
   else tmem_ld16(taddr, reinterpret_cast<uint32_t(&)[16]>(v));
@@ -277,66 +286,117 @@ __device__ __forceinline__ void epilogue_slice(const TcParams& p, uint32_t taddr
     float* o = (float*)p.out + obase + co0;
 #pragma unroll
     for (int e = 0; e < NC; ++e)
-      if (co0 + e < p.K) o[e] = __fmul_rn(F16 ? __uint_as_float(v[e]) : (float)(int)v[e], alpha_s[c0 + e]);
+      if (co0 + e < p.K)
+        o[e] = __fmul_rn(F16 ? __uint_as_float(v[e]) : (float)(int)v[e], __ldg(p.alpha + co0 + e));
   }
 }
 
 }  // namespace
 
+// ------------------------------------------------------------------ expansion
+// One thread per (plane, position): all channel chunks of that position.  Reads
+// are contiguous per thread, writes are 16 bytes per thread with consecutive
+// threads on consecutive positions (coalesced).  Every row of xa is written,
+// padding and tail included, so the scratch never needs clearing.
+template <bool F16>
+__global__ void __launch_bounds__(256) tc_expand_act_kernel(const TcParams p) {
+  const uint32_t q = blockIdx.x * 256u + threadIdx.x;
+  if (q >= p.Qpad) return;
+  const int pl = blockIdx.y, pa = pl >> 1, pb = pl & 1;
+  const int pix = position_to_pixel(p, q, pa, pb);
+  uint4* dst = reinterpret_cast<uint4*>(p.xa) + (size_t)pl * p.n_chunks * p.Qpad + q;
+  if (F16) {
+    const __half* src = (const __half*)p.act + (size_t)(pix < 0 ? 0 : pix) * p.C;
+    const bool vec = pix >= 0 && ((p.C & 7) == 0);
+    for (int c = 0; c < p.n_chunks; ++c) {
+      uint4 v = make_uint4(0, 0, 0, 0);
+      const int ch = c * 8;
+      if (vec && ch + 8 <= p.C) {
+        v = __ldg(reinterpret_cast<const uint4*>(src + ch));
+      } else if (pix >= 0) {
+        uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          if (ch + e < p.C) w[e >> 1] |= (uint32_t)__half_as_ushort(src[ch + e]) << (16 * (e & 1));
+        v = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      dst[(size_t)c * p.Qpad] = v;
+    }
+  } else {
+    const uint32_t* src = (const uint32_t*)p.act + (size_t)(pix < 0 ? 0 : pix) * p.Cw;
+    const int nw = p.n_chunks / 2;
+    const bool vec_ok = (p.Cw & 3) == 0;
+    for (int wb = 0; wb < nw; wb += 4) {
+      uint32_t b[4] = {0, 0, 0, 0};
+      if (pix >= 0) {
+        if (vec_ok && wb + 4 <= p.Cw) {
+          const uint4 t = __ldg(reinterpret_cast<const uint4*>(src + wb));
+          b[0] = t.x; b[1] = t.y; b[2] = t.z; b[3] = t.w;
+        } else {
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if (wb + k < p.Cw) b[k] = __ldg(src + wb + k);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int wg = wb + k;
+        if (wg < nw) {
+          uint4 lo, hi;
+          expand_word(b[k], p.C - wg * 32, pix >= 0 && wg < p.Cw, lo, hi);
+          dst[(size_t)(2 * wg) * p.Qpad] = lo;
+          dst[(size_t)(2 * wg + 1) * p.Qpad] = hi;
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------ GEMM
 template <bool F16, int MT>
-__global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
+__global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
-  // carve-up: [activation block][NS weight stages] ... [alpha][barriers, flags, A-offset table]
+  // carve-up: [NA activation units][NS weight stages][epilogue tiles][barriers, flags, table]
   uint8_t* a_smem = smem;
-  uint8_t* b_smem = smem + p.a_bytes;
-  float* alpha_s = reinterpret_cast<float*>(smem + p.tail_off);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(alpha_s + 256);
-  // bars: full[8], empty[8], a_ready, a_free, accum
-  const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + NS_MAX);
-  const uint32_t bar_aready = smem_u32(bars + 2 * NS_MAX), bar_afree = smem_u32(bars + 2 * NS_MAX + 1);
-  const uint32_t bar_accum = smem_u32(bars + 2 * NS_MAX + 2);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * NS_MAX + 3);
+  uint8_t* b_smem = smem + p.off_b;
+  uint8_t* epi_smem = smem + p.off_epi;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_tail);
+  // barriers: b_full[8] b_empty[8] a_full[4] a_empty[4] acc_full[2] acc_empty[2]
+  const uint32_t bar_bfull = smem_u32(bars), bar_bempty = smem_u32(bars + 8);
+  const uint32_t bar_afull = smem_u32(bars + 16), bar_aempty = smem_u32(bars + 20);
+  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 28);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* wait_flags = abort_flag + 1;  // [0..1] a_free waits, [2] accumulators complete
-  uint32_t* seg_units = const_cast<uint32_t*>(reinterpret_cast<volatile uint32_t*>(wait_flags + 3));
+  uint32_t* seg_units = tmem_slot + 2;  // [9 * segs_per_tap] A row offset of every (tap, k-segment)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t Q0 = blockIdx.x * (uint32_t)(128 * MT);
-  const int n0 = blockIdx.y * p.Nt;
-  const int NS = p.NS;
+  const int NS = p.NS, NA = p.NA;
+  const int segs_per_tap = p.kpt / p.st_k;
 
-  if (tid == 0) {
-    for (int s = 0; s < NS; ++s) {
-      mbar_init(bar_full + 8 * s, 1);
-      mbar_init(bar_empty + 8 * s, 1);
-    }
-    mbar_init(bar_aready, TC_WORKERS);
-    mbar_init(bar_afree, 1);
-    mbar_init(bar_accum, 1);
-    *abort_flag = 0;
-    wait_flags[0] = wait_flags[1] = wait_flags[2] = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  if (tid < 28) {
+    uint32_t count = 1;
+    if (tid >= 26) count = EPI_WARPS;  // acc_empty: one arrival per epilogue warp
+    mbar_init(smem_u32(bars + tid), count);
   }
-  if (warp == 0) {
+  if (tid == 32) *abort_flag = 0;
+  for (int e = tid; e < 9 * segs_per_tap; e += TC_THREADS) {
+    // rows (16-byte units) from the unit's origin to (tap, k-segment): plane offset + tap shift
+    // inside the plane + the segment's first chunk
+    const int t = e / segs_per_tap, seg = e - t * segs_per_tap;
+    const int ky = t / 3, kx = t % 3;
+    uint32_t u;
+    if (p.stride == 1) u = (uint32_t)(ky * p.Wq + kx);
+    else u = (uint32_t)((ky & 1) * 2 + (kx & 1)) * (uint32_t)(p.cb_chunks * p.Rr) +
+             (uint32_t)((ky >> 1) * p.Wq + (kx >> 1));
+    seg_units[e] = u + (uint32_t)(seg * p.st_k * 2) * (uint32_t)p.Rr;
+  }
+  if (warp == 2) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "r"(p.tmem_cols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  const int segs_per_tap = p.kpt / p.st_k;
-  {
-    // A-operand row offset (16-byte units) of every (tap, k-segment): plane offset + tap shift
-    // inside the plane + the segment's first chunk.  The issuing thread only reads this table.
-    for (int e = tid; e < 9 * segs_per_tap; e += TC_THREADS) {
-      const int t = e / segs_per_tap, seg = e - t * segs_per_tap;
-      const int ky = t / 3, kx = t % 3;
-      uint32_t u;
-      if (p.stride == 1) u = (uint32_t)(ky * p.Wq + kx);
-      else u = (uint32_t)((ky & 1) * 2 + (kx & 1)) * (uint32_t)(p.cb_chunks * p.Rr) +
-               (uint32_t)((ky >> 1) * p.Wq + (kx >> 1));
-      seg_units[e] = u + (uint32_t)(seg * p.st_k * 2) * (uint32_t)p.Rr;
-    }
-  }
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -344,50 +404,88 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
 
   // A weight stage holds st_taps whole taps, or st_k MMAs' worth of one tap.
   const int stages_per_cb = (9 / p.st_taps) * segs_per_tap;
-  const int n_stages = p.n_cb * stages_per_cb;
-  const uint32_t plane_bytes = (uint32_t)p.cb_chunks * p.Rr * 16;
+  const uint32_t acc_cols = (uint32_t)(MT * p.Nt);
 
-  if (warp == 9) {
-    // ------------------------------------------------ weight producer (one lane)
+  if (warp == 0) {
+    // ------------------------------------------------ producer (one lane)
     if (lane == 0) {
-      int issued = 0;
-      const size_t tile_base = (size_t)(n0 / p.NtL) * 9 * p.n_chunks;  // layout tile of this CTA's channels
-      const int n_in = n0 % p.NtL;
-      int slot = 0, cb = 0, rem = 0;
-      uint32_t phase = 1;  // parity of the *previous* use of the slot; meaningful from the second lap on
-      for (int i = 0; i < n_stages; ++i) {
-        if (*abort_flag) break;
-        if (i >= NS && !mbar_wait_backoff(bar_empty + 8 * slot, phase, 64)) {
-          *abort_flag = 1;
-          raise_status(p.status, 1);
-          break;
+      int a_slot = 0, b_slot = 0, a_issued = 0, b_issued = 0;
+      uint32_t a_phase = 1, b_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
+      bool ok = true;
+      bool first_tile = true;
+      const uint32_t unit_rows_bytes = (uint32_t)p.Rr * 16;
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+        const int mg = tile / p.n_ntiles, nti = tile - mg * p.n_ntiles;
+        const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
+        const int n0 = nti * p.Nt;
+        const size_t tile_base = (size_t)(n0 / p.NtL) * 9 * p.n_chunks;  // layout tile of these channels
+        const int n_in = n0 % p.NtL;
+        for (int cb = 0; cb < p.n_cb && ok; ++cb) {
+          // ---- activation unit: every (plane, chunk) of this channel block is one contiguous run of xa
+          if (*abort_flag) { ok = false; break; }
+          if (a_issued >= NA && !mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 32)) {
+            *abort_flag = 1;
+            raise_status(p.status, 1);
+            ok = false;
+            break;
+          }
+          mbar_expect_tx(bar_afull + 8 * a_slot, (uint32_t)(p.n_planes * p.cb_chunks) * unit_rows_bytes);
+          {
+            uint32_t dst = smem_u32(a_smem) + (uint32_t)a_slot * p.a_unit_bytes;
+            for (int pl = 0; pl < p.n_planes; ++pl) {
+              const uint8_t* src = p.xa + (((size_t)pl * p.n_chunks + (size_t)cb * p.cb_chunks) * p.Qpad + Q0) * 16;
+              for (int c = 0; c < p.cb_chunks; ++c) {
+                bulk_g2s(dst, src, unit_rows_bytes, bar_afull + 8 * a_slot);
+                dst += unit_rows_bytes;
+                src += (size_t)p.Qpad * 16;
+              }
+            }
+          }
+          ++a_issued;
+          if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
+          // ---- weight stages of this channel block (kept from the first tile on when resident)
+          if (p.b_resident && !first_tile) continue;
+          for (int rem = 0; rem < stages_per_cb; ++rem) {
+            if (b_issued >= NS && !mbar_wait_backoff(bar_bempty + 8 * b_slot, b_phase, 32)) {
+              *abort_flag = 1;
+              raise_status(p.status, 2);
+              ok = false;
+              break;
+            }
+            const int tg = rem / segs_per_tap, seg = rem - tg * segs_per_tap;
+            const int chunk0 = cb * p.cb_chunks + seg * p.st_k * 2;
+            const uint32_t dst = smem_u32(b_smem) + (uint32_t)b_slot * p.stage_bytes;
+            const uint8_t* src =
+                p.wt + ((tile_base + (size_t)(tg * p.st_taps) * p.n_chunks + chunk0) * p.NtL + n_in) * 16;
+            mbar_expect_tx(bar_bfull + 8 * b_slot, p.stage_bytes);
+            if (p.Nt == p.NtL) {
+              bulk_g2s(dst, src, p.stage_bytes, bar_bfull + 8 * b_slot);  // consecutive (tap, chunk) blocks are contiguous
+            } else {
+              const int nchunk = p.st_taps * p.st_k * 2;
+              for (int c = 0; c < nchunk; ++c)
+                bulk_g2s(dst + (uint32_t)c * p.Nt * 16, src + (size_t)c * p.NtL * 16, (uint32_t)p.Nt * 16,
+                         bar_bfull + 8 * b_slot);
+            }
+            ++b_issued;
+            if (++b_slot == NS) { b_slot = 0; b_phase ^= 1u; }
+          }
         }
-        const int tg = rem / segs_per_tap, seg = rem - tg * segs_per_tap;
-        const int chunk0 = cb * p.cb_chunks + seg * p.st_k * 2;
-        const uint32_t dst = smem_u32(b_smem + (size_t)slot * p.stage_bytes);
-        const uint8_t* src = p.wt + ((tile_base + (size_t)(tg * p.st_taps) * p.n_chunks + chunk0) * p.NtL + n_in) * 16;
-        mbar_expect_tx(bar_full + 8 * slot, p.stage_bytes);
-        if (p.Nt == p.NtL) {
-          bulk_g2s(dst, src, p.stage_bytes, bar_full + 8 * slot);  // consecutive (tap, chunk) blocks are contiguous
-        } else {
-          const int nchunk = p.st_taps * p.st_k * 2;
-          for (int c = 0; c < nchunk; ++c)
-            bulk_g2s(dst + (uint32_t)c * p.Nt * 16, src + (size_t)c * p.NtL * 16, (uint32_t)p.Nt * 16,
-                     bar_full + 8 * slot);
-        }
-        issued = i + 1;
-        if (++rem == stages_per_cb) { rem = 0; ++cb; }
-        if (++slot == NS) { slot = 0; phase ^= 1u; }
+        first_tile = false;
       }
       // never leave with copies in flight: wait (bounded) for the last load of every slot
+      for (int s = 0; s < NA; ++s) {
+        int last = -1;
+        for (int i = s; i < a_issued; i += NA) last = i;
+        if (last >= 0) mbar_wait_backoff(bar_afull + 8 * s, (last / NA) & 1, 64);
+      }
       for (int s = 0; s < NS; ++s) {
         int last = -1;
-        for (int i = s; i < issued; i += NS) last = i;
-        if (last >= 0) mbar_wait_backoff(bar_full + 8 * s, (last / NS) & 1, 64);
+        for (int i = s; i < b_issued; i += NS) last = i;
+        if (last >= 0) mbar_wait_backoff(bar_bfull + 8 * s, (last / NS) & 1, 64);
       }
     }
     __syncwarp();
-  } else if (warp == 8) {
+  } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer (one lane)
     if (lane == 0) {
       // instruction descriptor: D format, A/B formats, K-major both, N>>3, M>>4
@@ -398,179 +496,100 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
       // address field.
       const uint64_t a_desc0 = make_desc(smem_u32(a_smem), (uint32_t)p.Rr * 16, 128);
       const uint64_t b_desc0 = make_desc(smem_u32(b_smem), (uint32_t)p.Nt * 16, 128);
-      const uint32_t stage_units = p.stage_bytes >> 4;
+      const uint32_t stage_units = p.stage_bytes >> 4, unit_units = p.a_unit_bytes >> 4;
       const uint32_t a_step = 2u * (uint32_t)p.Rr, b_step = 2u * (uint32_t)p.Nt;  // two chunks per MMA
       const uint32_t nt = (uint32_t)p.Nt;
       const int st_k = p.st_k, st_taps = p.st_taps;
       bool ok = true;
-      uint32_t acc = 0;          // 0 only for the first MMA of every sub-tile
-      int slot = 0;              // ring position and its phase, stepped without divisions
-      uint32_t phase = 0;
-      for (int cb = 0; cb < p.n_cb && ok; ++cb) {
-        if (!mbar_wait(bar_aready, cb & 1)) { ok = false; break; }
-        tc_fence_after();
-        int e = 0;               // index into seg_units
-        for (int rem = 0; rem < stages_per_cb; ++rem) {
-          if (!mbar_wait(bar_full + 8 * slot, phase)) { ok = false; break; }
+      int a_slot = 0, b_slot = 0, acc_slot = 0;
+      uint32_t a_phase = 0, b_phase = 0, acc_phase = 1;
+      int tiles_done = 0;
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tiles_done) {
+        // the accumulator buffer must have been drained by the epilogue of its previous tile
+        if (tiles_done >= p.n_acc) {
+          if (!mbar_wait(bar_accempty + 8 * acc_slot, acc_phase)) { ok = false; break; }
           tc_fence_after();
-          uint64_t bd = b_desc0 + (uint64_t)((uint32_t)slot * stage_units);
-          for (int tt = 0; tt < st_taps; ++tt, ++e) {
-            uint64_t ad = a_desc0 + (uint64_t)seg_units[e];
-            int k = 0;
-            for (; k + 4 <= st_k; k += 4) {
+        }
+        const uint32_t d0 = tmem_base + (uint32_t)acc_slot * acc_cols;
+        uint32_t acc = 0;  // 0 only for the first MMA of every sub-tile
+        const bool wait_b = !(p.b_resident && tiles_done > 0);
+        for (int cb = 0; cb < p.n_cb && ok; ++cb) {
+          if (!mbar_wait(bar_afull + 8 * a_slot, a_phase)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t a_unit = a_desc0 + (uint64_t)((uint32_t)a_slot * unit_units);
+          int e = 0;  // index into seg_units
+          for (int rem = 0; rem < stages_per_cb; ++rem) {
+            if (wait_b) {
+              if (!mbar_wait(bar_bfull + 8 * b_slot, b_phase)) { ok = false; break; }
+              tc_fence_after();
+            }
+            uint64_t bd = b_desc0 + (uint64_t)((uint32_t)b_slot * stage_units);
+            for (int tt = 0; tt < st_taps; ++tt, ++e) {
+              uint64_t ad = a_unit + (uint64_t)seg_units[e];
+              int k = 0;
+              for (; k + 4 <= st_k; k += 4) {
 #pragma unroll
-              for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < 4; ++u) {
+#pragma unroll
+                  for (int mt = 0; mt < MT; ++mt)
+                    mma_ss<F16>(d0 + (uint32_t)mt * nt, ad + (uint64_t)(mt * 128), bd, idesc, acc);
+                  acc = 1;
+                  ad += a_step;
+                  bd += b_step;
+                }
+              }
+              for (; k < st_k; ++k) {
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt)
-                  mma_ss<F16>(tmem_base + (uint32_t)mt * nt, ad + (uint64_t)(mt * 128), bd, idesc, acc);
+                  mma_ss<F16>(d0 + (uint32_t)mt * nt, ad + (uint64_t)(mt * 128), bd, idesc, acc);
                 acc = 1;
                 ad += a_step;
                 bd += b_step;
               }
             }
-            for (; k < st_k; ++k) {
-#pragma unroll
-              for (int mt = 0; mt < MT; ++mt)
-                mma_ss<F16>(tmem_base + (uint32_t)mt * nt, ad + (uint64_t)(mt * 128), bd, idesc, acc);
-              acc = 1;
-              ad += a_step;
-              bd += b_step;
-            }
+            if (!p.b_resident) tc_commit(bar_bempty + 8 * b_slot);  // free once these MMAs have read it
+            if (++b_slot == NS) { b_slot = 0; b_phase ^= 1u; }
           }
-          tc_commit(bar_empty + 8 * slot);  // the slot is free once these MMAs have read it
-          if (++slot == NS) { slot = 0; phase ^= 1u; }
+          tc_commit(bar_aempty + 8 * a_slot);  // the activation unit may be overwritten
+          if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
         }
-        if (ok && cb + 1 < p.n_cb) tc_commit(bar_afree);  // activation block may be overwritten
+        tc_commit(bar_accfull + 8 * acc_slot);  // fires when this tile's MMAs are complete
+        if (++acc_slot == p.n_acc) { acc_slot = 0; acc_phase ^= 1u; }
       }
       if (!ok) {
         *abort_flag = 1;
-        raise_status(p.status, 2);
+        raise_status(p.status, 3);
       }
-      tc_commit(bar_accum);  // fires when everything issued so far is complete
-      const bool done = mbar_wait(bar_accum, 0);
-      if (!done) {
-        *abort_flag = 1;
-        raise_status(p.status, 4);
-      }
-      wait_flags[2] = done ? 1 : 0;
-      __threadfence_block();
     }
     __syncwarp();
-    accum_release();  // lets the workers into the epilogue
   } else {
-    // ------------------------------------------------ workers: expand activations, then epilogue
-    // this CTA's scales: requested now, parked in shared memory after the expansion (the
-    // epilogue reads them behind the accumulator barrier), so their latency is hidden
-    const float my_alpha = (tid < p.Nt && n0 + tid < p.K) ? __ldg(p.alpha + n0 + tid) : 0.f;
-    for (int cb = 0; cb < p.n_cb; ++cb) {
-      if (cb > 0) {
-        // one elected thread polls; the rest wait on a hardware barrier instead of spinning
-        if (tid == 0) wait_flags[cb & 1] = mbar_wait_backoff(bar_afree, (cb - 1) & 1, 200) ? 1 : 0;
-        worker_sync();
-        if (!wait_flags[cb & 1]) {
+    // ------------------------------------------------ epilogue warps
+    // Warp w reads TMEM lanes 32*(w%4).. (rows of the tile); the two warps of a lane quarter
+    // split the 32-column slices between them.  A slice goes through a per-warp shared-memory
+    // tile so that each store instruction writes whole 128-byte rows.
+    const int ew = warp - 2;
+    const int rq = warp & 3, half = ew >> 2;
+    uint8_t* stage = epi_smem + (size_t)ew * (32 * EPI_PITCH);
+    const int srow = lane >> 3, scol = lane & 7;  // this lane's (row mod 4, 16-byte column) when storing
+    const bool fast = ((p.K & 3) == 0) && ((p.Nt & 31) == 0);
+    int acc_slot = 0;
+    uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+      const int mg = tile / p.n_ntiles, nti = tile - mg * p.n_ntiles;
+      const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
+      const int n0 = nti * p.Nt;
+      int okw = 1;
+      if (lane == 0) okw = (!*abort_flag && mbar_wait_backoff(bar_accfull + 8 * acc_slot, acc_phase, 100)) ? 1 : 0;
+      okw = __shfl_sync(0xffffffffu, okw, 0);
+      if (!okw) {
+        if (lane == 0 && !*abort_flag) {
           *abort_flag = 1;
-          if (tid == 0) raise_status(p.status, 3);
+          raise_status(p.status, 4);
         }
+        break;
       }
-      if (!*abort_flag) {
-        for (int pl = 0; pl < p.n_planes; ++pl) {
-          const int pa = pl >> 1, pb = pl & 1;
-          uint8_t* a_plane = a_smem + (size_t)pl * plane_bytes;
-          if (F16) {
-#pragma unroll 2
-            for (int r = tid; r < p.Rr; r += TC_WORKERS) {
-              const int pix = position_to_pixel(p, Q0 + (uint32_t)r, pa, pb);
-              const int ch0 = cb * p.cb_chunks * 8;
-              const __half* src = (const __half*)p.act + (size_t)(pix < 0 ? 0 : pix) * p.C + ch0;
-              const bool vec = pix >= 0 && ((p.C & 7) == 0);
-              for (int c = 0; c < p.cb_chunks; ++c) {
-                uint4 v = make_uint4(0, 0, 0, 0);
-                const int ch = ch0 + c * 8;
-                if (vec && ch + 8 <= p.C) {
-                  v = __ldg(reinterpret_cast<const uint4*>(src + c * 8));
-                } else if (pix >= 0) {
-                  uint32_t w[4] = {0, 0, 0, 0};
-#pragma unroll
-                  for (int e = 0; e < 8; ++e)
-                    if (ch + e < p.C) w[e >> 1] |= (uint32_t)__half_as_ushort(src[c * 8 + e]) << (16 * (e & 1));
-                  v = make_uint4(w[0], w[1], w[2], w[3]);
-                }
-                *reinterpret_cast<uint4*>(a_plane + ((size_t)c * p.Rr + r) * 16) = v;
-              }
-            }
-          } else {
-            // two rows and up to eight 32-channel words per row are requested before any is
-            // expanded, so a thread has its global loads in flight together
-            const int nw = p.cb_chunks / 2, w0 = cb * nw;
-            const bool vec_ok = (p.Cw & 3) == 0 && (w0 & 3) == 0;
-            for (int rb = tid; rb < p.Rr; rb += 2 * TC_WORKERS) {
-              const int r1 = rb + TC_WORKERS;
-              const bool has1 = r1 < p.Rr;
-              const int pix0 = position_to_pixel(p, Q0 + (uint32_t)rb, pa, pb);
-              const int pix1 = has1 ? position_to_pixel(p, Q0 + (uint32_t)r1, pa, pb) : -1;
-              const uint32_t* s0 = (const uint32_t*)p.act + (size_t)(pix0 < 0 ? 0 : pix0) * p.Cw + w0;
-              const uint32_t* s1 = (const uint32_t*)p.act + (size_t)(pix1 < 0 ? 0 : pix1) * p.Cw + w0;
-              for (int wb = 0; wb < nw; wb += 8) {
-                uint32_t b0[8], b1[8];
-#pragma unroll
-                for (int k = 0; k < 8; ++k) b0[k] = b1[k] = 0;
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                  const int wq = wb + 4 * h;
-                  if (vec_ok && w0 + wq + 4 <= p.Cw && wq + 4 <= nw) {
-                    if (pix0 >= 0) {
-                      const uint4 t = __ldg(reinterpret_cast<const uint4*>(s0 + wq));
-                      b0[4 * h] = t.x; b0[4 * h + 1] = t.y; b0[4 * h + 2] = t.z; b0[4 * h + 3] = t.w;
-                    }
-                    if (pix1 >= 0) {
-                      const uint4 t = __ldg(reinterpret_cast<const uint4*>(s1 + wq));
-                      b1[4 * h] = t.x; b1[4 * h + 1] = t.y; b1[4 * h + 2] = t.z; b1[4 * h + 3] = t.w;
-                    }
-                  } else {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                      if (wq + k < nw && w0 + wq + k < p.Cw) {
-                        if (pix0 >= 0) b0[4 * h + k] = __ldg(s0 + wq + k);
-                        if (pix1 >= 0) b1[4 * h + k] = __ldg(s1 + wq + k);
-                      }
-                    }
-                  }
-                }
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                  if (wb + k < nw) {
-                    const int wg = w0 + wb + k;
-                    expand_word(b0[k], p.C - wg * 32, pix0 >= 0 && wg < p.Cw,
-                                a_plane + ((size_t)(2 * (wb + k)) * p.Rr + rb) * 16,
-                                a_plane + ((size_t)(2 * (wb + k) + 1) * p.Rr + rb) * 16);
-                    if (has1)
-                      expand_word(b1[k], p.C - wg * 32, pix1 >= 0 && wg < p.Cw,
-                                  a_plane + ((size_t)(2 * (wb + k)) * p.Rr + r1) * 16,
-                                  a_plane + ((size_t)(2 * (wb + k) + 1) * p.Rr + r1) * 16);
-                  }
-                }
-              }
-            }
-          }
-        }
-      }
-      fence_proxy_async();      // generic-proxy writes -> visible to the tensor core's reads
-      mbar_arrive(bar_aready);
-    }
-
-    alpha_s[tid] = my_alpha;
-    // ---- epilogue: row m of sub-tile mt lives in TMEM lane m, columns mt*Nt ..
-    accum_wait();               // released by the MMA warp when the accumulators are complete
-    tc_fence_after();
-    const bool go = __all_sync(0xffffffffu, wait_flags[2] != 0 && !*abort_flag);  // warp-uniform: TMEM loads are .aligned
-    if (go) {
-      // Warp w reads TMEM lanes 32*(w&3).. (rows of the tile); warps 0-3 take the even
-      // 32-column slices, warps 4-7 the odd ones.  A slice goes through a per-warp
-      // shared-memory tile so that each store instruction writes whole 128-byte rows.
-      const int rq = warp & 3, half = warp >> 2;
-      uint8_t* stage = smem + (size_t)warp * (32 * EPI_PITCH);  // activation block and weight ring are dead by now
-      const int srow = lane >> 3, scol = lane & 7;              // this lane's (row mod 4, 16-byte column) when storing
-      const bool fast = ((p.K & 3) == 0) && ((p.Nt & 31) == 0);
+      tc_fence_after();
+      const uint32_t d0 = tmem_base + (uint32_t)acc_slot * acc_cols;
 #pragma unroll 1
       for (int mt = 0; mt < MT; ++mt) {
         const uint32_t q = Q0 + (uint32_t)(mt * 128 + rq * 32 + lane);
@@ -578,9 +597,9 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
         const int x = (int)(q - rg * (uint32_t)p.Wq);
         const uint32_t n = fdiv(rg, p.dHq);
         const int y = (int)(rg - n * (uint32_t)p.Hq);
-        const bool valid = ((int)n < p.N) && (y < p.Ho) && (x < p.Wo);
+        const bool valid = ((long long)q < p.Qtot) && ((int)n < p.N) && (y < p.Ho) && (x < p.Wo);
         const size_t obase = (((size_t)n * p.Ho + y) * p.Wo + x) * p.K;
-        const uint32_t trow = tmem_base + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt);
+        const uint32_t trow = d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt);
         if (fast) {
           // element offsets of the eight rows this lane stores (row = srow + 4*i), -1 when not an output
           long long ro[8];
@@ -590,18 +609,20 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
           for (int c0 = 32 * half; c0 < p.Nt; c0 += 64) {
             uint32_t v[32];
             tmem_ld32(trow + (uint32_t)c0, v);
+            const int co = n0 + c0 + scol * 4;
+            float4 al = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (!p.out_i32 && co < p.K) al = __ldg(reinterpret_cast<const float4*>(p.alpha + co));
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 8; ++e)
-              *reinterpret_cast<uint4*>(stage + lane * EPI_PITCH + e * 16) =
+              *reinterpret_cast<uint4*>(stage + lane * EPI_PITCH + ((e ^ (lane & 7)) << 4)) =
                   make_uint4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
             __syncwarp();
-            const int co = n0 + c0 + scol * 4;
-            const float4 al = *reinterpret_cast<const float4*>(alpha_s + c0 + scol * 4);
             if (co < p.K) {  // K is a multiple of 4 here, so the four channels exist together
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                const uint4 u = *reinterpret_cast<const uint4*>(stage + (srow + 4 * i) * EPI_PITCH + scol * 16);
+                const int row = srow + 4 * i;
+                const uint4 u = *reinterpret_cast<const uint4*>(stage + row * EPI_PITCH + ((scol ^ (row & 7)) << 4));
                 if (ro[i] < 0) continue;
                 if (p.out_i32) {
                   *reinterpret_cast<uint4*>((int32_t*)p.out + ro[i] + co) = u;
@@ -619,19 +640,24 @@ __global__ void __launch_bounds__(TC_THREADS) tc_conv_kernel(const TcParams p) {
           }
         } else if ((p.Nt & 31) == 0) {
           for (int c0 = 32 * half; c0 < p.Nt; c0 += 64)
-            epilogue_slice<F16, 32>(p, trow + (uint32_t)c0, alpha_s, c0, n0, valid, obase);
+            epilogue_slice<F16, 32>(p, trow + (uint32_t)c0, c0, n0, valid, obase);
         } else {
           for (int c0 = 16 * half; c0 < p.Nt; c0 += 32)
-            epilogue_slice<F16, 16>(p, trow + (uint32_t)c0, alpha_s, c0, n0, valid, obase);
+            epilogue_slice<F16, 16>(p, trow + (uint32_t)c0, c0, n0, valid, obase);
         }
       }
+      // this warp has read its part of the accumulator buffer: hand it back to the MMA issuer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_accempty + 8 * acc_slot);
+      if (++acc_slot == p.n_acc) { acc_slot = 0; acc_phase ^= 1u; }
     }
   }
 
   // ---------------------------------------------------------------- teardown
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == 2) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols)
                  : "memory");
   }
@@ -707,7 +733,8 @@ cudaError_t tc_expand_weights(const LayerDev& L, const Geom& g, int act_type, cu
 struct TcPlan {
   TcParams p;
   size_t smem;
-  dim3 grid;
+  size_t xa_bytes;
+  dim3 grid, xgrid;
   bool ok;
 };
 
@@ -716,27 +743,34 @@ static int env_int(const char* name, int dflt) {
   return v ? atoi(v) : dflt;
 }
 
-constexpr size_t kSmemTwoPerSm = 113 * 1024;   // leaves room for two CTAs on an SM
-constexpr size_t kSmemOnePerSm = 225 * 1024;
+static int sm_count() {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148;
+  }
+  return sms;
+}
 
-// variant: 0 = heuristic; otherwise (mt_code) + 4*(stage_code) + 16*(one_per_sm), see tc_variant_count()
+constexpr size_t kSmemBudget = 226 * 1024;
+
+// variant: 0 = heuristic; otherwise mt_code (1..3 -> 1,2,4) + 4*stage_code (0..3 -> 48,16,32,64 KB)
 static TcPlan make_plan(const Geom& g, int act_type, int variant) {
   TcPlan pl{};
   TcParams& p = pl.p;
   const bool f16 = act_type == SNN_ACT_F16;
   pl.ok = false;
   if (g.N < 1) return pl;
-  int want_mt = 0, want_stage_kb = 0, want_one = 0;
+  int want_mt = 0, want_stage_kb = 0;
   if (variant > 0) {
     static const int mts[4] = {0, 1, 2, 4};
     static const int kbs[4] = {0, 16, 32, 64};
     want_mt = mts[variant & 3];
     want_stage_kb = kbs[(variant >> 2) & 3];
-    want_one = (variant >> 4) & 1;
   }
   if (int v = env_int("SNN_TC_MT", 0)) want_mt = v;
   if (int v = env_int("SNN_TC_STAGE_KB", 0)) want_stage_kb = v;
-  if (int v = env_int("SNN_TC_ONE_PER_SM", 0)) want_one = v;
   int Kpad, Cpad;
   tc_weight_bytes(g, act_type, &Kpad, &Cpad);
   p.N = g.N; p.H = g.H; p.W = g.W; p.C = g.C; p.K = g.K; p.Cw = g.Cw;
@@ -752,26 +786,29 @@ static TcPlan make_plan(const Geom& g, int act_type, int variant) {
   p.dWq = make_fastdiv((uint32_t)p.Wq);
   p.dHq = make_fastdiv((uint32_t)p.Hq);
   p.Qtot = (long long)g.N * p.Hq * p.Wq;
-  if (p.Qtot + 512 + p.halo >= (1ll << 31)) return pl;  // positions are 32-bit in the kernel
+  if (p.Qtot + 1024 + p.halo >= (1ll << 31)) return pl;  // positions are 32-bit in the kernels
   if ((long long)g.N * g.H * g.W >= (1ll << 31)) return pl;
+  p.Qpad = (uint32_t)((p.Qtot + 511) / 512 * 512 + ((p.halo + 15) / 16 * 16));  // any tile's rows exist
+  pl.xa_bytes = (size_t)p.n_planes * p.n_chunks * p.Qpad * 16;
   const long long mtiles = (p.Qtot + 127) / 128;
-  // channels per CTA: a layout tile, or a part of one on request
+  const int sms = sm_count();
+  // channels per tile: a layout tile, or a part of one on request
   int Nt = p.NtL;
   int forced_nt = env_int("SNN_TC_NT", 0);
   if (forced_nt >= 16 && forced_nt <= 256 && forced_nt % 16 == 0 && p.NtL % forced_nt == 0) Nt = forced_nt;
   p.Nt = Nt;
-  const int ntiles = Kpad / Nt;
-  // M sub-tiles per CTA: the largest that keeps the SMs evenly loaded
+  p.n_ntiles = Kpad / Nt;
+  // M sub-tiles per tile: large tiles stage less halo, small tiles balance the SMs better
   int MT = 1;
   {
     double best = -1.0;
     for (int mt = 1; mt <= 4; mt *= 2) {
-      if (mt * Nt > 256) break;
-      long long ctas = ((mtiles + mt - 1) / mt) * ntiles;
-      long long waves = (ctas + 295) / 296;
-      double eff = (double)ctas / (double)(waves * 296);
-      if (ctas < 148) eff = (double)ctas / 148.0 * 0.5;
-      eff += 0.02 * mt;  // a larger tile stages less halo and re-reads fewer weights
+      if (mt * Nt > 512) break;
+      long long tiles = ((mtiles + mt - 1) / mt) * p.n_ntiles;
+      long long rounds = (tiles + sms - 1) / sms;
+      double eff = (double)tiles / (double)(rounds * sms);          // load balance of the persistent CTAs
+      eff *= (double)(128 * mt) / (double)(128 * mt + p.halo);       // useful share of the staged rows
+      if (2 * mt * Nt > 512 && rounds > 1) eff *= 0.8;               // no second accumulator buffer
       if (eff > best) { best = eff; MT = mt; }
     }
   }
@@ -781,33 +818,60 @@ static TcPlan make_plan(const Geom& g, int act_type, int variant) {
   }
   p.MT = MT;
   p.Rr = 128 * MT + p.halo;
+  const long long mgroups = (mtiles + MT - 1) / MT;
+  if (mgroups * p.n_ntiles > 0x7fffffffLL) return pl;
+  p.total_tiles = (int)(mgroups * p.n_ntiles);
+  // persistent grid: one CTA per SM, a multiple of the channel tiles so that a CTA keeps its channel tile
+  int grid = sms;
+  if (grid > p.total_tiles) grid = p.total_tiles;
+  if (grid >= p.n_ntiles) grid = grid / p.n_ntiles * p.n_ntiles;
+  const int tiles_per_cta = (p.total_tiles + grid - 1) / grid;
+  p.n_acc = (2 * MT * Nt <= 512 && tiles_per_cta > 1) ? 2 : 1;
   uint32_t cols = 32;
-  while (cols < (uint32_t)(MT * Nt)) cols *= 2;
+  while (cols < (uint32_t)(p.n_acc * MT * Nt)) cols *= 2;
   p.tmem_cols = cols;
-  // ---- shared-memory plan: activation block (all channels when they fit, else equal channel
-  // blocks), then weight stages as large as the budget allows (every stage costs the issuing
-  // thread a ~200-cycle wait plus bookkeeping, so few large stages beat many small ones).
+
+  // ---- shared memory: activation units, weight stages, epilogue tiles, tail
   const size_t per_chunk = (size_t)p.n_planes * p.Rr * 16;
-  const size_t a_full = (size_t)p.n_chunks * per_chunk;
   const size_t kstep_bytes = (size_t)2 * Nt * 16;                 // weights of one MMA
+  const size_t fixed = (size_t)EPI_BYTES + kSmemTail;
   const size_t stage_cap = (size_t)(want_stage_kb > 0 ? want_stage_kb : 48) * 1024;
-  size_t total_budget = (a_full + 2 * kstep_bytes * 4 + kSmemTail <= kSmemTwoPerSm) ? kSmemTwoPerSm : kSmemOnePerSm;
-  if (want_one) total_budget = kSmemOnePerSm;
+  // activation units: the whole of C in one unit when the wanted number of units and two small
+  // stages fit; else equal channel blocks, two of them in flight so that loading overlaps the MMAs
+  const int want_na = tiles_per_cta > 1 ? 2 : 1;
   int cb_chunks = p.n_chunks;
-  if (a_full + 2 * kstep_bytes * 2 + kSmemTail > total_budget) {
-    const size_t budget = total_budget - 2 * kstep_bytes * 2 - kSmemTail;
-    cb_chunks = (int)(budget / per_chunk) / 2 * 2;
-    while (cb_chunks >= 2 && (p.n_chunks % cb_chunks)) cb_chunks -= 2;
-    if (cb_chunks < 2) return pl;
+  {
+    if (kSmemBudget < fixed + 4 * kstep_bytes + 2 * per_chunk * 2) return pl;
+    const size_t room = kSmemBudget - fixed - 4 * kstep_bytes;
+    if ((size_t)want_na * p.n_chunks * per_chunk > room) {
+      cb_chunks = (int)(room / (2 * per_chunk)) / 2 * 2;
+      if (cb_chunks > p.n_chunks) cb_chunks = p.n_chunks;
+      while (cb_chunks >= 2 && (p.n_chunks % cb_chunks)) cb_chunks -= 2;
+      if (cb_chunks < 2) return pl;
+    }
+  }
+  if (int v = env_int("SNN_TC_CB", 0)) {
+    if (v >= 2 && v % 2 == 0 && p.n_chunks % v == 0 && v <= cb_chunks) cb_chunks = v;
   }
   p.cb_chunks = cb_chunks;
   p.n_cb = p.n_chunks / cb_chunks;
   p.kpt = cb_chunks / 2;
-  p.a_bytes = (uint32_t)(((size_t)cb_chunks * per_chunk + 127) & ~(size_t)127);
-  const size_t b_budget = total_budget - p.a_bytes - kSmemTail;
-  const size_t all_bytes = (size_t)9 * p.kpt * kstep_bytes;      // every weight of the block
-  size_t cap = stage_cap < b_budget / 2 ? stage_cap : b_budget / 2;  // at least two stages in flight
-  if (p.n_cb == 1 && all_bytes <= b_budget && all_bytes <= stage_cap) cap = all_bytes;  // everything in one stage
+  p.a_unit_bytes = (uint32_t)(((size_t)cb_chunks * per_chunk + 127) & ~(size_t)127);
+  int na = (p.n_cb > 1 || tiles_per_cta > 1) ? 2 : 1;
+  if (p.n_cb > 2 && (size_t)3 * p.a_unit_bytes + 8 * kstep_bytes + fixed <= kSmemBudget) na = 3;
+  if ((size_t)na * p.a_unit_bytes + 4 * kstep_bytes + fixed > kSmemBudget) na = 1;
+  if ((size_t)na * p.a_unit_bytes + 2 * kstep_bytes + fixed > kSmemBudget) return pl;
+  if (na > NA_MAX) na = NA_MAX;
+  p.NA = na;
+  const size_t b_budget = kSmemBudget - fixed - (size_t)na * p.a_unit_bytes;
+  const size_t all_bytes = (size_t)9 * (p.n_chunks / 2) * kstep_bytes;   // every weight of a channel tile
+  // resident weights: the CTA's channel tile never changes and its weights fit next to the rest
+  p.b_resident = 0;
+  if (p.n_cb == 1 && tiles_per_cta > 1 && grid % p.n_ntiles == 0 && all_bytes <= b_budget &&
+      !env_int("SNN_TC_NO_RESIDENT", 0))
+    p.b_resident = 1;
+  size_t cap = stage_cap < b_budget / 2 ? stage_cap : b_budget / 2;    // at least two stages in flight
+  if (p.b_resident) cap = stage_cap;
   int kmax = (int)(cap / kstep_bytes);
   if (kmax < 1) return pl;
   if (p.kpt <= kmax) {
@@ -824,30 +888,36 @@ static TcPlan make_plan(const Geom& g, int act_type, int variant) {
   }
   if (9 * (p.kpt / p.st_k) > kMaxSegs) return pl;
   p.stage_bytes = (uint32_t)((size_t)p.st_taps * p.st_k * kstep_bytes);
-  const int n_stages = p.n_cb * (9 / p.st_taps) * (p.kpt / p.st_k);
+  const int stages_per_tile = p.n_cb * (9 / p.st_taps) * (p.kpt / p.st_k);
   int ns = (int)(b_budget / p.stage_bytes);
   if (ns > NS_MAX) ns = NS_MAX;
-  if (ns > n_stages) ns = n_stages;
-  int forced_ns = env_int("SNN_TC_NS", 0);
-  if (forced_ns >= 1 && forced_ns <= ns) ns = forced_ns;
-  if (ns < 1 || (ns < 2 && n_stages > 1)) return pl;
+  if (p.b_resident) {
+    if (stages_per_tile > ns) p.b_resident = 0;
+    else ns = stages_per_tile;
+  }
+  if (!p.b_resident) {
+    const long long all_stages = (long long)stages_per_tile * tiles_per_cta;
+    if (ns > all_stages) ns = (int)all_stages;
+    int forced_ns = env_int("SNN_TC_NS", 0);
+    if (forced_ns >= 1 && forced_ns <= ns) ns = forced_ns;
+    if (ns < 1 || (ns < 2 && all_stages > 1)) return pl;
+  }
   p.NS = ns;
-  size_t ab = (size_t)p.a_bytes + (size_t)ns * p.stage_bytes;
-  if (ab < (size_t)EPI_BYTES) ab = EPI_BYTES;  // the epilogue's transposition tiles reuse these two regions
-  p.tail_off = (uint32_t)ab;
-  pl.smem = ab + kSmemTail;
+  p.off_b = (uint32_t)((size_t)na * p.a_unit_bytes);
+  p.off_epi = p.off_b + (uint32_t)((size_t)ns * p.stage_bytes);
+  p.off_tail = p.off_epi + EPI_BYTES;
+  pl.smem = (size_t)p.off_tail + kSmemTail;
   if (pl.smem > (size_t)kMaxDynSmem) return pl;
   if (pl.smem >= (1u << 18)) return pl;               // shared-memory descriptor address range
   if ((uint32_t)p.Rr * 16 >= (1u << 18)) return pl;   // leading-offset field range
-  if (p.stage_bytes >= (1u << 20)) return pl;         // mbarrier transaction-count range
-  long long gx = (mtiles + MT - 1) / MT;
-  if (gx > 0x7fffffffLL) return pl;
-  pl.grid = dim3((unsigned)gx, (unsigned)ntiles);
+  if (p.stage_bytes >= (1u << 20) || (size_t)p.n_planes * p.cb_chunks * p.Rr * 16 >= (1u << 20)) return pl;  // tx counts
+  pl.grid = dim3((unsigned)grid);
+  pl.xgrid = dim3((p.Qpad + 255) / 256, (unsigned)p.n_planes);
   pl.ok = true;
   return pl;
 }
 
-int tc_variant_count() { return 32; }
+int tc_variant_count() { return 16; }
 
 bool tc_supported(const Geom& g, int act_type) {
   if (env_int("SNN_TC_DISABLE", 0)) return false;
@@ -858,25 +928,38 @@ bool tc_supported(const Geom& g, int act_type) {
 
 bool tc_variant_ok(const Geom& g, int act_type, int variant) {
   if (variant < 0 || variant >= tc_variant_count()) return false;
-  // skip encodings that name nothing new
-  if (variant > 0 && (variant & 3) == 0) return false;
-  if (((variant >> 2) & 3) == 0 && variant > 3) return false;
+  if (variant > 0 && (variant & 3) == 0) return false;  // names no tile size
   return make_plan(g, act_type, variant).ok;
 }
 
-cudaError_t tc_forward(const LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched,
-                       int* status_dev, int variant) {
+cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched, int* status_dev,
+                       int variant) {
   TcPlan pl = make_plan(g, act_type, variant);
   if (!pl.ok) return cudaErrorInvalidConfiguration;
   const bool f16 = act_type == SNN_ACT_F16;
   TcParams& p = pl.p;
+  // scratch for the expanded activations: grows on demand, so that a shape's first call may
+  // allocate (not inside a stream capture) and later calls never do
+  if (pl.xa_bytes > L.tc_scratch_bytes) {
+    if (L.tc_scratch) cudaFree(L.tc_scratch);
+    L.tc_scratch = nullptr;
+    L.tc_scratch_bytes = 0;
+    cudaError_t ea = cudaMalloc(&L.tc_scratch, pl.xa_bytes);
+    if (ea != cudaSuccess) return ea;
+    L.tc_scratch_bytes = pl.xa_bytes;
+  }
   p.act = l.act;
+  p.xa = (uint8_t*)L.tc_scratch;
   p.wt = f16 ? (const uint8_t*)L.w16 : (const uint8_t*)L.w8;
   p.alpha = L.alpha;
   p.out = l.out;
   p.out_i32 = l.out_i32;
   p.status = status_dev;
-  cudaError_t e = cudaErrorInvalidConfiguration;
+  if (f16) tc_expand_act_kernel<true><<<pl.xgrid, 256, 0, l.stream>>>(p);
+  else tc_expand_act_kernel<false><<<pl.xgrid, 256, 0, l.stream>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  *launched += 1;
 #define SNN_TC_LAUNCH(F, M)                                                                    \
   do {                                                                                         \
     static unsigned long long done = 0;                                                        \
