@@ -9,19 +9,23 @@
 // Two kernels per forward call.
 //
 // 1. tc_expand_act_kernel writes the activations once, as tensor-core operands,
-//    into a scratch buffer the layer handle owns:  xa[plane][16-byte channel
-//    chunk][position][16 B]  (bits -> +1/-1 bytes, or fp16 copied), over a
-//    padded, flattened position space that keeps one zero column per row and
-//    one zero row per image (shared by neighbours), so that zero padding is a
-//    literal zero operand (a zero contributes 0, as the definition requires).
+//    into a scratch buffer the layer handle owns, already cut into the units the
+//    GEMM stages:  xa[position group][channel block][plane][16-byte channel
+//    chunk][row][16 B]  (bits -> +1/-1 bytes, or fp16 copied), over a padded,
+//    flattened position space that keeps one zero column per row and one zero
+//    row per image (shared by neighbours), so that zero padding is a literal
+//    zero operand (a zero contributes 0, as the definition requires).  Rows a
+//    group shares with its neighbour (the halo of the taps) are written twice.
 //    Stride 2 splits the padded input into its four row/column parity planes.
 //
-// 2. tc_conv_kernel is a persistent, warp-specialised GEMM.  Because a chunk's
-//    positions are contiguous in xa, the A operand of a tile is a handful of
-//    plain bulk copies into shared memory in the K-major, no-swizzle layout
-//    (rows 16 bytes apart), and the A operand of tap (ky, kx) is the same
-//    shared-memory block read from a start address shifted by ky*pitch + kx
-//    rows: the nine taps reuse one staged tile, there is no im2col copy.
+// 2. tc_conv_kernel is a persistent, warp-specialised GEMM.  A unit of xa is the
+//    shared-memory image of one (tile, channel block) of the A operand in the
+//    K-major, no-swizzle layout (rows 16 bytes apart), so it arrives with one
+//    bulk copy, and the A operand of tap (ky, kx) is that block read from a
+//    start address shifted by ky*pitch + kx rows: the nine taps reuse one
+//    staged unit, there is no im2col copy.  The K loop runs channel block by
+//    channel block (then taps, then chunks), so the MMAs of a tile start when
+//    its first block has landed.
 //      warp 0      one thread streams A units and weight stages (cp.async.bulk
 //                  onto mbarriers; rings of NA units and NS stages)
 //      warp 1      one thread issues tcgen05.mma into one of two TMEM
@@ -50,12 +54,10 @@ namespace {
 constexpr int TC_THREADS = 320;               // warp 0 producer, warp 1 MMA issue, warps 2-9 epilogue
 constexpr int EPI_WARPS = 8;
 constexpr int NS_MAX = 8;                     // most weight stages in flight
-constexpr int NA_MAX = 4;                     // most activation units in flight
 constexpr uint32_t WAIT_LIMIT = 1u << 20;     // try_wait attempts before a wait gives up
 constexpr int EPI_PITCH = 128;                // bytes per staged output row; 16-byte columns are XOR-swizzled by row
 constexpr int EPI_BYTES = EPI_WARPS * 32 * EPI_PITCH;
-constexpr int kMaxSegs = 192;                 // entries of the A-offset table
-constexpr size_t kSmemTail = 1280;            // barriers, flags, A-offset table
+constexpr size_t kSmemTail = 512;             // barriers, flags, tap offsets
 
 // Division by a run-time constant as multiply-high + shifts (round-up method,
 // exact for every 32-bit numerator).
@@ -79,8 +81,8 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t q, const FastDiv& f) {
 
 struct TcParams {
   const void* act;        // uint32 [N][H][W][Cw] or half [N][H][W][C]      (expansion kernel)
-  uint8_t* xa;            // expanded activations [plane][chunk][Qpad][16 B]  (scratch)
-  const uint8_t* wt;      // tiled weights: [layout tile][tap][chunk][NtL][16 B]
+  uint8_t* xa;            // expanded activations [group][block][plane][chunk][Rr][16 B]  (scratch)
+  const uint8_t* wt;      // tiled weights: [layout tile][block][tap][chunk][NtL][16 B]
   const float* alpha;
   void* out;
   int* status;            // mapped host word, set on a timed-out wait
@@ -93,12 +95,11 @@ struct TcParams {
   int n_planes;           // 1 (stride 1) or 4 (stride 2)
   int halo;               // largest tap shift in rows
   int Rr;                 // staged rows per plane = 128*MT + halo
-  uint32_t Qpad;          // positions per (plane, chunk) row of xa
+  int n_mgroups;          // position groups (tiles along M)
   int MT, Nt;             // M sub-tiles per tile, channels per tile
-  int cb_chunks, n_cb;    // chunks per activation unit (a channel block of one tile), units per tile
-  int kpt;                // MMAs per sub-tile and tap within a unit (= cb_chunks / 2)
-  int st_taps;            // taps per weight stage (1, 3 or 9; more than 1 only with one unit per tile)
-  int st_k;               // MMAs per sub-tile, tap and stage (= kpt when a stage holds whole taps)
+  int cb_chunks, n_cb;    // chunks per channel block (fixed when the layer is created), blocks
+  int kpt;                // MMAs per sub-tile and tap within a block (= cb_chunks / 2, at most 4)
+  int st_taps;            // taps per weight stage (1, 3 or 9)
   int NS, NA;             // weight stages / activation units in flight
   int n_acc;              // TMEM accumulator buffers (1 or 2)
   int b_resident;         // the whole weight set of the CTA's channel tile stays in the ring
@@ -294,66 +295,59 @@ __device__ __forceinline__ void epilogue_slice(const TcParams& p, uint32_t taddr
 }  // namespace
 
 // ------------------------------------------------------------------ expansion
-// One thread per (plane, position): all channel chunks of that position.  Reads
-// are contiguous per thread, writes are 16 bytes per thread with consecutive
-// threads on consecutive positions (coalesced).  Every row of xa is written,
-// padding and tail included, so the scratch never needs clearing.
+// One thread per (position group, row, plane, group of four 32-channel words).
+// Reads are contiguous per thread, writes are 16 bytes per thread with
+// consecutive threads on consecutive rows (coalesced).  Every row of every unit
+// is written, padding and tail included, so the scratch never needs clearing.
 template <bool F16>
 __global__ void __launch_bounds__(256) tc_expand_act_kernel(const TcParams p) {
-  const uint32_t q = blockIdx.x * 256u + threadIdx.x;
-  if (q >= p.Qpad) return;
+  const uint32_t row_id = blockIdx.x * 256u + threadIdx.x;  // (group, row)
+  if (row_id >= (uint32_t)p.n_mgroups * (uint32_t)p.Rr) return;
+  const uint32_t mg = row_id / (uint32_t)p.Rr;
+  const int r = (int)(row_id - mg * (uint32_t)p.Rr);
   const int pl = blockIdx.y, pa = pl >> 1, pb = pl & 1;
+  const uint32_t q = mg * (uint32_t)(128 * p.MT) + (uint32_t)r;
   const int pix = position_to_pixel(p, q, pa, pb);
-  uint4* dst = reinterpret_cast<uint4*>(p.xa) + (size_t)pl * p.n_chunks * p.Qpad + q;
-  if (F16) {
-    const __half* src = (const __half*)p.act + (size_t)(pix < 0 ? 0 : pix) * p.C;
-    const bool vec = pix >= 0 && ((p.C & 7) == 0);
-    for (int c = 0; c < p.n_chunks; ++c) {
-      uint4 v = make_uint4(0, 0, 0, 0);
-      const int ch = c * 8;
-      if (vec && ch + 8 <= p.C) {
-        v = __ldg(reinterpret_cast<const uint4*>(src + ch));
-      } else if (pix >= 0) {
-        uint32_t w[4] = {0, 0, 0, 0};
+  // chunk c of block cb lands at ((((mg*n_cb + cb)*n_planes + pl)*cb_chunks + c)*Rr + r)
+  uint4* base = reinterpret_cast<uint4*>(p.xa);
+  const int steps = p.n_chunks / 2;               // two chunks (32 int8 / 16 fp16 channels) per step
+  for (int st = blockIdx.z * 4; st < steps && st < blockIdx.z * 4 + 4; ++st) {
+    uint4 v[2];
+    if (F16) {
+      const __half* src = (const __half*)p.act + (size_t)(pix < 0 ? 0 : pix) * p.C;
+      const bool vec = pix >= 0 && ((p.C & 7) == 0);
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
-          if (ch + e < p.C) w[e >> 1] |= (uint32_t)__half_as_ushort(src[ch + e]) << (16 * (e & 1));
-        v = make_uint4(w[0], w[1], w[2], w[3]);
+      for (int k = 0; k < 2; ++k) {
+        v[k] = make_uint4(0, 0, 0, 0);
+        const int ch = (st * 2 + k) * 8;
+        if (vec && ch + 8 <= p.C) {
+          v[k] = __ldg(reinterpret_cast<const uint4*>(src + ch));
+        } else if (pix >= 0) {
+          uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            if (ch + e < p.C) w[e >> 1] |= (uint32_t)__half_as_ushort(src[ch + e]) << (16 * (e & 1));
+          v[k] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
       }
-      dst[(size_t)c * p.Qpad] = v;
+    } else {
+      // one 32-channel word -> two chunks of 16 int8 channels
+      uint32_t bits = 0;
+      if (pix >= 0 && st < p.Cw) bits = __ldg((const uint32_t*)p.act + (size_t)pix * p.Cw + st);
+      expand_word(bits, p.C - st * 32, pix >= 0 && st < p.Cw, v[0], v[1]);
     }
-  } else {
-    const uint32_t* src = (const uint32_t*)p.act + (size_t)(pix < 0 ? 0 : pix) * p.Cw;
-    const int nw = p.n_chunks / 2;
-    const bool vec_ok = (p.Cw & 3) == 0;
-    for (int wb = 0; wb < nw; wb += 4) {
-      uint32_t b[4] = {0, 0, 0, 0};
-      if (pix >= 0) {
-        if (vec_ok && wb + 4 <= p.Cw) {
-          const uint4 t = __ldg(reinterpret_cast<const uint4*>(src + wb));
-          b[0] = t.x; b[1] = t.y; b[2] = t.z; b[3] = t.w;
-        } else {
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            if (wb + k < p.Cw) b[k] = __ldg(src + wb + k);
-        }
-      }
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int wg = wb + k;
-        if (wg < nw) {
-          uint4 lo, hi;
-          expand_word(b[k], p.C - wg * 32, pix >= 0 && wg < p.Cw, lo, hi);
-          dst[(size_t)(2 * wg) * p.Qpad] = lo;
-          dst[(size_t)(2 * wg + 1) * p.Qpad] = hi;
-        }
-      }
+    for (int k = 0; k < 2; ++k) {
+      const int chunk = st * 2 + k;
+      const int cb = chunk / p.cb_chunks, c = chunk - cb * p.cb_chunks;
+      base[((((size_t)mg * p.n_cb + cb) * p.n_planes + pl) * p.cb_chunks + c) * p.Rr + r] = v[k];
     }
   }
 }
 
 // ------------------------------------------------------------------ GEMM
-template <bool F16, int MT>
+// KPT = MMAs per sub-tile and tap when known at compile time (2 or 4), 0 = read from the parameters
+template <bool F16, int MT, int KPT>
 __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   // carve-up: [NA activation units][NS weight stages][epilogue tiles][barriers, flags, table]
@@ -367,11 +361,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
   const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 28);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  uint32_t* seg_units = tmem_slot + 2;  // [9 * segs_per_tap] A row offset of every (tap, k-segment)
+  uint32_t* tap_units = tmem_slot + 2;  // [9] A row offset of every tap inside a unit
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int NS = p.NS, NA = p.NA;
-  const int segs_per_tap = p.kpt / p.st_k;
 
   if (tid < 28) {
     uint32_t count = 1;
@@ -379,16 +372,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
     mbar_init(smem_u32(bars + tid), count);
   }
   if (tid == 32) *abort_flag = 0;
-  for (int e = tid; e < 9 * segs_per_tap; e += TC_THREADS) {
-    // rows (16-byte units) from the unit's origin to (tap, k-segment): plane offset + tap shift
-    // inside the plane + the segment's first chunk
-    const int t = e / segs_per_tap, seg = e - t * segs_per_tap;
-    const int ky = t / 3, kx = t % 3;
+  if (tid >= 64 && tid < 73) {
+    // rows (16-byte units) from a unit's origin to tap t: plane offset + shift inside the plane
+    const int t = tid - 64, ky = t / 3, kx = t % 3;
     uint32_t u;
     if (p.stride == 1) u = (uint32_t)(ky * p.Wq + kx);
     else u = (uint32_t)((ky & 1) * 2 + (kx & 1)) * (uint32_t)(p.cb_chunks * p.Rr) +
              (uint32_t)((ky >> 1) * p.Wq + (kx >> 1));
-    seg_units[e] = u + (uint32_t)(seg * p.st_k * 2) * (uint32_t)p.Rr;
+    tap_units[t] = u;
   }
   if (warp == 2) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -402,8 +393,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // A weight stage holds st_taps whole taps, or st_k MMAs' worth of one tap.
-  const int stages_per_cb = (9 / p.st_taps) * segs_per_tap;
+  // A weight stage holds st_taps whole taps of one channel block.
+  const int stages_per_cb = 9 / p.st_taps;
   const uint32_t acc_cols = (uint32_t)(MT * p.Nt);
 
   if (warp == 0) {
@@ -413,15 +404,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       uint32_t a_phase = 1, b_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
       bool ok = true;
       bool first_tile = true;
-      const uint32_t unit_rows_bytes = (uint32_t)p.Rr * 16;
+      const uint32_t unit_bytes = (uint32_t)(p.n_planes * p.cb_chunks * p.Rr) * 16;  // exact bytes of a unit
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
         const int mg = tile / p.n_ntiles, nti = tile - mg * p.n_ntiles;
-        const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
         const int n0 = nti * p.Nt;
-        const size_t tile_base = (size_t)(n0 / p.NtL) * 9 * p.n_chunks;  // layout tile of these channels
+        const size_t wtile = (size_t)(n0 / p.NtL) * p.n_cb;   // layout tile of these channels, in blocks
         const int n_in = n0 % p.NtL;
         for (int cb = 0; cb < p.n_cb && ok; ++cb) {
-          // ---- activation unit: every (plane, chunk) of this channel block is one contiguous run of xa
+          // ---- activation unit (tile, channel block): one contiguous run of xa
           if (*abort_flag) { ok = false; break; }
           if (a_issued >= NA && !mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 32)) {
             *abort_flag = 1;
@@ -429,39 +419,28 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
             ok = false;
             break;
           }
-          mbar_expect_tx(bar_afull + 8 * a_slot, (uint32_t)(p.n_planes * p.cb_chunks) * unit_rows_bytes);
-          {
-            uint32_t dst = smem_u32(a_smem) + (uint32_t)a_slot * p.a_unit_bytes;
-            for (int pl = 0; pl < p.n_planes; ++pl) {
-              const uint8_t* src = p.xa + (((size_t)pl * p.n_chunks + (size_t)cb * p.cb_chunks) * p.Qpad + Q0) * 16;
-              for (int c = 0; c < p.cb_chunks; ++c) {
-                bulk_g2s(dst, src, unit_rows_bytes, bar_afull + 8 * a_slot);
-                dst += unit_rows_bytes;
-                src += (size_t)p.Qpad * 16;
-              }
-            }
-          }
+          mbar_expect_tx(bar_afull + 8 * a_slot, unit_bytes);
+          bulk_g2s(smem_u32(a_smem) + (uint32_t)a_slot * p.a_unit_bytes,
+                   p.xa + ((size_t)mg * p.n_cb + cb) * unit_bytes, unit_bytes, bar_afull + 8 * a_slot);
           ++a_issued;
           if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
           // ---- weight stages of this channel block (kept from the first tile on when resident)
           if (p.b_resident && !first_tile) continue;
-          for (int rem = 0; rem < stages_per_cb; ++rem) {
+          for (int sg = 0; sg < stages_per_cb; ++sg) {
             if (b_issued >= NS && !mbar_wait_backoff(bar_bempty + 8 * b_slot, b_phase, 32)) {
               *abort_flag = 1;
               raise_status(p.status, 2);
               ok = false;
               break;
             }
-            const int tg = rem / segs_per_tap, seg = rem - tg * segs_per_tap;
-            const int chunk0 = cb * p.cb_chunks + seg * p.st_k * 2;
             const uint32_t dst = smem_u32(b_smem) + (uint32_t)b_slot * p.stage_bytes;
             const uint8_t* src =
-                p.wt + ((tile_base + (size_t)(tg * p.st_taps) * p.n_chunks + chunk0) * p.NtL + n_in) * 16;
+                p.wt + ((((wtile + cb) * 9 + (size_t)sg * p.st_taps) * p.cb_chunks) * p.NtL + n_in) * 16;
             mbar_expect_tx(bar_bfull + 8 * b_slot, p.stage_bytes);
             if (p.Nt == p.NtL) {
-              bulk_g2s(dst, src, p.stage_bytes, bar_bfull + 8 * b_slot);  // consecutive (tap, chunk) blocks are contiguous
+              bulk_g2s(dst, src, p.stage_bytes, bar_bfull + 8 * b_slot);  // (tap, chunk) blocks are contiguous
             } else {
-              const int nchunk = p.st_taps * p.st_k * 2;
+              const int nchunk = p.st_taps * p.cb_chunks;
               for (int c = 0; c < nchunk; ++c)
                 bulk_g2s(dst + (uint32_t)c * p.Nt * 16, src + (size_t)c * p.NtL * 16, (uint32_t)p.Nt * 16,
                          bar_bfull + 8 * b_slot);
@@ -499,7 +478,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       const uint32_t stage_units = p.stage_bytes >> 4, unit_units = p.a_unit_bytes >> 4;
       const uint32_t a_step = 2u * (uint32_t)p.Rr, b_step = 2u * (uint32_t)p.Nt;  // two chunks per MMA
       const uint32_t nt = (uint32_t)p.Nt;
-      const int st_k = p.st_k, st_taps = p.st_taps;
+      const int kpt = KPT ? KPT : p.kpt, st_taps = p.st_taps;
       bool ok = true;
       int a_slot = 0, b_slot = 0, acc_slot = 0;
       uint32_t a_phase = 0, b_phase = 0, acc_phase = 1;
@@ -517,19 +496,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
           if (!mbar_wait(bar_afull + 8 * a_slot, a_phase)) { ok = false; break; }
           tc_fence_after();
           const uint64_t a_unit = a_desc0 + (uint64_t)((uint32_t)a_slot * unit_units);
-          int e = 0;  // index into seg_units
-          for (int rem = 0; rem < stages_per_cb; ++rem) {
+          int t = 0;
+          for (int sg = 0; sg < stages_per_cb; ++sg) {
             if (wait_b) {
               if (!mbar_wait(bar_bfull + 8 * b_slot, b_phase)) { ok = false; break; }
               tc_fence_after();
             }
             uint64_t bd = b_desc0 + (uint64_t)((uint32_t)b_slot * stage_units);
-            for (int tt = 0; tt < st_taps; ++tt, ++e) {
-              uint64_t ad = a_unit + (uint64_t)seg_units[e];
-              int k = 0;
-              for (; k + 4 <= st_k; k += 4) {
+            for (int tt = 0; tt < st_taps; ++tt, ++t) {
+              uint64_t ad = a_unit + (uint64_t)tap_units[t];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+              for (int k = 0; k < (KPT ? KPT : 4); ++k) {
+                if (KPT || k < kpt) {
 #pragma unroll
                   for (int mt = 0; mt < MT; ++mt)
                     mma_ss<F16>(d0 + (uint32_t)mt * nt, ad + (uint64_t)(mt * 128), bd, idesc, acc);
@@ -537,14 +515,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
                   ad += a_step;
                   bd += b_step;
                 }
-              }
-              for (; k < st_k; ++k) {
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt)
-                  mma_ss<F16>(d0 + (uint32_t)mt * nt, ad + (uint64_t)(mt * 128), bd, idesc, acc);
-                acc = 1;
-                ad += a_step;
-                bd += b_step;
               }
             }
             if (!p.b_resident) tc_commit(bar_bempty + 8 * b_slot);  // free once these MMAs have read it
@@ -619,22 +589,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
                   make_uint4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
             __syncwarp();
             if (co < p.K) {  // K is a multiple of 4 here, so the four channels exist together
+              // loads and conversions first, the (predicated) stores last: no branch sits between
+              // the eight independent chains, so their latencies overlap
+              uint4 u[8];
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 const int row = srow + 4 * i;
-                const uint4 u = *reinterpret_cast<const uint4*>(stage + row * EPI_PITCH + ((scol ^ (row & 7)) << 4));
-                if (ro[i] < 0) continue;
-                if (p.out_i32) {
-                  *reinterpret_cast<uint4*>((int32_t*)p.out + ro[i] + co) = u;
-                } else {
-                  float4 yv;
-                  yv.x = __fmul_rn(F16 ? __uint_as_float(u.x) : (float)(int)u.x, al.x);
-                  yv.y = __fmul_rn(F16 ? __uint_as_float(u.y) : (float)(int)u.y, al.y);
-                  yv.z = __fmul_rn(F16 ? __uint_as_float(u.z) : (float)(int)u.z, al.z);
-                  yv.w = __fmul_rn(F16 ? __uint_as_float(u.w) : (float)(int)u.w, al.w);
-                  *reinterpret_cast<float4*>((float*)p.out + ro[i] + co) = yv;
+                u[i] = *reinterpret_cast<const uint4*>(stage + row * EPI_PITCH + ((scol ^ (row & 7)) << 4));
+              }
+              if (!p.out_i32) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  u[i].x = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].x) : (float)(int)u[i].x, al.x));
+                  u[i].y = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].y) : (float)(int)u[i].y, al.y));
+                  u[i].z = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].z) : (float)(int)u[i].z, al.z));
+                  u[i].w = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].w) : (float)(int)u[i].w, al.w));
                 }
               }
+              uint32_t* obase32 = reinterpret_cast<uint32_t*>(p.out) + co;  // int32 and fp32 outputs share the layout
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                if (ro[i] >= 0) *reinterpret_cast<uint4*>(obase32 + ro[i]) = u[i];
             }
             __syncwarp();
           }
@@ -664,25 +639,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
 }
 
 // ------------------------------------------------------------ create-time operand
-// wt[layout tile][tap][chunk][NtL][16 B]: chunk = 16 (int8) or 8 (fp16) consecutive input
-// channels, NtL output channels per layout tile.  A CTA that owns a whole layout tile reads
-// every weight stage (consecutive chunks, consecutive taps) as one contiguous block.
+// wt[layout tile][channel block][tap][chunk][NtL][16 B]: chunk = 16 (int8) or 8 (fp16)
+// consecutive input channels, cb_chunks chunks per block, NtL output channels per layout tile.
+// A CTA that owns a whole layout tile reads every weight stage (consecutive taps of one channel
+// block) as one contiguous piece.
 template <bool F16>
 __global__ void tc_expand_weights_kernel(const uint32_t* __restrict__ wplanes, uint8_t* __restrict__ wt, int C, int K,
-                                         int Cw, int Kpad, int n_chunks, int NtL) {
+                                         int Cw, long long total, int cb_chunks, int n_cb, int NtL) {
   long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-  long long total = (long long)9 * n_chunks * Kpad;
   if (i >= total) return;
   int row = (int)(i % NtL);
   long long r = i / NtL;
-  int chunk = (int)(r % n_chunks);
-  r /= n_chunks;
-  int t = (int)(r % 9), tile = (int)(r / 9);
+  int c = (int)(r % cb_chunks);
+  r /= cb_chunks;
+  int t = (int)(r % 9);
+  r /= 9;
+  int cb = (int)(r % n_cb), tile = (int)(r / n_cb);
   int co = tile * NtL + row;
   const int cpc = F16 ? 8 : 16;
   uint4 v = make_uint4(0, 0, 0, 0);
   if (co < K) {
-    int ch0 = chunk * cpc;
+    int ch0 = (cb * cb_chunks + c) * cpc;
     int wd = ch0 >> 5, sh = ch0 & 31;
     uint32_t bits = wd < Cw ? wplanes[((size_t)t * Cw + wd) * K + co] >> sh : 0u;
     uint32_t w[4] = {0, 0, 0, 0};
@@ -705,26 +682,41 @@ static int round_up(int v, int m) { return (v + m - 1) / m * m; }
 // Layout tile of the weight operand: all channels when they fit one MMA (N <= 256), else 128.
 static int layout_tile(int K) { return K <= 256 ? round_up(K, 16) : 128; }
 
+// Channel blocks of the K loop: at most 8 chunks (128 int8 / 64 fp16 channels) each.  The
+// chunk count is even (an MMA consumes two); when no block size in 4..8 divides it, the
+// channels are padded with zeros to a multiple of 8 chunks.
+static void channel_blocks(int C, bool f16, int* n_chunks, int* cb_chunks) {
+  const int cpc = f16 ? 8 : 16;
+  const int raw = round_up(C, 2 * cpc) / cpc;
+  if (raw <= 8) { *n_chunks = raw; *cb_chunks = raw; return; }
+  for (int d = 8; d >= 4; d -= 2)
+    if (raw % d == 0) { *n_chunks = raw; *cb_chunks = d; return; }
+  *n_chunks = round_up(raw, 8);
+  *cb_chunks = 8;
+}
+
 size_t tc_weight_bytes(const Geom& g, int act_type, int* Kpad, int* Cpad) {
   const bool f16 = act_type == SNN_ACT_F16;
+  int n_chunks, cb;
+  channel_blocks(g.C, f16, &n_chunks, &cb);
   *Kpad = round_up(g.K, layout_tile(g.K));
-  *Cpad = round_up(g.C, f16 ? 16 : 32);
-  const int n_chunks = *Cpad / (f16 ? 8 : 16);
+  *Cpad = n_chunks * (f16 ? 8 : 16);
   return (size_t)9 * n_chunks * (*Kpad) * 16;
 }
 
 cudaError_t tc_expand_weights(const LayerDev& L, const Geom& g, int act_type, cudaStream_t s, int* launched) {
   const bool f16 = act_type == SNN_ACT_F16;
-  const int n_chunks = L.Cpad / (f16 ? 8 : 16);
-  long long total = (long long)9 * n_chunks * L.Kpad;
+  int n_chunks, cb;
+  channel_blocks(g.C, f16, &n_chunks, &cb);
+  const long long total = (long long)9 * n_chunks * L.Kpad;
   unsigned blocks = (unsigned)((total + 255) / 256);
   const int NtL = layout_tile(g.K);
   if (f16)
-    tc_expand_weights_kernel<true><<<blocks, 256, 0, s>>>(L.wplanes, (uint8_t*)L.w16, g.C, g.K, g.Cw, L.Kpad, n_chunks,
-                                                         NtL);
+    tc_expand_weights_kernel<true><<<blocks, 256, 0, s>>>(L.wplanes, (uint8_t*)L.w16, g.C, g.K, g.Cw, total, cb,
+                                                         n_chunks / cb, NtL);
   else
-    tc_expand_weights_kernel<false><<<blocks, 256, 0, s>>>(L.wplanes, (uint8_t*)L.w8, g.C, g.K, g.Cw, L.Kpad, n_chunks,
-                                                          NtL);
+    tc_expand_weights_kernel<false><<<blocks, 256, 0, s>>>(L.wplanes, (uint8_t*)L.w8, g.C, g.K, g.Cw, total, cb,
+                                                          n_chunks / cb, NtL);
   *launched += 1;
   return cudaGetLastError();
 }
@@ -736,6 +728,7 @@ struct TcPlan {
   size_t xa_bytes;
   dim3 grid, xgrid;
   bool ok;
+  double score;
 };
 
 static int env_int(const char* name, int dflt) {
@@ -755,29 +748,21 @@ static int sm_count() {
 
 constexpr size_t kSmemBudget = 226 * 1024;
 
-// variant: 0 = heuristic; otherwise mt_code (1..3 -> 1,2,4) + 4*stage_code (0..3 -> 48,16,32,64 KB)
-static TcPlan make_plan(const Geom& g, int act_type, int variant) {
+// Everything that follows from a choice of sub-tiles per tile (MT) and weight-stage size.
+static TcPlan plan_for(const Geom& g, int act_type, int MT, int stage_kb) {
   TcPlan pl{};
   TcParams& p = pl.p;
   const bool f16 = act_type == SNN_ACT_F16;
   pl.ok = false;
-  if (g.N < 1) return pl;
-  int want_mt = 0, want_stage_kb = 0;
-  if (variant > 0) {
-    static const int mts[4] = {0, 1, 2, 4};
-    static const int kbs[4] = {0, 16, 32, 64};
-    want_mt = mts[variant & 3];
-    want_stage_kb = kbs[(variant >> 2) & 3];
-  }
-  if (int v = env_int("SNN_TC_MT", 0)) want_mt = v;
-  if (int v = env_int("SNN_TC_STAGE_KB", 0)) want_stage_kb = v;
   int Kpad, Cpad;
   tc_weight_bytes(g, act_type, &Kpad, &Cpad);
   p.N = g.N; p.H = g.H; p.W = g.W; p.C = g.C; p.K = g.K; p.Cw = g.Cw;
   p.stride = g.stride; p.pad = g.pad; p.Ho = g.Ho; p.Wo = g.Wo;
   p.Kpad = Kpad;
   p.NtL = layout_tile(g.K);
-  p.n_chunks = Cpad / (f16 ? 8 : 16);
+  channel_blocks(g.C, f16, &p.n_chunks, &p.cb_chunks);
+  p.n_cb = p.n_chunks / p.cb_chunks;
+  p.kpt = p.cb_chunks / 2;
   if (g.stride == 1) {
     p.Hq = g.H + g.pad; p.Wq = g.W + g.pad; p.n_planes = 1; p.halo = 2 * p.Wq + 2;
   } else {
@@ -788,8 +773,6 @@ static TcPlan make_plan(const Geom& g, int act_type, int variant) {
   p.Qtot = (long long)g.N * p.Hq * p.Wq;
   if (p.Qtot + 1024 + p.halo >= (1ll << 31)) return pl;  // positions are 32-bit in the kernels
   if ((long long)g.N * g.H * g.W >= (1ll << 31)) return pl;
-  p.Qpad = (uint32_t)((p.Qtot + 511) / 512 * 512 + ((p.halo + 15) / 16 * 16));  // any tile's rows exist
-  pl.xa_bytes = (size_t)p.n_planes * p.n_chunks * p.Qpad * 16;
   const long long mtiles = (p.Qtot + 127) / 128;
   const int sms = sm_count();
   // channels per tile: a layout tile, or a part of one on request
@@ -798,28 +781,12 @@ static TcPlan make_plan(const Geom& g, int act_type, int variant) {
   if (forced_nt >= 16 && forced_nt <= 256 && forced_nt % 16 == 0 && p.NtL % forced_nt == 0) Nt = forced_nt;
   p.Nt = Nt;
   p.n_ntiles = Kpad / Nt;
-  // M sub-tiles per tile: large tiles stage less halo, small tiles balance the SMs better
-  int MT = 1;
-  {
-    double best = -1.0;
-    for (int mt = 1; mt <= 4; mt *= 2) {
-      if (mt * Nt > 512) break;
-      long long tiles = ((mtiles + mt - 1) / mt) * p.n_ntiles;
-      long long rounds = (tiles + sms - 1) / sms;
-      double eff = (double)tiles / (double)(rounds * sms);          // load balance of the persistent CTAs
-      eff *= (double)(128 * mt) / (double)(128 * mt + p.halo);       // useful share of the staged rows
-      if (2 * mt * Nt > 512 && rounds > 1) eff *= 0.8;               // no second accumulator buffer
-      if (eff > best) { best = eff; MT = mt; }
-    }
-  }
-  if (want_mt == 1 || want_mt == 2 || want_mt == 4) {
-    if (want_mt * Nt > 512) return pl;
-    MT = want_mt;
-  }
+  if (MT * Nt > 512) return pl;
   p.MT = MT;
   p.Rr = 128 * MT + p.halo;
   const long long mgroups = (mtiles + MT - 1) / MT;
-  if (mgroups * p.n_ntiles > 0x7fffffffLL) return pl;
+  if (mgroups * p.n_ntiles > 0x7fffffffLL || mgroups * p.Rr >= (1ll << 31)) return pl;
+  p.n_mgroups = (int)mgroups;
   p.total_tiles = (int)(mgroups * p.n_ntiles);
   // persistent grid: one CTA per SM, a multiple of the channel tiles so that a CTA keeps its channel tile
   int grid = sms;
@@ -832,63 +799,31 @@ static TcPlan make_plan(const Geom& g, int act_type, int variant) {
   p.tmem_cols = cols;
 
   // ---- shared memory: activation units, weight stages, epilogue tiles, tail
-  const size_t per_chunk = (size_t)p.n_planes * p.Rr * 16;
-  const size_t kstep_bytes = (size_t)2 * Nt * 16;                 // weights of one MMA
+  const size_t unit_exact = (size_t)p.n_planes * p.cb_chunks * p.Rr * 16;
+  p.a_unit_bytes = (uint32_t)((unit_exact + 127) & ~(size_t)127);
+  const size_t kstep_bytes = (size_t)2 * Nt * 16;        // weights of one MMA
+  const size_t tap_bytes = (size_t)p.kpt * kstep_bytes;  // weights of one tap of one channel block
   const size_t fixed = (size_t)EPI_BYTES + kSmemTail;
-  const size_t stage_cap = (size_t)(want_stage_kb > 0 ? want_stage_kb : 48) * 1024;
-  // activation units: the whole of C in one unit when the wanted number of units and two small
-  // stages fit; else equal channel blocks, two of them in flight so that loading overlaps the MMAs
-  const int want_na = tiles_per_cta > 1 ? 2 : 1;
-  int cb_chunks = p.n_chunks;
-  {
-    if (kSmemBudget < fixed + 4 * kstep_bytes + 2 * per_chunk * 2) return pl;
-    const size_t room = kSmemBudget - fixed - 4 * kstep_bytes;
-    if ((size_t)want_na * p.n_chunks * per_chunk > room) {
-      cb_chunks = (int)(room / (2 * per_chunk)) / 2 * 2;
-      if (cb_chunks > p.n_chunks) cb_chunks = p.n_chunks;
-      while (cb_chunks >= 2 && (p.n_chunks % cb_chunks)) cb_chunks -= 2;
-      if (cb_chunks < 2) return pl;
-    }
-  }
-  if (int v = env_int("SNN_TC_CB", 0)) {
-    if (v >= 2 && v % 2 == 0 && p.n_chunks % v == 0 && v <= cb_chunks) cb_chunks = v;
-  }
-  p.cb_chunks = cb_chunks;
-  p.n_cb = p.n_chunks / cb_chunks;
-  p.kpt = cb_chunks / 2;
-  p.a_unit_bytes = (uint32_t)(((size_t)cb_chunks * per_chunk + 127) & ~(size_t)127);
-  int na = (p.n_cb > 1 || tiles_per_cta > 1) ? 2 : 1;
-  if (p.n_cb > 2 && (size_t)3 * p.a_unit_bytes + 8 * kstep_bytes + fixed <= kSmemBudget) na = 3;
-  if ((size_t)na * p.a_unit_bytes + 4 * kstep_bytes + fixed > kSmemBudget) na = 1;
-  if ((size_t)na * p.a_unit_bytes + 2 * kstep_bytes + fixed > kSmemBudget) return pl;
-  if (na > NA_MAX) na = NA_MAX;
+  const size_t stage_cap = (size_t)(stage_kb > 0 ? stage_kb : 48) * 1024;
+  const long long units_per_cta = (long long)tiles_per_cta * p.n_cb;
+  int na = units_per_cta >= 3 && p.n_cb >= 2 ? 3 : (units_per_cta >= 2 ? 2 : 1);
+  while (na > 1 && (size_t)na * p.a_unit_bytes + 2 * tap_bytes + fixed > kSmemBudget) --na;
+  if ((size_t)na * p.a_unit_bytes + tap_bytes + fixed > kSmemBudget) return pl;
   p.NA = na;
   const size_t b_budget = kSmemBudget - fixed - (size_t)na * p.a_unit_bytes;
-  const size_t all_bytes = (size_t)9 * (p.n_chunks / 2) * kstep_bytes;   // every weight of a channel tile
+  const size_t all_bytes = (size_t)9 * p.n_cb * tap_bytes;  // every weight of a channel tile
   // resident weights: the CTA's channel tile never changes and its weights fit next to the rest
   p.b_resident = 0;
   if (p.n_cb == 1 && tiles_per_cta > 1 && grid % p.n_ntiles == 0 && all_bytes <= b_budget &&
       !env_int("SNN_TC_NO_RESIDENT", 0))
     p.b_resident = 1;
-  size_t cap = stage_cap < b_budget / 2 ? stage_cap : b_budget / 2;    // at least two stages in flight
+  size_t cap = stage_cap < b_budget / 2 ? stage_cap : b_budget / 2;  // at least two stages in flight
   if (p.b_resident) cap = stage_cap;
-  int kmax = (int)(cap / kstep_bytes);
-  if (kmax < 1) return pl;
-  if (p.kpt <= kmax) {
-    p.st_k = p.kpt;
-    p.st_taps = 1;
-    if (p.n_cb == 1) {
-      if (9 * p.kpt <= kmax) p.st_taps = 9;
-      else if (3 * p.kpt <= kmax) p.st_taps = 3;
-    }
-  } else {
-    p.st_taps = 1;
-    p.st_k = kmax;
-    while (p.kpt % p.st_k) --p.st_k;
-  }
-  if (9 * (p.kpt / p.st_k) > kMaxSegs) return pl;
-  p.stage_bytes = (uint32_t)((size_t)p.st_taps * p.st_k * kstep_bytes);
-  const int stages_per_tile = p.n_cb * (9 / p.st_taps) * (p.kpt / p.st_k);
+  if (cap < tap_bytes) cap = tap_bytes <= b_budget ? tap_bytes : 0;
+  if (cap == 0) return pl;
+  p.st_taps = 9 * tap_bytes <= cap ? 9 : (3 * tap_bytes <= cap ? 3 : 1);
+  p.stage_bytes = (uint32_t)((size_t)p.st_taps * tap_bytes);
+  const int stages_per_tile = p.n_cb * (9 / p.st_taps);
   int ns = (int)(b_budget / p.stage_bytes);
   if (ns > NS_MAX) ns = NS_MAX;
   if (p.b_resident) {
@@ -900,7 +835,7 @@ static TcPlan make_plan(const Geom& g, int act_type, int variant) {
     if (ns > all_stages) ns = (int)all_stages;
     int forced_ns = env_int("SNN_TC_NS", 0);
     if (forced_ns >= 1 && forced_ns <= ns) ns = forced_ns;
-    if (ns < 1 || (ns < 2 && all_stages > 1)) return pl;
+    if (ns < 1) return pl;
   }
   p.NS = ns;
   p.off_b = (uint32_t)((size_t)na * p.a_unit_bytes);
@@ -910,11 +845,43 @@ static TcPlan make_plan(const Geom& g, int act_type, int variant) {
   if (pl.smem > (size_t)kMaxDynSmem) return pl;
   if (pl.smem >= (1u << 18)) return pl;               // shared-memory descriptor address range
   if ((uint32_t)p.Rr * 16 >= (1u << 18)) return pl;   // leading-offset field range
-  if (p.stage_bytes >= (1u << 20) || (size_t)p.n_planes * p.cb_chunks * p.Rr * 16 >= (1u << 20)) return pl;  // tx counts
+  if (p.stage_bytes >= (1u << 20) || unit_exact >= (1u << 20)) return pl;  // mbarrier transaction counts
+  pl.xa_bytes = (size_t)mgroups * p.n_cb * unit_exact;
   pl.grid = dim3((unsigned)grid);
-  pl.xgrid = dim3((p.Qpad + 255) / 256, (unsigned)p.n_planes);
+  const long long xrows = mgroups * p.Rr;
+  pl.xgrid = dim3((unsigned)((xrows + 255) / 256), (unsigned)p.n_planes, (unsigned)((p.n_chunks / 2 + 3) / 4));
+  // heuristic score: balance of the persistent CTAs x useful share of the staged rows
+  const long long rounds = tiles_per_cta;
+  double eff = (double)p.total_tiles / (double)(rounds * grid) * (double)grid / (double)sms;
+  eff *= (double)(128 * MT) / (double)(128 * MT + p.halo);
+  if (p.n_acc == 1 && rounds > 1) eff *= 0.8;   // epilogue cannot overlap the next tile's MMAs
+  if (p.b_resident) eff *= 1.1;
+  pl.score = eff;
   pl.ok = true;
   return pl;
+}
+
+// variant: 0 = heuristic; otherwise mt_code (1..3 -> 1,2,4) + 4*stage_code (0..3 -> 48,16,32,64 KB)
+static TcPlan make_plan(const Geom& g, int act_type, int variant) {
+  TcPlan none{};
+  none.ok = false;
+  if (g.N < 1) return none;
+  int want_mt = 0, want_stage_kb = 0;
+  if (variant > 0) {
+    static const int mts[4] = {0, 1, 2, 4};
+    static const int kbs[4] = {0, 16, 32, 64};
+    want_mt = mts[variant & 3];
+    want_stage_kb = kbs[(variant >> 2) & 3];
+  }
+  if (int v = env_int("SNN_TC_MT", 0)) want_mt = v;
+  if (int v = env_int("SNN_TC_STAGE_KB", 0)) want_stage_kb = v;
+  if (want_mt == 1 || want_mt == 2 || want_mt == 4) return plan_for(g, act_type, want_mt, want_stage_kb);
+  TcPlan best = none;
+  for (int mt = 1; mt <= 4; mt *= 2) {
+    TcPlan c = plan_for(g, act_type, mt, want_stage_kb);
+    if (c.ok && (!best.ok || c.score > best.score)) best = c;
+  }
+  return best;
 }
 
 int tc_variant_count() { return 16; }
@@ -960,21 +927,28 @@ cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   *launched += 1;
-#define SNN_TC_LAUNCH(F, M)                                                                    \
-  do {                                                                                         \
-    static unsigned long long done = 0;                                                        \
-    e = allow_max_smem(tc_conv_kernel<F, M>, &done);                                           \
-    if (e == cudaSuccess) tc_conv_kernel<F, M><<<pl.grid, TC_THREADS, pl.smem, l.stream>>>(p); \
+#define SNN_TC_LAUNCH(F, M, KP)                                                                    \
+  do {                                                                                             \
+    static unsigned long long done = 0;                                                            \
+    e = allow_max_smem(tc_conv_kernel<F, M, KP>, &done);                                           \
+    if (e == cudaSuccess) tc_conv_kernel<F, M, KP><<<pl.grid, TC_THREADS, pl.smem, l.stream>>>(p); \
+  } while (0)
+#define SNN_TC_LAUNCH_K(F, M)                 \
+  do {                                        \
+    if (p.kpt == 4) SNN_TC_LAUNCH(F, M, 4);   \
+    else if (p.kpt == 2) SNN_TC_LAUNCH(F, M, 2); \
+    else SNN_TC_LAUNCH(F, M, 0);              \
   } while (0)
   if (f16) {
-    if (p.MT == 1) SNN_TC_LAUNCH(true, 1);
-    else if (p.MT == 2) SNN_TC_LAUNCH(true, 2);
-    else SNN_TC_LAUNCH(true, 4);
+    if (p.MT == 1) SNN_TC_LAUNCH_K(true, 1);
+    else if (p.MT == 2) SNN_TC_LAUNCH_K(true, 2);
+    else SNN_TC_LAUNCH_K(true, 4);
   } else {
-    if (p.MT == 1) SNN_TC_LAUNCH(false, 1);
-    else if (p.MT == 2) SNN_TC_LAUNCH(false, 2);
-    else SNN_TC_LAUNCH(false, 4);
+    if (p.MT == 1) SNN_TC_LAUNCH_K(false, 1);
+    else if (p.MT == 2) SNN_TC_LAUNCH_K(false, 2);
+    else SNN_TC_LAUNCH_K(false, 4);
   }
+#undef SNN_TC_LAUNCH_K
 #undef SNN_TC_LAUNCH
   if (e != cudaSuccess) return e;
   *launched += 1;
