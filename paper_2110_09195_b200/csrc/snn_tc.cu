@@ -165,6 +165,13 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// Programmatic dependent launch: a kernel launched with the serialization attribute may start
+// while its predecessor in the stream still runs; grid_dep_wait() blocks until the predecessor has
+// completed and its writes are visible (a no-op for an ordinary launch), grid_dep_launch() lets the
+// successor start being scheduled.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Shared-memory matrix descriptor, K-major, no swizzle: rows 16 B apart inside an
 // 8-row group, groups `sbo` bytes apart, the two 16-byte K chunks `lbo` bytes apart.
 __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
@@ -301,6 +308,8 @@ __device__ __forceinline__ void epilogue_slice(const TcParams& p, uint32_t taddr
 // is written, padding and tail included, so the scratch never needs clearing.
 template <bool F16>
 __global__ void __launch_bounds__(256) tc_expand_act_kernel(const TcParams p) {
+  grid_dep_launch();  // the GEMM may set itself up (barriers, TMEM, weight prefetch) meanwhile
+  grid_dep_wait();    // the activations, and the scratch a previous GEMM may still read, are ready
   const uint32_t row_id = blockIdx.x * 256u + threadIdx.x;  // (group, row)
   if (row_id >= (uint32_t)p.n_mgroups * (uint32_t)p.Rr) return;
   const uint32_t mg = row_id / (uint32_t)p.Rr;
@@ -392,9 +401,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  grid_dep_launch();  // the next kernel in the stream may be scheduled; it waits for this grid to finish
 
   // A weight stage holds st_taps whole taps of one channel block.
   const int stages_per_cb = 9 / p.st_taps;
+  const int stages_per_tile = p.n_cb * stages_per_cb;
   const uint32_t acc_cols = (uint32_t)(MT * p.Nt);
 
   if (warp == 0) {
@@ -405,11 +416,47 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       bool ok = true;
       bool first_tile = true;
       const uint32_t unit_bytes = (uint32_t)(p.n_planes * p.cb_chunks * p.Rr) * 16;  // exact bytes of a unit
-      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-        const int mg = tile / p.n_ntiles, nti = tile - mg * p.n_ntiles;
+      // Weight stages are issued in the order the MMAs consume them; `w_next` counts the stages
+      // already requested, so that the first ones can be requested before the expanded
+      // activations exist (the weights are constants of the layer).
+      long long w_next = 0;
+      auto issue_weights = [&](int tile, long long upto) -> bool {
+        // requests stages [w_next, upto) of this CTA's stage sequence, stopping when the ring is full
+        const int nti = tile % p.n_ntiles;
         const int n0 = nti * p.Nt;
-        const size_t wtile = (size_t)(n0 / p.NtL) * p.n_cb;   // layout tile of these channels, in blocks
+        const size_t wtile = (size_t)(n0 / p.NtL) * p.n_cb;
         const int n_in = n0 % p.NtL;
+        while (w_next < upto) {
+          const int in_tile = (int)(w_next % stages_per_tile);
+          const int cb = in_tile / stages_per_cb, sg = in_tile - cb * stages_per_cb;
+          if (b_issued >= NS && !mbar_wait_backoff(bar_bempty + 8 * b_slot, b_phase, 32)) return false;
+          const uint32_t dst = smem_u32(b_smem) + (uint32_t)b_slot * p.stage_bytes;
+          const uint8_t* src =
+              p.wt + ((((wtile + cb) * 9 + (size_t)sg * p.st_taps) * p.cb_chunks) * p.NtL + n_in) * 16;
+          mbar_expect_tx(bar_bfull + 8 * b_slot, p.stage_bytes);
+          if (p.Nt == p.NtL) {
+            bulk_g2s(dst, src, p.stage_bytes, bar_bfull + 8 * b_slot);  // (tap, chunk) blocks are contiguous
+          } else {
+            const int nchunk = p.st_taps * p.cb_chunks;
+            for (int c = 0; c < nchunk; ++c)
+              bulk_g2s(dst + (uint32_t)c * p.Nt * 16, src + (size_t)c * p.NtL * 16, (uint32_t)p.Nt * 16,
+                       bar_bfull + 8 * b_slot);
+          }
+          ++b_issued;
+          ++w_next;
+          if (++b_slot == NS) { b_slot = 0; b_phase ^= 1u; }
+        }
+        return true;
+      };
+      // before the activations are there: as many weight stages of the first tile as the ring holds
+      if ((int)blockIdx.x < p.total_tiles) {
+        const long long first = stages_per_tile < NS ? stages_per_tile : NS;
+        issue_weights(blockIdx.x, first);
+      }
+      grid_dep_wait();  // the expansion kernel's writes to xa are complete and visible
+      long long tiles_seen = 0;
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tiles_seen) {
+        const int mg = tile / p.n_ntiles;
         for (int cb = 0; cb < p.n_cb && ok; ++cb) {
           // ---- activation unit (tile, channel block): one contiguous run of xa
           if (*abort_flag) { ok = false; break; }
@@ -426,27 +473,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
           if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
           // ---- weight stages of this channel block (kept from the first tile on when resident)
           if (p.b_resident && !first_tile) continue;
-          for (int sg = 0; sg < stages_per_cb; ++sg) {
-            if (b_issued >= NS && !mbar_wait_backoff(bar_bempty + 8 * b_slot, b_phase, 32)) {
-              *abort_flag = 1;
-              raise_status(p.status, 2);
-              ok = false;
-              break;
-            }
-            const uint32_t dst = smem_u32(b_smem) + (uint32_t)b_slot * p.stage_bytes;
-            const uint8_t* src =
-                p.wt + ((((wtile + cb) * 9 + (size_t)sg * p.st_taps) * p.cb_chunks) * p.NtL + n_in) * 16;
-            mbar_expect_tx(bar_bfull + 8 * b_slot, p.stage_bytes);
-            if (p.Nt == p.NtL) {
-              bulk_g2s(dst, src, p.stage_bytes, bar_bfull + 8 * b_slot);  // (tap, chunk) blocks are contiguous
-            } else {
-              const int nchunk = p.st_taps * p.cb_chunks;
-              for (int c = 0; c < nchunk; ++c)
-                bulk_g2s(dst + (uint32_t)c * p.Nt * 16, src + (size_t)c * p.NtL * 16, (uint32_t)p.Nt * 16,
-                         bar_bfull + 8 * b_slot);
-            }
-            ++b_issued;
-            if (++b_slot == NS) { b_slot = 0; b_phase ^= 1u; }
+          if (!issue_weights(tile, tiles_seen * stages_per_tile + (long long)(cb + 1) * stages_per_cb)) {
+            *abort_flag = 1;
+            raise_status(p.status, 2);
+            ok = false;
+            break;
           }
         }
         first_tile = false;
@@ -534,6 +565,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
     __syncwarp();
   } else {
     // ------------------------------------------------ epilogue warps
+    grid_dep_wait();  // an earlier kernel in the stream may still read the output buffer
     // Warp w reads TMEM lanes 32*(w%4).. (rows of the tile); the two warps of a lane quarter
     // split the 32-column slices between them.  A slice goes through a per-warp shared-memory
     // tile so that each store instruction writes whole 128-byte rows.
@@ -560,65 +592,89 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       }
       tc_fence_after();
       const uint32_t d0 = tmem_base + (uint32_t)acc_slot * acc_cols;
-#pragma unroll 1
-      for (int mt = 0; mt < MT; ++mt) {
+      // row of sub-tile mt this lane owns in TMEM -> is it an output, and where does it go
+      auto row_info = [&](int mt, bool* valid, size_t* obase) {
         const uint32_t q = Q0 + (uint32_t)(mt * 128 + rq * 32 + lane);
         const uint32_t rg = fdiv(q, p.dWq);
         const int x = (int)(q - rg * (uint32_t)p.Wq);
         const uint32_t n = fdiv(rg, p.dHq);
         const int y = (int)(rg - n * (uint32_t)p.Hq);
-        const bool valid = ((long long)q < p.Qtot) && ((int)n < p.N) && (y < p.Ho) && (x < p.Wo);
-        const size_t obase = (((size_t)n * p.Ho + y) * p.Wo + x) * p.K;
-        const uint32_t trow = d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt);
-        if (fast) {
-          // element offsets of the eight rows this lane stores (row = srow + 4*i), -1 when not an output
-          long long ro[8];
-          const long long mine = valid ? (long long)obase : -1;
+        *valid = ((long long)q < p.Qtot) && ((int)n < p.N) && (y < p.Ho) && (x < p.Wo);
+        *obase = (((size_t)n * p.Ho + y) * p.Wo + x) * p.K;
+      };
+      if (fast) {
+        // The warp's slices (sub-tile mt, columns c0..c0+31) form one sequence.  The TMEM load of
+        // slice s+1 is issued as soon as slice s sits in the staging tile, so it flies while
+        // slice s is converted and stored, and the store path never waits for a TMEM load.
+        const int per_mt = (p.Nt - 32 * half + 63) / 64;
+        const int total = MT * per_mt;
+        uint32_t v[32];
+        long long ro[8];
+        if (total > 0) tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(32 * half), v);
+#pragma unroll 1
+        for (int sl = 0; sl < total; ++sl) {
+          const int mt = sl / per_mt, c0 = 32 * half + 64 * (sl - mt * per_mt);
+          if (sl - mt * per_mt == 0) {
+            // element offsets of the eight rows this lane stores (row = srow + 4*i), -1 when not an output
+            bool valid;
+            size_t obase;
+            row_info(mt, &valid, &obase);
+            const long long mine = valid ? (long long)obase : -1;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) ro[i] = __shfl_sync(0xffffffffu, mine, srow + 4 * i);
-          for (int c0 = 32 * half; c0 < p.Nt; c0 += 64) {
-            uint32_t v[32];
-            tmem_ld32(trow + (uint32_t)c0, v);
-            const int co = n0 + c0 + scol * 4;
-            float4 al = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (!p.out_i32 && co < p.K) al = __ldg(reinterpret_cast<const float4*>(p.alpha + co));
-            tmem_ld_wait();
+            for (int i = 0; i < 8; ++i) ro[i] = __shfl_sync(0xffffffffu, mine, srow + 4 * i);
+          }
+          const int co = n0 + c0 + scol * 4;
+          float4 al = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (!p.out_i32 && co < p.K) al = __ldg(reinterpret_cast<const float4*>(p.alpha + co));
+          tmem_ld_wait();
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-              *reinterpret_cast<uint4*>(stage + lane * EPI_PITCH + ((e ^ (lane & 7)) << 4)) =
-                  make_uint4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
-            __syncwarp();
-            if (co < p.K) {  // K is a multiple of 4 here, so the four channels exist together
-              // loads and conversions first, the (predicated) stores last: no branch sits between
-              // the eight independent chains, so their latencies overlap
-              uint4 u[8];
+          for (int e = 0; e < 8; ++e)
+            *reinterpret_cast<uint4*>(stage + lane * EPI_PITCH + ((e ^ (lane & 7)) << 4)) =
+                make_uint4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+          __syncwarp();
+          if (sl + 1 < total) {
+            const int nmt = (sl + 1) / per_mt, nc0 = 32 * half + 64 * (sl + 1 - nmt * per_mt);
+            tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(nmt * p.Nt + nc0), v);
+          }
+          if (co < p.K) {  // K is a multiple of 4 here, so the four channels exist together
+            // loads and conversions first, the (predicated) stores last: no branch sits between
+            // the eight independent chains, so their latencies overlap
+            uint4 u[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int row = srow + 4 * i;
+              u[i] = *reinterpret_cast<const uint4*>(stage + row * EPI_PITCH + ((scol ^ (row & 7)) << 4));
+            }
+            if (!p.out_i32) {
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                const int row = srow + 4 * i;
-                u[i] = *reinterpret_cast<const uint4*>(stage + row * EPI_PITCH + ((scol ^ (row & 7)) << 4));
+                u[i].x = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].x) : (float)(int)u[i].x, al.x));
+                u[i].y = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].y) : (float)(int)u[i].y, al.y));
+                u[i].z = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].z) : (float)(int)u[i].z, al.z));
+                u[i].w = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].w) : (float)(int)u[i].w, al.w));
               }
-              if (!p.out_i32) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                  u[i].x = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].x) : (float)(int)u[i].x, al.x));
-                  u[i].y = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].y) : (float)(int)u[i].y, al.y));
-                  u[i].z = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].z) : (float)(int)u[i].z, al.z));
-                  u[i].w = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].w) : (float)(int)u[i].w, al.w));
-                }
-              }
-              uint32_t* obase32 = reinterpret_cast<uint32_t*>(p.out) + co;  // int32 and fp32 outputs share the layout
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                if (ro[i] >= 0) *reinterpret_cast<uint4*>(obase32 + ro[i]) = u[i];
             }
-            __syncwarp();
+            uint32_t* obase32 = reinterpret_cast<uint32_t*>(p.out) + co;  // int32 and fp32 outputs share the layout
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              if (ro[i] >= 0) *reinterpret_cast<uint4*>(obase32 + ro[i]) = u[i];
           }
-        } else if ((p.Nt & 31) == 0) {
-          for (int c0 = 32 * half; c0 < p.Nt; c0 += 64)
-            epilogue_slice<F16, 32>(p, trow + (uint32_t)c0, c0, n0, valid, obase);
-        } else {
-          for (int c0 = 16 * half; c0 < p.Nt; c0 += 32)
-            epilogue_slice<F16, 16>(p, trow + (uint32_t)c0, c0, n0, valid, obase);
+          __syncwarp();
+        }
+      } else {
+#pragma unroll 1
+        for (int mt = 0; mt < MT; ++mt) {
+          bool valid;
+          size_t obase;
+          row_info(mt, &valid, &obase);
+          const uint32_t trow = d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt);
+          if ((p.Nt & 31) == 0) {
+            for (int c0 = 32 * half; c0 < p.Nt; c0 += 64)
+              epilogue_slice<F16, 32>(p, trow + (uint32_t)c0, c0, n0, valid, obase);
+          } else {
+            for (int c0 = 16 * half; c0 < p.Nt; c0 += 32)
+              epilogue_slice<F16, 16>(p, trow + (uint32_t)c0, c0, n0, valid, obase);
+          }
         }
       }
       // this warp has read its part of the accumulator buffer: hand it back to the MMA issuer
@@ -922,16 +978,31 @@ cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l
   p.out = l.out;
   p.out_i32 = l.out_i32;
   p.status = status_dev;
-  if (f16) tc_expand_act_kernel<true><<<pl.xgrid, 256, 0, l.stream>>>(p);
-  else tc_expand_act_kernel<false><<<pl.xgrid, 256, 0, l.stream>>>(p);
-  cudaError_t e = cudaGetLastError();
+  // Both kernels are launched as programmatic dependents of their predecessor in the stream:
+  // their set-up overlaps its tail, and each waits on the device for it before touching its data.
+  const bool pdl = env_int("SNN_TC_PDL", 1) != 0;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.stream = l.stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  cfg.gridDim = pl.xgrid;
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cudaError_t e = f16 ? cudaLaunchKernelEx(&cfg, tc_expand_act_kernel<true>, p)
+                      : cudaLaunchKernelEx(&cfg, tc_expand_act_kernel<false>, p);
   if (e != cudaSuccess) return e;
   *launched += 1;
+  cfg.gridDim = pl.grid;
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = pl.smem;
 #define SNN_TC_LAUNCH(F, M, KP)                                                                    \
   do {                                                                                             \
     static unsigned long long done = 0;                                                            \
     e = allow_max_smem(tc_conv_kernel<F, M, KP>, &done);                                           \
-    if (e == cudaSuccess) tc_conv_kernel<F, M, KP><<<pl.grid, TC_THREADS, pl.smem, l.stream>>>(p); \
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tc_conv_kernel<F, M, KP>, p);               \
   } while (0)
 #define SNN_TC_LAUNCH_K(F, M)                 \
   do {                                        \
