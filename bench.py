@@ -183,10 +183,10 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     import paper_2110_09195_b200 as snn
+    from paper_2110_09195_b200 import replicas
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    info = replicas.rank_info()
+    rank, world, local_rank = info.rank, info.world, info.local_rank
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local_rank)
@@ -315,11 +315,8 @@ def run_ours(args):
     h2d = sum(a.numel() * a.element_size() for a in host_acts)
     d2h = sum(o.numel() * o.element_size() for o in host_outs)
 
-    # max over ranks (device-timed)
-    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(t[0]), float(t[1])
+    # max over ranks of the device-timed totals; every rank ran a batch of its own (weak scaling)
+    total_ms, e2e_ms = replicas.max_over_ranks([total_ms, e2e_ms], world, dev)
     ms_per_step = total_ms / args.steps
     value = nb * world / (ms_per_step * 1e-3)
     e2e_value = nb * world / (e2e_ms * 1e-3)

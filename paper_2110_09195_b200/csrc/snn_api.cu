@@ -275,7 +275,6 @@ snn_status_t snn_conv_destroy(snn_conv_t* h) {
   cudaFree(h->L.match9);
   cudaFree(h->L.w8);
   cudaFree(h->L.w16);
-  cudaFree(h->L.tc_scratch);
   cudaFree(h->stage_in);
   cudaFree(h->stage_out);
   if (h->tc_status_host) cudaFreeHost(h->tc_status_host);

@@ -6,33 +6,28 @@
 //   M = 128 consecutive positions of a padded, flattened copy of the input,
 //   N = a tile of output channels, K = (tap, input channel).
 //
-// Two kernels per forward call.
+// One persistent, warp-specialised kernel per forward call.
 //
-// 1. tc_expand_act_kernel writes the activations once, as tensor-core operands,
-//    into a scratch buffer the layer handle owns, already cut into the units the
-//    GEMM stages:  xa[position group][channel block][plane][16-byte channel
-//    chunk][row][16 B]  (bits -> +1/-1 bytes, or fp16 copied), over a padded,
-//    flattened position space that keeps one zero column per row and one zero
-//    row per image (shared by neighbours), so that zero padding is a literal
-//    zero operand (a zero contributes 0, as the definition requires).  Rows a
-//    group shares with its neighbour (the halo of the taps) are written twice.
-//    Stride 2 splits the padded input into its four row/column parity planes.
-//
-// 2. tc_conv_kernel is a persistent, warp-specialised GEMM.  A unit of xa is the
-//    shared-memory image of one (tile, channel block) of the A operand in the
-//    K-major, no-swizzle layout (rows 16 bytes apart), so it arrives with one
-//    bulk copy, and the A operand of tap (ky, kx) is that block read from a
-//    start address shifted by ky*pitch + kx rows: the nine taps reuse one
-//    staged unit, there is no im2col copy.  The K loop runs channel block by
-//    channel block (then taps, then chunks), so the MMAs of a tile start when
-//    its first block has landed.
-//      warp 0      one thread streams A units and weight stages (cp.async.bulk
-//                  onto mbarriers; rings of NA units and NS stages)
-//      warp 1      one thread issues tcgen05.mma into one of two TMEM
-//                  accumulator buffers and commits barriers
-//      warps 2-9   epilogue: TMEM -> registers -> per-warp shared-memory
-//                  transposition -> alpha scale -> 128-byte row stores, for
-//                  tile i while the MMAs of tile i+1 run
+// The A operand lives in shared memory as units  [plane][16-byte channel
+// chunk][row][16 B]  (one unit = one tile of positions x one channel block), the
+// K-major, no-swizzle layout whose rows are 16 bytes apart.  The flattened
+// position space keeps one zero column per row and one zero row per image
+// (shared by neighbours), so zero padding is a literal zero operand (a zero
+// contributes 0, as the definition requires) and the A operand of tap (ky, kx)
+// is the same unit read from a start address shifted by ky*pitch + kx rows:
+// the nine taps reuse one staged unit, there is no im2col copy.  Stride 2
+// splits the padded input into its four row/column parity planes.  The K loop
+// runs channel block by channel block (then taps, then chunks), so the MMAs of
+// a tile start when its first block is staged.
+//      warp 0        one thread streams weight stages (cp.async.bulk onto
+//                    mbarriers, a ring of NS stages; resident when they fit)
+//      warp 1        one thread issues tcgen05.mma into one of two TMEM
+//                    accumulator buffers and commits barriers
+//      warps 2-9     epilogue: TMEM -> registers -> per-warp shared-memory
+//                    transposition -> alpha scale -> 128-byte row stores, for
+//                    tile i while the MMAs of tile i+1 run
+//      warps 10-17   expanders: packed bits -> +1/-1 bytes (or fp16 copied)
+//                    straight into the A units of a ring of NA, ahead of the MMAs
 //    Measured on B200 and shaping this code: a thread alone on its warp retires
 //    about one instruction per 5-8 cycles (more when other warps compete) and
 //    an mbarrier wait costs ~200 cycles even when it is ready, so the issuing
@@ -51,8 +46,10 @@ namespace snn {
 
 namespace {
 
-constexpr int TC_THREADS = 320;               // warp 0 producer, warp 1 MMA issue, warps 2-9 epilogue
+constexpr int EXP_WARPS = 8, EXP_THREADS = 32 * EXP_WARPS;
+constexpr int TC_THREADS = 320 + EXP_THREADS;  // warp 0 producer, 1 MMA issue, 2-9 epilogue, 10-17 expanders
 constexpr int EPI_WARPS = 8;
+constexpr int EXP_ROWS = 3;                   // rows of a unit one expander thread loads together
 constexpr int NS_MAX = 8;                     // most weight stages in flight
 constexpr uint32_t WAIT_LIMIT = 1u << 20;     // try_wait attempts before a wait gives up
 constexpr int EPI_PITCH = 128;                // bytes per staged output row; 16-byte columns are XOR-swizzled by row
@@ -80,13 +77,13 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t q, const FastDiv& f) {
 }
 
 struct TcParams {
-  const void* act;        // uint32 [N][H][W][Cw] or half [N][H][W][C]      (expansion kernel)
-  uint8_t* xa;            // expanded activations [group][block][plane][chunk][Rr][16 B]  (scratch)
+  const void* act;        // uint32 [N][H][W][Cw] or half [N][H][W][C]
   const uint8_t* wt;      // tiled weights: [layout tile][block][tap][chunk][NtL][16 B]
   const float* alpha;
   void* out;
   int* status;            // mapped host word, set on a timed-out wait
   int out_i32;
+  int act_vec;            // the activation rows may be read with 8/16-byte loads
   int N, H, W, C, K, Cw, stride, pad, Ho, Wo;
   int Kpad, n_chunks;     // padded channels out; 16-byte chunks along the padded channels in
   int NtL;                // channels per layout tile of the weight operand
@@ -109,7 +106,7 @@ struct TcParams {
   uint32_t tmem_cols;     // power of two >= n_acc*MT*Nt
   uint32_t a_unit_bytes;  // bytes of one staged activation unit
   uint32_t stage_bytes;   // bytes of one weight stage
-  uint32_t off_b, off_epi, off_tail;  // shared-memory offsets
+  uint32_t off_b, off_epi, off_pix, off_tail;  // shared-memory offsets
 };
 
 // ---------------------------------------------------------------- PTX helpers
@@ -159,6 +156,7 @@ __device__ __forceinline__ void raise_status(int* status, int code) {
   *reinterpret_cast<volatile int*>(status) = code;
   __threadfence_system();
 }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -301,59 +299,6 @@ __device__ __forceinline__ void epilogue_slice(const TcParams& p, uint32_t taddr
 
 }  // namespace
 
-// ------------------------------------------------------------------ expansion
-// One thread per (position group, row, plane, group of four 32-channel words).
-// Reads are contiguous per thread, writes are 16 bytes per thread with
-// consecutive threads on consecutive rows (coalesced).  Every row of every unit
-// is written, padding and tail included, so the scratch never needs clearing.
-template <bool F16>
-__global__ void __launch_bounds__(256) tc_expand_act_kernel(const TcParams p) {
-  grid_dep_launch();  // the GEMM may set itself up (barriers, TMEM, weight prefetch) meanwhile
-  grid_dep_wait();    // the activations, and the scratch a previous GEMM may still read, are ready
-  const uint32_t row_id = blockIdx.x * 256u + threadIdx.x;  // (group, row)
-  if (row_id >= (uint32_t)p.n_mgroups * (uint32_t)p.Rr) return;
-  const uint32_t mg = row_id / (uint32_t)p.Rr;
-  const int r = (int)(row_id - mg * (uint32_t)p.Rr);
-  const int pl = blockIdx.y, pa = pl >> 1, pb = pl & 1;
-  const uint32_t q = mg * (uint32_t)(128 * p.MT) + (uint32_t)r;
-  const int pix = position_to_pixel(p, q, pa, pb);
-  // chunk c of block cb lands at ((((mg*n_cb + cb)*n_planes + pl)*cb_chunks + c)*Rr + r)
-  uint4* base = reinterpret_cast<uint4*>(p.xa);
-  const int steps = p.n_chunks / 2;               // two chunks (32 int8 / 16 fp16 channels) per step
-  for (int st = blockIdx.z * 4; st < steps && st < blockIdx.z * 4 + 4; ++st) {
-    uint4 v[2];
-    if (F16) {
-      const __half* src = (const __half*)p.act + (size_t)(pix < 0 ? 0 : pix) * p.C;
-      const bool vec = pix >= 0 && ((p.C & 7) == 0);
-#pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        v[k] = make_uint4(0, 0, 0, 0);
-        const int ch = (st * 2 + k) * 8;
-        if (vec && ch + 8 <= p.C) {
-          v[k] = __ldg(reinterpret_cast<const uint4*>(src + ch));
-        } else if (pix >= 0) {
-          uint32_t w[4] = {0, 0, 0, 0};
-#pragma unroll
-          for (int e = 0; e < 8; ++e)
-            if (ch + e < p.C) w[e >> 1] |= (uint32_t)__half_as_ushort(src[ch + e]) << (16 * (e & 1));
-          v[k] = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-      }
-    } else {
-      // one 32-channel word -> two chunks of 16 int8 channels
-      uint32_t bits = 0;
-      if (pix >= 0 && st < p.Cw) bits = __ldg((const uint32_t*)p.act + (size_t)pix * p.Cw + st);
-      expand_word(bits, p.C - st * 32, pix >= 0 && st < p.Cw, v[0], v[1]);
-    }
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const int chunk = st * 2 + k;
-      const int cb = chunk / p.cb_chunks, c = chunk - cb * p.cb_chunks;
-      base[((((size_t)mg * p.n_cb + cb) * p.n_planes + pl) * p.cb_chunks + c) * p.Rr + r] = v[k];
-    }
-  }
-}
-
 // ------------------------------------------------------------------ GEMM
 // KPT = MMAs per sub-tile and tap when known at compile time (2 or 4), 0 = read from the parameters
 template <bool F16, int MT, int KPT>
@@ -363,6 +308,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
   uint8_t* a_smem = smem;
   uint8_t* b_smem = smem + p.off_b;
   uint8_t* epi_smem = smem + p.off_epi;
+  int* pix_tab = reinterpret_cast<int*>(smem + p.off_pix);  // [plane][row] input pixel of a staged row
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_tail);
   // barriers: b_full[8] b_empty[8] a_full[4] a_empty[4] acc_full[2] acc_empty[2]
   const uint32_t bar_bfull = smem_u32(bars), bar_bempty = smem_u32(bars + 8);
@@ -370,14 +316,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
   const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 28);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  uint32_t* tap_units = tmem_slot + 2;  // [9] A row offset of every tap inside a unit
+  uint32_t* tap_units = tmem_slot + 3;  // [9] A row offset of every tap inside a unit (tmem_slot[2] = expander flag)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int NS = p.NS, NA = p.NA;
 
   if (tid < 28) {
     uint32_t count = 1;
-    if (tid >= 26) count = EPI_WARPS;  // acc_empty: one arrival per epilogue warp
+    if (tid >= 26) count = EPI_WARPS;                // acc_empty: one arrival per epilogue warp
+    if (tid >= 16 && tid < 20) count = EXP_THREADS;  // a_full: every expander thread arrives
     mbar_init(smem_u32(bars + tid), count);
   }
   if (tid == 32) *abort_flag = 0;
@@ -411,11 +358,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
   if (warp == 0) {
     // ------------------------------------------------ producer (one lane)
     if (lane == 0) {
-      int a_slot = 0, b_slot = 0, a_issued = 0, b_issued = 0;
-      uint32_t a_phase = 1, b_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
+      int b_slot = 0, b_issued = 0;
+      uint32_t b_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
       bool ok = true;
-      bool first_tile = true;
-      const uint32_t unit_bytes = (uint32_t)(p.n_planes * p.cb_chunks * p.Rr) * 16;  // exact bytes of a unit
       // Weight stages are issued in the order the MMAs consume them; `w_next` counts the stages
       // already requested, so that the first ones can be requested before the expanded
       // activations exist (the weights are constants of the layer).
@@ -448,46 +393,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
         }
         return true;
       };
-      // before the activations are there: as many weight stages of the first tile as the ring holds
-      if ((int)blockIdx.x < p.total_tiles) {
-        const long long first = stages_per_tile < NS ? stages_per_tile : NS;
-        issue_weights(blockIdx.x, first);
-      }
-      grid_dep_wait();  // the expansion kernel's writes to xa are complete and visible
       long long tiles_seen = 0;
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x, ++tiles_seen) {
-        const int mg = tile / p.n_ntiles;
-        for (int cb = 0; cb < p.n_cb && ok; ++cb) {
-          // ---- activation unit (tile, channel block): one contiguous run of xa
-          if (*abort_flag) { ok = false; break; }
-          if (a_issued >= NA && !mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 32)) {
-            *abort_flag = 1;
-            raise_status(p.status, 1);
-            ok = false;
-            break;
-          }
-          mbar_expect_tx(bar_afull + 8 * a_slot, unit_bytes);
-          bulk_g2s(smem_u32(a_smem) + (uint32_t)a_slot * p.a_unit_bytes,
-                   p.xa + ((size_t)mg * p.n_cb + cb) * unit_bytes, unit_bytes, bar_afull + 8 * a_slot);
-          ++a_issued;
-          if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
-          // ---- weight stages of this channel block (kept from the first tile on when resident)
-          if (p.b_resident && !first_tile) continue;
-          if (!issue_weights(tile, tiles_seen * stages_per_tile + (long long)(cb + 1) * stages_per_cb)) {
-            *abort_flag = 1;
-            raise_status(p.status, 2);
-            ok = false;
-            break;
-          }
+        if (p.b_resident && tiles_seen > 0) break;  // kept from the first tile on
+        if (*abort_flag) break;
+        if (!issue_weights(tile, (tiles_seen + 1) * stages_per_tile)) {
+          *abort_flag = 1;
+          raise_status(p.status, 2);
+          ok = false;
         }
-        first_tile = false;
       }
       // never leave with copies in flight: wait (bounded) for the last load of every slot
-      for (int s = 0; s < NA; ++s) {
-        int last = -1;
-        for (int i = s; i < a_issued; i += NA) last = i;
-        if (last >= 0) mbar_wait_backoff(bar_afull + 8 * s, (last / NA) & 1, 64);
-      }
       for (int s = 0; s < NS; ++s) {
         int last = -1;
         for (int i = s; i < b_issued; i += NS) last = i;
@@ -563,7 +479,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       }
     }
     __syncwarp();
-  } else {
+  } else if (warp < 2 + EPI_WARPS) {
     // ------------------------------------------------ epilogue warps
     grid_dep_wait();  // an earlier kernel in the stream may still read the output buffer
     // Warp w reads TMEM lanes 32*(w%4).. (rows of the tile); the two warps of a lane quarter
@@ -609,17 +525,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
         const int per_mt = (p.Nt - 32 * half + 63) / 64;
         const int total = MT * per_mt;
         uint32_t v[32];
-        long long ro[8];
+        int ro[8];
         if (total > 0) tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(32 * half), v);
 #pragma unroll 1
         for (int sl = 0; sl < total; ++sl) {
           const int mt = sl / per_mt, c0 = 32 * half + 64 * (sl - mt * per_mt);
           if (sl - mt * per_mt == 0) {
-            // element offsets of the eight rows this lane stores (row = srow + 4*i), -1 when not an output
+            // output pixels of the eight rows this lane stores (row = srow + 4*i), -1 when not an output
             bool valid;
             size_t obase;
             row_info(mt, &valid, &obase);
-            const long long mine = valid ? (long long)obase : -1;
+            const int mine = valid ? (int)(obase / (size_t)p.K) : -1;  // output pixel (fits: pixels are 32-bit here)
 #pragma unroll
             for (int i = 0; i < 8; ++i) ro[i] = __shfl_sync(0xffffffffu, mine, srow + 4 * i);
           }
@@ -657,7 +573,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
             uint32_t* obase32 = reinterpret_cast<uint32_t*>(p.out) + co;  // int32 and fp32 outputs share the layout
 #pragma unroll
             for (int i = 0; i < 8; ++i)
-              if (ro[i] >= 0) *reinterpret_cast<uint4*>(obase32 + ro[i]) = u[i];
+              if (ro[i] >= 0) *reinterpret_cast<uint4*>(obase32 + (size_t)ro[i] * (size_t)p.K) = u[i];
           }
           __syncwarp();
         }
@@ -682,6 +598,132 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_accempty + 8 * acc_slot);
       if (++acc_slot == p.n_acc) { acc_slot = 0; acc_phase ^= 1u; }
+    }
+  }
+  else {
+    // ------------------------------------------------ expanders (warps 10-17)
+    // Fill activation unit (tile, channel block) of the ring: for every plane, row and 32-channel
+    // word, bits -> two 16-byte chunks of +1/-1 bytes (fp16: copy two 8-channel chunks).  A thread
+    // takes EXP_ROWS rows at a time and issues their loads together.
+    grid_dep_wait();  // the activations may come from the previous kernel in the stream
+    const int et = tid - (2 + EPI_WARPS) * 32;
+    int a_slot = 0, a_done = 0;
+    uint32_t a_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
+    volatile int* exp_flag = abort_flag + 1;
+    const int nstep = p.cb_chunks / 2;  // pairs of chunks per unit
+    for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+      const int mg = tile / p.n_ntiles;
+      const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
+      bool stop = false;
+      // input pixel of every staged row, once per tile: -1 where the row is padding.  A thread
+      // reads back only the entries it wrote, so no barrier is needed.
+      for (int pl = 0; pl < p.n_planes; ++pl)
+        for (int r = et; r < p.Rr; r += EXP_THREADS)
+          pix_tab[pl * p.Rr + r] = position_to_pixel(p, Q0 + (uint32_t)r, pl >> 1, pl & 1);
+      for (int cb = 0; cb < p.n_cb; ++cb) {
+        if (a_done >= NA) {
+          // one elected thread polls; the rest wait on a hardware barrier instead of spinning
+          if (et == 0) *exp_flag = (!*abort_flag && mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 64)) ? 1 : 0;
+          asm volatile("bar.sync 3, %0;" ::"n"(EXP_THREADS) : "memory");
+          const int okf = *exp_flag;
+          asm volatile("bar.sync 3, %0;" ::"n"(EXP_THREADS) : "memory");
+          if (!okf) {
+            if (et == 0 && !*abort_flag) {
+              *abort_flag = 1;
+              raise_status(p.status, 1);
+            }
+            stop = true;
+            break;
+          }
+        }
+        uint8_t* unit = a_smem + (size_t)a_slot * p.a_unit_bytes;
+        for (int pl = 0; pl < p.n_planes; ++pl) {
+          uint8_t* plane = unit + (size_t)pl * p.cb_chunks * p.Rr * 16;
+          for (int rb = 0; rb < p.Rr; rb += EXP_ROWS * EXP_THREADS) {
+            int pix[EXP_ROWS];  // input pixel of each of this thread's rows; -1 padding, -2 past the unit
+#pragma unroll
+            for (int j = 0; j < EXP_ROWS; ++j) {
+              const int r = rb + et + j * EXP_THREADS;
+              pix[j] = r < p.Rr ? pix_tab[pl * p.Rr + r] : -2;
+            }
+            if (F16) {
+              for (int c0 = 0; c0 < p.cb_chunks; c0 += 2) {
+                uint4 v[EXP_ROWS][2];
+#pragma unroll
+                for (int j = 0; j < EXP_ROWS; ++j) {
+#pragma unroll
+                  for (int k = 0; k < 2; ++k) {
+                    v[j][k] = make_uint4(0, 0, 0, 0);
+                    const int ch = (cb * p.cb_chunks + c0 + k) * 8;  // first channel of the chunk
+                    if (pix[j] >= 0 && ch < p.C) {
+                      const __half* src = (const __half*)p.act + (size_t)pix[j] * p.C + ch;
+                      if (p.act_vec) {
+                        v[j][k] = __ldg(reinterpret_cast<const uint4*>(src));
+                      } else {
+                        uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                          if (ch + e < p.C) w[e >> 1] |= (uint32_t)__half_as_ushort(src[e]) << (16 * (e & 1));
+                        v[j][k] = make_uint4(w[0], w[1], w[2], w[3]);
+                      }
+                    }
+                  }
+                }
+#pragma unroll
+                for (int j = 0; j < EXP_ROWS; ++j) {
+                  const int r = rb + et + j * EXP_THREADS;
+                  if (pix[j] != -2) {
+                    *reinterpret_cast<uint4*>(plane + ((size_t)c0 * p.Rr + r) * 16) = v[j][0];
+                    *reinterpret_cast<uint4*>(plane + ((size_t)(c0 + 1) * p.Rr + r) * 16) = v[j][1];
+                  }
+                }
+              }
+            } else {
+              // up to four 32-channel words per row and block, as one vector load when aligned
+              const int w0 = cb * nstep;
+              uint32_t bits[EXP_ROWS][4];
+#pragma unroll
+              for (int j = 0; j < EXP_ROWS; ++j) {
+                bits[j][0] = bits[j][1] = bits[j][2] = bits[j][3] = 0;
+                if (pix[j] >= 0 && w0 < p.Cw) {
+                  const uint32_t* src = (const uint32_t*)p.act + (size_t)pix[j] * p.Cw + w0;
+                  if (p.act_vec && nstep == 4) {
+                    const uint4 t = __ldg(reinterpret_cast<const uint4*>(src));
+                    bits[j][0] = t.x; bits[j][1] = t.y; bits[j][2] = t.z; bits[j][3] = t.w;
+                  } else if (p.act_vec && nstep == 2) {
+                    const uint2 t = __ldg(reinterpret_cast<const uint2*>(src));
+                    bits[j][0] = t.x; bits[j][1] = t.y;
+                  } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                      if (k < nstep && w0 + k < p.Cw) bits[j][k] = __ldg(src + k);
+                  }
+                }
+              }
+#pragma unroll
+              for (int j = 0; j < EXP_ROWS; ++j) {
+                const int r = rb + et + j * EXP_THREADS;
+                if (pix[j] != -2) {
+#pragma unroll
+                  for (int k = 0; k < 4; ++k) {
+                    if (k < nstep) {
+                      uint4 lo, hi;
+                      expand_word(bits[j][k], p.C - (w0 + k) * 32, pix[j] >= 0 && w0 + k < p.Cw, lo, hi);
+                      *reinterpret_cast<uint4*>(plane + ((size_t)(2 * k) * p.Rr + r) * 16) = lo;
+                      *reinterpret_cast<uint4*>(plane + ((size_t)(2 * k + 1) * p.Rr + r) * 16) = hi;
+                    }
+                  }
+                }
+              }
+            }
+          }
+        }
+        fence_proxy_async();  // generic-proxy writes -> visible to the tensor core's reads
+        mbar_arrive(bar_afull + 8 * a_slot);
+        ++a_done;
+        if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
+      }
+      if (stop) break;
     }
   }
 
@@ -781,8 +823,7 @@ cudaError_t tc_expand_weights(const LayerDev& L, const Geom& g, int act_type, cu
 struct TcPlan {
   TcParams p;
   size_t smem;
-  size_t xa_bytes;
-  dim3 grid, xgrid;
+  dim3 grid;
   bool ok;
   double score;
 };
@@ -859,7 +900,8 @@ static TcPlan plan_for(const Geom& g, int act_type, int MT, int stage_kb) {
   p.a_unit_bytes = (uint32_t)((unit_exact + 127) & ~(size_t)127);
   const size_t kstep_bytes = (size_t)2 * Nt * 16;        // weights of one MMA
   const size_t tap_bytes = (size_t)p.kpt * kstep_bytes;  // weights of one tap of one channel block
-  const size_t fixed = (size_t)EPI_BYTES + kSmemTail;
+  const size_t pix_bytes = ((size_t)p.n_planes * p.Rr * 4 + 127) & ~(size_t)127;
+  const size_t fixed = (size_t)EPI_BYTES + pix_bytes + kSmemTail;
   const size_t stage_cap = (size_t)(stage_kb > 0 ? stage_kb : 48) * 1024;
   const long long units_per_cta = (long long)tiles_per_cta * p.n_cb;
   int na = units_per_cta >= 3 && p.n_cb >= 2 ? 3 : (units_per_cta >= 2 ? 2 : 1);
@@ -896,16 +938,14 @@ static TcPlan plan_for(const Geom& g, int act_type, int MT, int stage_kb) {
   p.NS = ns;
   p.off_b = (uint32_t)((size_t)na * p.a_unit_bytes);
   p.off_epi = p.off_b + (uint32_t)((size_t)ns * p.stage_bytes);
-  p.off_tail = p.off_epi + EPI_BYTES;
+  p.off_pix = p.off_epi + EPI_BYTES;
+  p.off_tail = p.off_pix + (uint32_t)pix_bytes;
   pl.smem = (size_t)p.off_tail + kSmemTail;
   if (pl.smem > (size_t)kMaxDynSmem) return pl;
   if (pl.smem >= (1u << 18)) return pl;               // shared-memory descriptor address range
   if ((uint32_t)p.Rr * 16 >= (1u << 18)) return pl;   // leading-offset field range
   if (p.stage_bytes >= (1u << 20) || unit_exact >= (1u << 20)) return pl;  // mbarrier transaction counts
-  pl.xa_bytes = (size_t)mgroups * p.n_cb * unit_exact;
   pl.grid = dim3((unsigned)grid);
-  const long long xrows = mgroups * p.Rr;
-  pl.xgrid = dim3((unsigned)((xrows + 255) / 256), (unsigned)p.n_planes, (unsigned)((p.n_chunks / 2 + 3) / 4));
   // heuristic score: balance of the persistent CTAs x useful share of the staged rows
   const long long rounds = tiles_per_cta;
   double eff = (double)p.total_tiles / (double)(rounds * grid) * (double)grid / (double)sms;
@@ -961,25 +1001,23 @@ cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l
   if (!pl.ok) return cudaErrorInvalidConfiguration;
   const bool f16 = act_type == SNN_ACT_F16;
   TcParams& p = pl.p;
-  // scratch for the expanded activations: grows on demand, so that a shape's first call may
-  // allocate (not inside a stream capture) and later calls never do
-  if (pl.xa_bytes > L.tc_scratch_bytes) {
-    if (L.tc_scratch) cudaFree(L.tc_scratch);
-    L.tc_scratch = nullptr;
-    L.tc_scratch_bytes = 0;
-    cudaError_t ea = cudaMalloc(&L.tc_scratch, pl.xa_bytes);
-    if (ea != cudaSuccess) return ea;
-    L.tc_scratch_bytes = pl.xa_bytes;
-  }
   p.act = l.act;
-  p.xa = (uint8_t*)L.tc_scratch;
+  {
+    // vector loads of a row's words need the base pointer and the row pitch aligned to the load
+    const uintptr_t addr = (uintptr_t)l.act;
+    if (f16) p.act_vec = (addr & 15) == 0 && (g.C & 7) == 0;
+    else if (p.cb_chunks == 8) p.act_vec = (addr & 15) == 0 && (g.Cw & 3) == 0;
+    else if (p.cb_chunks == 4) p.act_vec = (addr & 7) == 0 && (g.Cw & 1) == 0;
+    else p.act_vec = 0;
+  }
   p.wt = f16 ? (const uint8_t*)L.w16 : (const uint8_t*)L.w8;
   p.alpha = L.alpha;
   p.out = l.out;
   p.out_i32 = l.out_i32;
   p.status = status_dev;
-  // Both kernels are launched as programmatic dependents of their predecessor in the stream:
-  // their set-up overlaps its tail, and each waits on the device for it before touching its data.
+  // The kernel is launched as a programmatic dependent of its predecessor in the stream: its
+  // set-up and first weight loads overlap that kernel's tail, and it waits on the device for it
+  // before it reads the activations or writes the output.
   const bool pdl = env_int("SNN_TC_PDL", 1) != 0;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -988,13 +1026,7 @@ cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l
   cfg.stream = l.stream;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
-  cfg.gridDim = pl.xgrid;
-  cfg.blockDim = dim3(256);
-  cfg.dynamicSmemBytes = 0;
-  cudaError_t e = f16 ? cudaLaunchKernelEx(&cfg, tc_expand_act_kernel<true>, p)
-                      : cudaLaunchKernelEx(&cfg, tc_expand_act_kernel<false>, p);
-  if (e != cudaSuccess) return e;
-  *launched += 1;
+  cudaError_t e = cudaSuccess;
   cfg.gridDim = pl.grid;
   cfg.blockDim = dim3(TC_THREADS);
   cfg.dynamicSmemBytes = pl.smem;
