@@ -239,6 +239,7 @@ snn_status_t snn_conv_create(const snn_conv_desc_t* d, snn_conv_t** out) {
   if (tcw) {
     if (h->act_type == SNN_ACT_BIN) alloc((void**)&h->L.w8, tcw);
     else alloc((void**)&h->L.w16, tcw);
+    alloc(&h->L.wcm, cm_weight_bytes(g, h->act_type));
   }
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->host_stream, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&h->tc_status_host, sizeof(int), cudaHostAllocMapped);
@@ -251,6 +252,7 @@ snn_status_t snn_conv_create(const snn_conv_desc_t* d, snn_conv_t** out) {
   int launched = 0;
   if (e == cudaSuccess) e = decode_layer(h->L, d_stream, g, h->act_type, s, &launched);
   if (e == cudaSuccess && tcw) e = tc_expand_weights(h->L, g, h->act_type, s, &launched);
+  if (e == cudaSuccess && tcw) e = cm_expand_weights(h->L, g, h->act_type, s, &launched);
   g_launches += launched;
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (d_stream) cudaFree(d_stream);
@@ -275,6 +277,7 @@ snn_status_t snn_conv_destroy(snn_conv_t* h) {
   cudaFree(h->L.match9);
   cudaFree(h->L.w8);
   cudaFree(h->L.w16);
+  cudaFree(h->L.wcm);
   cudaFree(h->stage_in);
   cudaFree(h->stage_out);
   if (h->tc_status_host) cudaFreeHost(h->tc_status_host);

@@ -28,8 +28,7 @@ struct LayerDev {
   uint8_t* match9 = nullptr;     // [T/16 or 1][512][16] matching-tap counts per (window, codebook kernel)
   int8_t* w8 = nullptr;          // tensor-core operand: +/-1 int8 weights, tiled (snn_tc.cu)
   uint16_t* w16 = nullptr;       // tensor-core operand: +/-1 fp16 weights, tiled (fp16 activations)
-
-
+  void* wcm = nullptr;           // channel-major tensor-core operand, [channel tile][K step][128][32 B] (snn_tcm.cu)
   int Kpad = 0;                  // K rounded up for the tensor-core tiling
   int Cpad = 0;                  // C rounded up for the tensor-core tiling
 };
@@ -61,6 +60,16 @@ cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l
                        int variant);
 size_t tc_weight_bytes(const Geom& g, int act_type, int* Kpad, int* Cpad);
 cudaError_t tc_expand_weights(const LayerDev& L, const Geom& g, int act_type, cudaStream_t s, int* launched);
+
+// Channel-major tensor-core kernel (weights in tensor memory); its variants are the positions
+// per tile.  tc_variant_count()/tc_variant_ok()/tc_forward() present them after the
+// position-major kernel's variants.
+int cm_variant_count();
+bool cm_variant_ok(const Geom& g, int act_type, int variant);
+cudaError_t cm_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched, int* status_dev,
+                       int variant);
+size_t cm_weight_bytes(const Geom& g, int act_type);
+cudaError_t cm_expand_weights(const LayerDev& L, const Geom& g, int act_type, cudaStream_t s, int* launched);
 
 cudaError_t microbench(int kind, double* rate);
 

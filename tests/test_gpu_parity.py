@@ -211,18 +211,56 @@ def test_tensor_core_path_runs_the_stack_shapes(snn):
 
 @pytest.mark.parametrize("c_in,c_out,h,w,stride", [(64, 64, 20, 20, 1), (256, 128, 9, 9, 1), (128, 256, 12, 12, 2)])
 def test_tensor_core_tile_variants(snn, oracle_mod, monkeypatch, c_in, c_out, h, w, stride):
-    """Every tile shape the tuner may pick (sub-tiles per CTA, weight-stage size, CTAs per SM)
-    gives the same sums."""
+    """Every tile shape of the position-major kernel the tuner may pick (sub-tiles per CTA,
+    weight-stage size) gives the same sums."""
     shape = wl.LayerShape(c_in, c_out, h, w, stride, 1)
     for mt in (1, 2, 4):
         for kb in (16, 32, 64):
-            for one in (0, 1):
-                monkeypatch.setenv("SNN_TC_MT", str(mt))
-                monkeypatch.setenv("SNN_TC_STAGE_KB", str(kb))
-                monkeypatch.setenv("SNN_TC_ONE_PER_SM", str(one))
-                p = wl.draw_layer_params(shape, 5, 77)
-                layer = snn.SnnConv(c_in, c_out, 5, p.codebook, p.idx_packed, p.alpha, stride, 1)
-                ok = layer.path_supported(snn.PATH_DECODED_TC, 3, h, w)
-                layer.destroy()
-                if ok:
-                    check_bin_layer(snn, oracle_mod, shape, 5, 3, 77, paths=[snn.PATH_DECODED_TC])
+            monkeypatch.setenv("SNN_TC_MT", str(mt))
+            monkeypatch.setenv("SNN_TC_STAGE_KB", str(kb))
+            p = wl.draw_layer_params(shape, 5, 77)
+            layer = snn.SnnConv(c_in, c_out, 5, p.codebook, p.idx_packed, p.alpha, stride, 1)
+            ok = layer.path_supported(snn.PATH_DECODED_TC, 3, h, w)
+            layer.destroy()
+            if ok:
+                check_bin_layer(snn, oracle_mod, shape, 5, 3, 77, paths=[snn.PATH_DECODED_TC])
+
+
+CM_SHAPES = [
+    (64, 64, 20, 20, 1, 3),      # resident weights, several tiles per CTA
+    (16, 16, 8, 8, 1, 2),        # one K step per tap, channels far below one tile
+    (256, 128, 9, 9, 1, 3),      # streamed weights, two channel blocks
+    (128, 256, 12, 12, 2, 3),    # stride 2 (four parity planes), two channel tiles
+    (200, 130, 7, 5, 1, 2),      # ragged channels in and out
+    (1056, 48, 9, 8, 2, 1),      # padded channel blocks
+    (512, 512, 7, 7, 1, 4),      # deep layer: 144 K steps, four channel tiles
+]
+
+
+@pytest.mark.parametrize("c_in,c_out,h,w,stride,n", CM_SHAPES)
+def test_channel_major_variants(snn, oracle_mod, monkeypatch, c_in, c_out, h, w, stride, n):
+    """The channel-major tensor-core kernel (weights in tensor memory) at every tile width."""
+    shape = wl.LayerShape(c_in, c_out, h, w, stride, 1)
+    ran = 0
+    for variant in range(16, 22):
+        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
+        check_bin_layer(snn, oracle_mod, shape, 5, n, 91, paths=[snn.PATH_DECODED_TC])
+        ran += 1
+    assert ran == 6
+
+
+def test_channel_major_many_tiles(snn, oracle_mod, monkeypatch):
+    """More tiles than CTAs: both accumulator buffers, ring wrap-around, streamed weights over
+    several tiles of one CTA."""
+    for variant, shape, n in [(16, wl.LayerShape(128, 128, 28, 28, 1, 1), 40), (20, wl.LayerShape(64, 64, 56, 56, 1, 1), 8),
+                              (17, wl.LayerShape(256, 256, 14, 14, 1, 1), 48)]:
+        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
+        check_bin_layer(snn, oracle_mod, shape, 5, n, 93, paths=[snn.PATH_DECODED_TC])
+
+
+def test_channel_major_fp16(snn, oracle_mod, monkeypatch):
+    for variant in (16, 17, 18):
+        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
+        for shape, n in [(wl.LayerShape(64, 64, 14, 14, 1, 1), 3), (wl.LayerShape(136, 72, 9, 7, 2, 1), 2)]:
+            ran = check_f16_layer(snn, oracle_mod, shape, 5, n, 95)
+            assert snn.PATH_DECODED_TC in ran
