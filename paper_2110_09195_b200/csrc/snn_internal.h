@@ -28,7 +28,7 @@ struct LayerDev {
   uint8_t* match9 = nullptr;     // [T/16 or 1][512][16] matching-tap counts per (window, codebook kernel)
   int8_t* w8 = nullptr;          // tensor-core operand: +/-1 int8 weights, tiled (snn_tc.cu)
   uint16_t* w16 = nullptr;       // tensor-core operand: +/-1 fp16 weights, tiled (fp16 activations)
-  void* wcm = nullptr;           // channel-major tensor-core operand, [channel tile][K step][128][32 B] (snn_tcm.cu)
+  void* wcm = nullptr;           // channel-major tensor-core operand, [channel tile][K step][half][128][16 B] (snn_tcm.cu)
   int Kpad = 0;                  // K rounded up for the tensor-core tiling
   int Cpad = 0;                  // C rounded up for the tensor-core tiling
 };

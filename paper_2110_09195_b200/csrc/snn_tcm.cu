@@ -15,17 +15,18 @@
 // only shared-memory operand is the activation tile (32*Np bytes per MMA), and tap
 // (ky, kx) is again the same staged unit read from a start address shifted by
 // ky*pitch + kx rows.  The accumulator holds channels in TMEM lanes and positions in
-// columns, so an epilogue thread owns one channel: its alpha is one register, and a
-// warp's store of one position is 32 consecutive channels = one 128-byte line of the
-// [N][Ho][Wo][K] output, with no transposition through shared memory.
+// columns, so a draining thread owns one channel; 16-position chunks are transposed
+// through a small shared-memory tile so that a store instruction writes four full
+// 128-byte lines of the [N][Ho][Wo][K] output.
 //
 //      warp 0        allocates tensor memory
 //      warp 1        one thread issues tcgen05.mma (A from TMEM, B from shared memory)
-//      warps 2-9     epilogue: TMEM -> registers -> alpha -> 128-byte line stores
+//      warps 2-9     drain the accumulators: TMEM -> registers -> transposition tile ->
+//                    alpha -> line stores, for tile i while the MMAs of tile i+1 run
 //      warps 10-17   expanders: packed bits -> +1/-1 bytes into the activation ring
-//      warps 18-25   weight loaders, two per TMEM lane quarter, alternating stages of
-//                    four K steps: 32 B per thread and K step from global memory,
-//                    one tcgen05.st per stage into a ring of TMEM columns
+//      warps 18-25   weight loaders, two per TMEM lane quarter, each filling half of a
+//                    stage of eight K steps: 32 B per thread and K step from global
+//                    memory, one tcgen05.st per half stage into a ring of TMEM columns
 // When all K steps of a channel tile fit the ring they are loaded once and kept.
 // Every wait is bounded; one that runs out raises a status word the host reads, and
 // the CTA still frees its tensor memory and returns.
@@ -40,14 +41,15 @@ constexpr int CM_EXP_THREADS = 32 * CM_EXP_WARPS;
 constexpr int CM_FIRST_EXP = 2 + CM_EPI_WARPS, CM_FIRST_LOAD = CM_FIRST_EXP + CM_EXP_WARPS;
 constexpr int CM_THREADS = 32 * (CM_FIRST_LOAD + CM_LOAD_WARPS);
 constexpr int CM_EXP_ROWS = 3;        // rows of a unit one expander thread loads together
-constexpr int CM_WST = 4;             // K steps per weight stage (8 TMEM columns each)
-constexpr int CM_RING_MAX = 12;       // most weight stages in the ring
+constexpr int CM_WST = 8;             // K steps per weight stage (8 TMEM columns each); a loader warp fills half a stage
+constexpr int CM_RING_MAX = 8;        // most weight stages in the ring
+constexpr int CM_EPI_STAGE = 2048;    // bytes of an epilogue warp's transposition tile: 16 positions x 32 channels
 constexpr int CM_NA_MAX = 8;          // most activation units in flight
 constexpr size_t kCmTail = 512;
 
 struct CmParams {
   const void* act;        // uint32 [N][H][W][Cw] or half [N][H][W][C]
-  const uint8_t* wa;      // [channel tile][K step][128 channels][32 B]
+  const uint8_t* wa;      // [channel tile][K step][16-byte half][128 channels][16 B]
   const float* alpha;
   void* out;
   int* status;
@@ -60,13 +62,14 @@ struct CmParams {
   int n_mgroups, n_cotiles, total_tiles;
   int cb_chunks, n_cb, kpt;
   int KS;                 // K steps per tile = 9 * n_cb * kpt, ordered (block, tap, step)
-  int n_wstages;          // weight stages per tile = ceil(KS / 4)
+  int spc;                // weight stages per channel block = ceil(9 * kpt / 4); the last may be short
+  int n_wstages;          // weight stages per tile = n_cb * spc
   int NW;                 // stages in the TMEM ring
   int w_resident;         // all stages of the CTA's channel tile stay in the ring
   int NA, n_acc;
   long long Qtot;
   uint32_t ring_col0;     // first TMEM column of the weight ring
-  uint32_t a_unit_bytes, off_pix, off_tail;
+  uint32_t a_unit_bytes, off_pix, off_epi, off_tail;
 };
 
 __device__ __forceinline__ int cm_input_pixel(const CmParams& p, uint32_t q, int pa, int pb) {
@@ -126,19 +129,21 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 
 }  // namespace
 
-template <bool F16>
+// KPT = MMAs per tap and channel block (cb_chunks / 2), a compile-time constant so that the
+// issuing thread runs straight-line code.
+template <bool F16, int KPT>
 __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t* a_smem = smem;                                      // [NA activation units]
   int* pix_tab = reinterpret_cast<int*>(smem + p.off_pix);    // [plane][row] input pixel of a staged row
+  uint8_t* epi_smem = smem + p.off_epi;                       // [epilogue warp][16 positions][32 channels]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_tail);
-  // barriers: w_full[12] w_empty[12] a_full[8] a_empty[8] acc_full[2] acc_empty[2]
+  // barriers: w_full[8] (+4 unused) w_empty[8] (+4 unused) a_full[8] a_empty[8] acc_full[2] acc_empty[2]
   const uint32_t bar_wfull = smem_u32(bars), bar_wempty = smem_u32(bars + 12);
   const uint32_t bar_afull = smem_u32(bars + 24), bar_aempty = smem_u32(bars + 32);
   const uint32_t bar_accfull = smem_u32(bars + 40), bar_accempty = smem_u32(bars + 42);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 44);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* exp_flag = abort_flag + 1;
   uint32_t* tap_units = tmem_slot + 3;  // [9] row offset of every tap inside a unit
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -146,7 +151,7 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
 
   if (tid < 44) {
     uint32_t count = 1;
-    if (tid < 12) count = 4;                          // w_full: one arrival per lane quarter
+    if (tid < 12) count = CM_LOAD_WARPS;              // w_full: every loader warp arrives
     if (tid >= 24 && tid < 32) count = CM_EXP_THREADS;  // a_full: every expander thread arrives
     if (tid >= 42) count = CM_EPI_WARPS;              // acc_empty: one arrival per epilogue warp
     mbar_init(smem_u32(bars + tid), count);
@@ -187,7 +192,6 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
       const uint32_t unit_units = p.a_unit_bytes >> 4;
       const uint32_t a_step = 2u * (uint32_t)p.Rr;  // two chunks per MMA
       const uint32_t ring = tmem_base + p.ring_col0;
-      const int kpt = p.kpt, KS = p.KS;
       uint32_t tapu[9];
 #pragma unroll
       for (int t = 0; t < 9; ++t) tapu[t] = tap_units[t];
@@ -196,37 +200,39 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
       uint32_t a_phase = 0, w_phase = 0, acc_phase = 1;
       for (int it = 0; it < my_tiles && ok; ++it) {
         if (it >= p.n_acc) {
-          if (!mbar_wait(bar_accempty + 8 * acc_slot, acc_phase)) { ok = false; break; }
+          if (!mbar_wait_backoff(bar_accempty + 8 * acc_slot, acc_phase, 20)) { ok = false; break; }
           tc_fence_after();
         }
         const uint32_t d0 = tmem_base + (uint32_t)(acc_slot * p.Np);
         uint32_t acc = 0;
         const bool wait_w = !(p.w_resident && it > 0);
         if (p.w_resident) { w_slot = 0; w_phase = 0; }
-        int ks = 0, in_stage = 0;
         for (int cb = 0; cb < p.n_cb && ok; ++cb) {
-          if (!mbar_wait(bar_afull + 8 * a_slot, a_phase)) { ok = false; break; }
+          if (!mbar_wait_backoff(bar_afull + 8 * a_slot, a_phase, 20)) { ok = false; break; }
           tc_fence_after();
           const uint32_t unit = b_lo0 + (uint32_t)a_slot * unit_units;
+          uint32_t wbase = 0;
+          // K step j = tap*KPT + k of this block sits in column group j%4 of weight stage j/4
 #pragma unroll
           for (int t = 0; t < 9; ++t) {
-            uint32_t bd = unit + tapu[t];
-            for (int k = 0; k < kpt; ++k) {
-              if (in_stage == 0 && wait_w) {
-                if (!mbar_wait(bar_wfull + 8 * w_slot, w_phase)) { ok = false; break; }
-                tc_fence_after();
+            const uint32_t bt = unit + tapu[t];
+#pragma unroll
+            for (int k = 0; k < KPT; ++k) {
+              const int j = t * KPT + k;
+              if (j % CM_WST == 0) {
+                if (wait_w && ok) {
+                  if (!mbar_wait_backoff(bar_wfull + 8 * w_slot, w_phase, 20)) ok = false;
+                  tc_fence_after();
+                }
+                wbase = ring + (uint32_t)(w_slot * (8 * CM_WST));
               }
-              mma_ts<F16>(d0, ring + (uint32_t)(w_slot * (8 * CM_WST) + in_stage * 8), bd, b_hi, idesc, acc);
+              mma_ts<F16>(d0, wbase + (uint32_t)((j % CM_WST) * 8), bt + (uint32_t)k * a_step, b_hi, idesc, acc);
               acc = 1;
-              bd += a_step;
-              ++ks;
-              if (++in_stage == CM_WST || ks == KS) {
+              if (j % CM_WST == CM_WST - 1 || j == 9 * KPT - 1) {
                 if (!p.w_resident) tc_commit(bar_wempty + 8 * w_slot);  // the ring stage may be overwritten
-                in_stage = 0;
                 if (++w_slot == NW) { w_slot = 0; w_phase ^= 1u; }
               }
             }
-            if (!ok) break;
           }
           tc_commit(bar_aempty + 8 * a_slot);
           if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
@@ -240,66 +246,26 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
       }
     }
     __syncwarp();
-  } else if (warp >= 2 && warp < CM_FIRST_EXP) {
-    // ------------------------------------------------ epilogue warps
-    grid_dep_wait();  // an earlier kernel in the stream may still read the output buffer
-    // Warp w reads TMEM lanes 32*(w%4).. = 32 channels; the two warps of a lane quarter take
-    // alternate 16-position chunks.  Lane l also works out the output pixel of position l%16 of
-    // the chunk, which the warp then reads by shuffle.
-    const int qtr = warp & 3, half = (warp - 2) >> 2;
-    const int nchunk = p.Np >> 4;
-    int acc_slot = 0;
-    uint32_t acc_phase = 0;
-    for (int it = 0; it < my_tiles; ++it) {
-      const int tile = (int)blockIdx.x + it * (int)gridDim.x;
-      const int mg = tile / p.n_cotiles, ct = tile - mg * p.n_cotiles;
-      const uint32_t Q0 = (uint32_t)mg * (uint32_t)p.Np;
-      const int co = ct * 128 + qtr * 32 + lane;
-      const bool co_ok = co < p.K;
-      const float al = (!p.out_i32 && co_ok) ? __ldg(p.alpha + co) : 0.f;
-      int okw = 1;
-      if (lane == 0) okw = (!*abort_flag && mbar_wait_backoff(bar_accfull + 8 * acc_slot, acc_phase, 100)) ? 1 : 0;
-      okw = __shfl_sync(0xffffffffu, okw, 0);
-      if (!okw) {
-        if (lane == 0 && !*abort_flag) {
-          *abort_flag = 1;
-          raise_status(p.status, 4);
-        }
-        break;
-      }
-      tc_fence_after();
-      const uint32_t d0 = tmem_base + (uint32_t)(acc_slot * p.Np) + ((uint32_t)(qtr * 32) << 16);
-      uint32_t* out32 = reinterpret_cast<uint32_t*>(p.out) + co;  // int32 and fp32 outputs share the layout
-      uint32_t v[16];
-      if (half < nchunk) tmem_ld16(d0 + (uint32_t)(half * 16), v);
-#pragma unroll 1
-      for (int c = half; c < nchunk; c += 2) {
-        const int mypix = cm_output_pixel(p, Q0 + (uint32_t)(c * 16 + (lane & 15)));
-        uint32_t u[16];
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 16; ++j)
-          u[j] = p.out_i32 ? v[j] : __float_as_uint(__fmul_rn(F16 ? __uint_as_float(v[j]) : (float)(int)v[j], al));
-        if (c + 2 < nchunk) tmem_ld16(d0 + (uint32_t)((c + 2) * 16), v);  // flies while this chunk is stored
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int pj = __shfl_sync(0xffffffffu, mypix, j);
-          if (pj >= 0 && co_ok) out32[(size_t)pj * (size_t)p.K] = u[j];
-        }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_accempty + 8 * acc_slot);
-      if (++acc_slot == p.n_acc) { acc_slot = 0; acc_phase ^= 1u; }
-    }
-  } else if (warp >= CM_FIRST_EXP && warp < CM_FIRST_LOAD) {
-    // ------------------------------------------------ expanders
-    grid_dep_wait();  // the activations may come from the previous kernel in the stream
-    const int et = tid - CM_FIRST_EXP * 32;
+  } else if (warp >= 2 && warp < CM_FIRST_LOAD) {
+    // ------------------------------------------------ drain warps (2-9) and expanders (10-17)
+    grid_dep_wait();  // activations may come from, and the output may still be read by, the previous kernel
+    const int et = tid - CM_FIRST_EXP * 32;  // rank among the expander threads
     int a_slot = 0, a_done = 0;
     uint32_t a_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
     const int nstep = p.cb_chunks / 2;
-    for (int it = 0; it < my_tiles; ++it) {
+    // Draining: warp w reads TMEM lanes 32*(w%4).. = 32 channels (one per thread); the warps of a lane
+    // quarter take the 16-position chunks in turn.  A chunk is transposed through a 2 KB tile of
+    // shared memory (this kernel leaves half of the shared-memory bandwidth unused), so that a
+    // thread then holds four consecutive channels of one position and a store instruction writes
+    // four full 128-byte lines: the store path takes as long for a 4-byte-per-thread instruction
+    // as for a 16-byte one.
+    const int qtr = warp & 3, sub = (warp - 2) >> 2;
+    const int nchunk = p.Np >> 4;
+    uint8_t* stg = epi_smem + (size_t)(warp - 2) * CM_EPI_STAGE;
+    const int rpos = lane >> 3, cgrp = lane & 7;  // when storing: position (mod 4) and channel group of this lane
+    int acc_slot = 0;
+    uint32_t acc_phase = 0;
+    auto expand_tile = [&](int it) -> bool {
       const int tile = (int)blockIdx.x + it * (int)gridDim.x;
       const int mg = tile / p.n_cotiles;
       const uint32_t Q0 = (uint32_t)mg * (uint32_t)p.Np;
@@ -309,12 +275,13 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
           pix_tab[pl * p.Rr + r] = cm_input_pixel(p, Q0 + (uint32_t)r, pl >> 1, pl & 1);
       for (int cb = 0; cb < p.n_cb; ++cb) {
         if (a_done >= NA) {
-          if (et == 0) *exp_flag = (!*abort_flag && mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 64)) ? 1 : 0;
-          asm volatile("bar.sync 3, %0;" ::"n"(CM_EXP_THREADS) : "memory");
-          const int okf = *exp_flag;
-          asm volatile("bar.sync 3, %0;" ::"n"(CM_EXP_THREADS) : "memory");
+          // every warp polls for itself (one lane, sleeping between attempts): no wait in this
+          // kernel depends on another warp having taken the same exit
+          int okf = 1;
+          if (lane == 0) okf = (!*abort_flag && mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 64)) ? 1 : 0;
+          okf = __shfl_sync(0xffffffffu, okf, 0);
           if (!okf) {
-            if (et == 0 && !*abort_flag) {
+            if (lane == 0 && !*abort_flag) {
               *abort_flag = 1;
               raise_status(p.status, 1);
             }
@@ -408,32 +375,123 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
         ++a_done;
         if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
       }
-      if (stop) break;
+      return !stop;
+    };
+    auto drain_tile = [&](int it) -> bool {
+      const int tile = (int)blockIdx.x + it * (int)gridDim.x;
+      const int mg = tile / p.n_cotiles, ct = tile - mg * p.n_cotiles;
+      const uint32_t Q0 = (uint32_t)mg * (uint32_t)p.Np;
+      const int co4 = ct * 128 + qtr * 32 + cgrp * 4;  // first of the four channels this lane stores
+      float al[4] = {0.f, 0.f, 0.f, 0.f};
+      if (!p.out_i32) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (co4 + e < p.K) al[e] = __ldg(p.alpha + co4 + e);
+      }
+      int okw = 1;
+      if (lane == 0) okw = (!*abort_flag && mbar_wait_backoff(bar_accfull + 8 * acc_slot, acc_phase, 100)) ? 1 : 0;
+      okw = __shfl_sync(0xffffffffu, okw, 0);
+      if (!okw) {
+        if (lane == 0 && !*abort_flag) {
+          *abort_flag = 1;
+          raise_status(p.status, 4);
+        }
+        return false;
+      }
+      tc_fence_after();
+      const uint32_t d0 = tmem_base + (uint32_t)(acc_slot * p.Np) + ((uint32_t)(qtr * 32) << 16);
+      uint32_t* out32 = reinterpret_cast<uint32_t*>(p.out);  // int32 and fp32 outputs share the layout
+      const bool vec = (p.K & 3) == 0;  // groups of 4 channels exist together and are 16-byte aligned
+      uint32_t v[16];
+      if (sub < nchunk) tmem_ld16(d0 + (uint32_t)(sub * 16), v);
+#pragma unroll 1
+      for (int c = sub; c < nchunk; c += CM_EPI_WARPS / 4) {
+        const int mypix = cm_output_pixel(p, Q0 + (uint32_t)(c * 16 + (lane & 15)));
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) *reinterpret_cast<uint32_t*>(stg + j * 128 + lane * 4) = v[j];
+        __syncwarp();
+        if (c + CM_EPI_WARPS / 4 < nchunk) tmem_ld16(d0 + (uint32_t)((c + CM_EPI_WARPS / 4) * 16), v);  // flies while this chunk is stored
+        uint4 w[4];
+        int pj[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          w[r] = *reinterpret_cast<const uint4*>(stg + (r * 4 + rpos) * 128 + cgrp * 16);
+          pj[r] = __shfl_sync(0xffffffffu, mypix, r * 4 + rpos);
+        }
+        if (!p.out_i32) {
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            w[r].x = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].x) : (float)(int)w[r].x, al[0]));
+            w[r].y = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].y) : (float)(int)w[r].y, al[1]));
+            w[r].z = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].z) : (float)(int)w[r].z, al[2]));
+            w[r].w = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].w) : (float)(int)w[r].w, al[3]));
+          }
+        }
+        if (vec) {
+#pragma unroll
+          for (int r = 0; r < 4; ++r)
+            if (pj[r] >= 0 && co4 < p.K) *reinterpret_cast<uint4*>(out32 + (size_t)pj[r] * (size_t)p.K + co4) = w[r];
+        } else {
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            if (pj[r] >= 0) {
+              uint32_t* o = out32 + (size_t)pj[r] * (size_t)p.K + co4;
+              if (co4 + 0 < p.K) o[0] = w[r].x;
+              if (co4 + 1 < p.K) o[1] = w[r].y;
+              if (co4 + 2 < p.K) o[2] = w[r].z;
+              if (co4 + 3 < p.K) o[3] = w[r].w;
+            }
+          }
+        }
+        __syncwarp();  // the tile is rewritten by the next chunk
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_accempty + 8 * acc_slot);
+      if (++acc_slot == p.n_acc) { acc_slot = 0; acc_phase ^= 1u; }
+      return true;
+    };
+    if (warp < CM_FIRST_EXP) {
+      for (int it = 0; it < my_tiles; ++it)
+        if (!drain_tile(it)) break;
+    } else {
+      for (int it = 0; it < my_tiles; ++it)
+        if (!expand_tile(it)) break;
     }
   } else if (warp >= CM_FIRST_LOAD) {
     // ------------------------------------------------ weight loaders
     // The weights are constants of the layer, so there is no wait for the previous kernel.
     const int lw = warp - CM_FIRST_LOAD;
-    const int qtr = warp & 3, pair = lw >> 2;      // lane quarter this warp may write; which of its two warps
+    const int qtr = warp & 3, pair = lw >> 2;      // lane quarter this warp may write; which half of a stage it fills
     const int row = qtr * 32 + lane;               // channel inside the tile
+    const int per_cb = 9 * p.kpt;
     const long long n_stages = p.w_resident ? (long long)p.n_wstages : (long long)my_tiles * p.n_wstages;
-    for (long long g = pair; g < n_stages; g += 2) {
+    uint32_t v[32];
+    // this warp's half of stage g -> registers; returns the number of K steps in it (<= 0: none)
+    auto load_half = [&](long long g) -> int {
       const int it = (int)(g / p.n_wstages), s = (int)(g - (long long)it * p.n_wstages);
       const int tile = (int)blockIdx.x + it * (int)gridDim.x;
       const int ct = tile % p.n_cotiles;
-      const int ks0 = s * CM_WST;
-      const uint8_t* src = p.wa + (((size_t)ct * p.KS + ks0) * 128 + row) * 32;
-      uint32_t v[32];
+      const int cb = s / p.spc, si = s - cb * p.spc;
+      const int first = si * CM_WST + pair * 4;   // first K step of the half inside the channel block
+      const int nks = min(4, per_cb - first);
+      // a warp reads 512 contiguous bytes per instruction: the two halves of a K step's rows are stored apart
+      const uint8_t* src = p.wa + ((size_t)ct * p.KS + (size_t)cb * per_cb + first) * 4096 + (size_t)row * 16;
 #pragma unroll
-      for (int j = 0; j < CM_WST; ++j) {
+      for (int j = 0; j < 4; ++j) {
         uint4 x = make_uint4(0, 0, 0, 0), y = x;
-        if (ks0 + j < p.KS) {
-          x = __ldg(reinterpret_cast<const uint4*>(src + (size_t)j * 128 * 32));
-          y = __ldg(reinterpret_cast<const uint4*>(src + (size_t)j * 128 * 32 + 16));
+        if (j < nks) {
+          x = __ldg(reinterpret_cast<const uint4*>(src + (size_t)j * 4096));
+          y = __ldg(reinterpret_cast<const uint4*>(src + (size_t)j * 4096 + 2048));
         }
         v[8 * j + 0] = x.x; v[8 * j + 1] = x.y; v[8 * j + 2] = x.z; v[8 * j + 3] = x.w;
         v[8 * j + 4] = y.x; v[8 * j + 5] = y.y; v[8 * j + 6] = y.z; v[8 * j + 7] = y.w;
       }
+      return nks;
+    };
+    int nks = n_stages > 0 ? load_half(0) : 0;
+    for (long long g = 0; g < n_stages; ++g) {
       const int slot = (int)(g % NW);
       const long long use = g / NW;
       if (use >= 1) {
@@ -450,8 +508,13 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
         }
         tc_fence_after();
       }
-      tmem_st32(tmem_base + p.ring_col0 + (uint32_t)(slot * 8 * CM_WST) + ((uint32_t)(qtr * 32) << 16), v);
-      tmem_st_wait();
+      const bool stored = nks > 0;
+      if (stored)
+        tmem_st32(tmem_base + p.ring_col0 + (uint32_t)(slot * 8 * CM_WST + pair * 32) + ((uint32_t)(qtr * 32) << 16), v);
+      // The store has read its registers once it is issued: the next stage's loads go out now
+      // and fly while the store completes and the stage is published.
+      if (g + 1 < n_stages) nks = load_half(g + 1);
+      if (stored) tmem_st_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_wfull + 8 * slot);
@@ -467,18 +530,20 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
 }
 
 // ------------------------------------------------------------ create-time operand
-// wa[channel tile][K step][128][32 B]; K step ks = (block*9 + tap)*kpt + k holds the 32 int8
-// (16 fp16) channels of chunks 2k, 2k+1 of channel block `block`; rows past c_out are zero.
+// wa[channel tile][K step][half][128][16 B]; K step ks = (block*9 + tap)*kpt + k holds the 32 int8
+// (16 fp16) channels of chunks 2k (half 0) and 2k+1 (half 1) of channel block `block`; rows past
+// c_out are zero.
 template <bool F16>
 __global__ void cm_expand_weights_kernel(const uint32_t* __restrict__ wplanes, uint8_t* __restrict__ wa, int C, int K,
                                          int Cw, long long total, int cb_chunks, int n_cb) {
   // one thread per 16-byte half row
   long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
   if (i >= total) return;
-  const int hf = (int)(i & 1);
-  long long r = i >> 1;
+  long long r = i;
   const int row = (int)(r % 128);
   r /= 128;
+  const int hf = (int)(r & 1);
+  r >>= 1;
   const int kpt = cb_chunks / 2;
   const int KS = 9 * n_cb * kpt;
   const int ks = (int)(r % KS), ct = (int)(r / KS);
@@ -542,7 +607,7 @@ struct CmPlan {
 constexpr size_t kCmSmemBudget = 226 * 1024;
 
 // positions per tile offered as variants
-const int kCmNp[] = {128, 256, 112, 176, 64, 192};
+const int kCmNp[] = {128, 256, 96, 176, 64, 192};
 constexpr int kCmVariants = (int)(sizeof(kCmNp) / sizeof(kCmNp[0]));
 
 CmPlan cm_plan(const Geom& g, int act_type, int Np) {
@@ -558,7 +623,8 @@ CmPlan cm_plan(const Geom& g, int act_type, int Np) {
   p.n_cb = n_chunks / p.cb_chunks;
   p.kpt = p.cb_chunks / 2;
   p.KS = 9 * p.n_cb * p.kpt;
-  p.n_wstages = (p.KS + CM_WST - 1) / CM_WST;
+  p.spc = (9 * p.kpt + CM_WST - 1) / CM_WST;
+  p.n_wstages = p.n_cb * p.spc;
   if (g.stride == 1) {
     p.Hq = g.H + g.pad; p.Wq = g.W + g.pad; p.n_planes = 1; p.halo = 2 * p.Wq + 2;
   } else {
@@ -594,7 +660,8 @@ CmPlan cm_plan(const Geom& g, int act_type, int Np) {
   const size_t unit_exact = (size_t)p.n_planes * p.cb_chunks * p.Rr * 16;
   p.a_unit_bytes = (uint32_t)((unit_exact + 127) & ~(size_t)127);
   const size_t pix_bytes = ((size_t)p.n_planes * p.Rr * 4 + 127) & ~(size_t)127;
-  const size_t fixed = pix_bytes + kCmTail;
+  const size_t epi_bytes = (size_t)CM_EPI_WARPS * CM_EPI_STAGE;
+  const size_t fixed = pix_bytes + epi_bytes + kCmTail;
   if (p.a_unit_bytes + fixed > kCmSmemBudget) return pl;
   long long na = (long long)((kCmSmemBudget - fixed) / p.a_unit_bytes);
   const long long units_per_cta = (long long)tiles_per_cta * p.n_cb;
@@ -603,7 +670,8 @@ CmPlan cm_plan(const Geom& g, int act_type, int Np) {
   if (int v = env_int("SNN_CM_NA", 0)) if (v >= 1 && v < na) na = v;
   p.NA = (int)na;
   p.off_pix = (uint32_t)((size_t)p.NA * p.a_unit_bytes);
-  p.off_tail = p.off_pix + (uint32_t)pix_bytes;
+  p.off_epi = p.off_pix + (uint32_t)pix_bytes;
+  p.off_tail = p.off_epi + (uint32_t)epi_bytes;
   pl.smem = (size_t)p.off_tail + kCmTail;
   if (pl.smem > (size_t)kMaxDynSmem || pl.smem >= (1u << 18)) return pl;   // descriptor address range
   if ((uint32_t)p.Rr * 16 >= (1u << 18)) return pl;                        // leading-offset field range
@@ -657,16 +725,24 @@ cudaError_t cm_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l
   cfg.gridDim = pl.grid;
   cfg.blockDim = dim3(CM_THREADS);
   cfg.dynamicSmemBytes = pl.smem;
-  cudaError_t e;
-  if (f16) {
-    static unsigned long long done = 0;
-    e = allow_max_smem(cm_conv_kernel<true>, &done);
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, cm_conv_kernel<true>, p);
-  } else {
-    static unsigned long long done = 0;
-    e = allow_max_smem(cm_conv_kernel<false>, &done);
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, cm_conv_kernel<false>, p);
-  }
+  cudaError_t e = cudaErrorInvalidConfiguration;
+#define SNN_CM_LAUNCH(F, KP)                                                          \
+  do {                                                                                \
+    static unsigned long long done = 0;                                               \
+    e = allow_max_smem(cm_conv_kernel<F, KP>, &done);                                 \
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, cm_conv_kernel<F, KP>, p);     \
+  } while (0)
+#define SNN_CM_LAUNCH_K(F)                     \
+  do {                                         \
+    if (p.kpt == 4) SNN_CM_LAUNCH(F, 4);       \
+    else if (p.kpt == 3) SNN_CM_LAUNCH(F, 3);  \
+    else if (p.kpt == 2) SNN_CM_LAUNCH(F, 2);  \
+    else if (p.kpt == 1) SNN_CM_LAUNCH(F, 1);  \
+  } while (0)
+  if (f16) SNN_CM_LAUNCH_K(true);
+  else SNN_CM_LAUNCH_K(false);
+#undef SNN_CM_LAUNCH_K
+#undef SNN_CM_LAUNCH
   if (e != cudaSuccess) return e;
   *launched += 1;
   return cudaGetLastError();
