@@ -168,6 +168,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if (warp >= 2 + EPI_WARPS) {
+    // The expanders' table for their first tile (input pixel of every staged row, -1 = padding)
+    // depends on nothing but the parameters: it is worked out here, beside the set-up and before
+    // the wait for the previous kernel.  A thread reads back only entries it wrote itself.
+    const int et0 = tid - (2 + EPI_WARPS) * 32;
+    const uint32_t Q00 = (uint32_t)((int)blockIdx.x / p.n_ntiles) * (uint32_t)(128 * MT);
+    for (int pl = 0; pl < p.n_planes; ++pl)
+      for (int r = et0; r < p.Rr; r += EXP_THREADS)
+        pix_tab[pl * p.Rr + r] = position_to_pixel(p, Q00 + (uint32_t)r, pl >> 1, pl & 1);
+  }
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   tc_fence_before();
   __syncthreads();
@@ -440,11 +450,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       const int mg = tile / p.n_ntiles;
       const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
       bool stop = false;
-      // input pixel of every staged row, once per tile: -1 where the row is padding.  A thread
-      // reads back only the entries it wrote, so no barrier is needed.
-      for (int pl = 0; pl < p.n_planes; ++pl)
-        for (int r = et; r < p.Rr; r += EXP_THREADS)
-          pix_tab[pl * p.Rr + r] = position_to_pixel(p, Q0 + (uint32_t)r, pl >> 1, pl & 1);
+      // input pixel of every staged row, once per tile (the first tile's table was made during set-up)
+      if (tile != (int)blockIdx.x)
+        for (int pl = 0; pl < p.n_planes; ++pl)
+          for (int r = et; r < p.Rr; r += EXP_THREADS)
+            pix_tab[pl * p.Rr + r] = position_to_pixel(p, Q0 + (uint32_t)r, pl >> 1, pl & 1);
       for (int cb = 0; cb < p.n_cb; ++cb) {
         if (a_done >= NA) {
           // one elected thread polls; the rest wait on a hardware barrier instead of spinning

@@ -172,6 +172,16 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if (warp >= CM_FIRST_EXP && warp < CM_FIRST_LOAD) {
+    // The expanders' table for their first tile (input pixel of every staged row, -1 = padding)
+    // depends on nothing but the parameters: it is worked out here, beside the set-up and before
+    // the wait for the previous kernel.  A thread reads back only entries it wrote itself.
+    const int et0 = tid - CM_FIRST_EXP * 32;
+    const uint32_t Q00 = (uint32_t)((int)blockIdx.x / p.n_cotiles) * (uint32_t)p.Np;
+    for (int pl = 0; pl < p.n_planes; ++pl)
+      for (int r = et0; r < p.Rr; r += CM_EXP_THREADS)
+        pix_tab[pl * p.Rr + r] = cm_input_pixel(p, Q00 + (uint32_t)r, pl >> 1, pl & 1);
+  }
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   tc_fence_before();
   __syncthreads();
@@ -270,9 +280,10 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
       const int mg = tile / p.n_cotiles;
       const uint32_t Q0 = (uint32_t)mg * (uint32_t)p.Np;
       bool stop = false;
-      for (int pl = 0; pl < p.n_planes; ++pl)
-        for (int r = et; r < p.Rr; r += CM_EXP_THREADS)
-          pix_tab[pl * p.Rr + r] = cm_input_pixel(p, Q0 + (uint32_t)r, pl >> 1, pl & 1);
+      if (it > 0)  // the first tile's table was made during set-up
+        for (int pl = 0; pl < p.n_planes; ++pl)
+          for (int r = et; r < p.Rr; r += CM_EXP_THREADS)
+            pix_tab[pl * p.Rr + r] = cm_input_pixel(p, Q0 + (uint32_t)r, pl >> 1, pl & 1);
       for (int cb = 0; cb < p.n_cb; ++cb) {
         if (a_done >= NA) {
           // every warp polls for itself (one lane, sleeping between attempts): no wait in this
