@@ -63,13 +63,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (mbar_try(bar, parity)) return true;
   return false;
 }
-// The same for a thread whose wait is not on the critical path: it sleeps
-// between attempts so that its polling does not crowd the issuing threads.
+// try_wait with a suspend-time hint: the hardware parks the thread until the phase completes
+// or about `ns` nanoseconds have passed, so a waiting thread issues almost no instructions
+// and wakes as soon as the barrier flips.
+__device__ __forceinline__ uint32_t mbar_try_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
+      : "memory");
+  return ok;
+}
+// Bounded wait for a thread whose wait is not on the critical path.  `ns` scales the time the
+// hardware may keep the thread parked per attempt; the attempt limit bounds the whole wait
+// (to a second or so) whatever the hardware makes of the hint.
 __device__ __forceinline__ bool mbar_wait_backoff(uint32_t bar, uint32_t parity, uint32_t ns) {
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-    if (mbar_try(bar, parity)) return true;
-    __nanosleep(ns);
-  }
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
+    if (mbar_try_hint(bar, parity, 20u * ns)) return true;
   return false;
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
