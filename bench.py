@@ -207,6 +207,11 @@ def run_ours(args):
     forced = {"auto": snn.PATH_AUTO, "reuse": snn.PATH_REUSE, "decoded": snn.PATH_DECODED,
               "decoded_tc": snn.PATH_DECODED_TC}[args.path]
 
+    # Micro-batches: the batch is cut into `mb` equal parts, each of which runs the layers in order on
+    # a stream of its own, so that one part's kernel start-up and tail overlap the other parts' work.
+    mb = max(1, args.microbatch)
+    if nb % mb:
+        raise SystemExit(f"--microbatch {mb} does not divide the batch {nb}")
     layers, acts, outs, host_acts, host_outs, paths = [], [], [], [], [], []
     for i, shape in enumerate(workload.layers, start=first_layer):
         seed = wl.layer_seed(workload.config, i) + 7919 * rank
@@ -222,16 +227,31 @@ def run_ours(args):
         outs.append(layer.alloc_out(nb, shape.h, shape.w))
         host_outs.append(layer.alloc_out(nb, shape.h, shape.w, pin=True))
         if forced == snn.PATH_AUTO:
-            layer.tune(nb, shape.h, shape.w)
-        paths.append(layer.chosen_path(nb, shape.h, shape.w) if forced == snn.PATH_AUTO else forced)
+            layer.tune(nb // mb, shape.h, shape.w)
+        paths.append(layer.chosen_path(nb // mb, shape.h, shape.w) if forced == snn.PATH_AUTO else forced)
         layers.append(layer)
 
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)  # > 126 MB L2
     side = torch.cuda.Stream(dev)
 
-    def launch_layers(idxs, stream):
+    part = nb // mb
+    part_streams = [torch.cuda.Stream(dev) for _ in range(mb - 1)]
+
+    def launch_part(idxs, m, stream):
         for j in idxs:
-            layers[j].forward(acts[j], outs[j], snn.OUT_F32, paths[j], stream)
+            layers[j].forward(acts[j][m * part:(m + 1) * part], outs[j][m * part:(m + 1) * part], snn.OUT_F32,
+                              paths[j], stream)
+
+    def launch_layers(idxs, stream):
+        """One pass over layers `idxs`: micro-batch 0 on `stream`, the others on streams forked from
+        and joined back into it (the pattern stream capture needs)."""
+        for ps in part_streams:
+            ps.wait_stream(stream)
+        launch_part(idxs, 0, stream)
+        for m, ps in enumerate(part_streams, start=1):
+            launch_part(idxs, m, ps)
+        for ps in part_streams:
+            stream.wait_stream(ps)
 
     def capture(idxs):
         """The launches of one step (or one layer) as a CUDA graph, so that the host's
@@ -278,7 +298,7 @@ def run_ours(args):
         e1.record(stream)
     barrier()
     wall = time.perf_counter() - wall0
-    launches = (snn.kernel_launches() - launches0) if not use_graph else len(layers) * args.steps
+    launches = (snn.kernel_launches() - launches0) if not use_graph else len(layers) * mb * args.steps
     step_ms = [e0.elapsed_time(e1) for e0, e1 in ev]
     total_ms = float(sum(step_ms))
 
@@ -369,7 +389,9 @@ def run_ours(args):
         "dtype": "int32" if workload.act == "bin" else "f16", "data": "synthetic",
         "config": {"workload": _workload_name(workload), "layers": len(layers), "batch_per_gpu": nb,
                    "tau": workload.tau, "l2": "flushed between timed steps (256 MB write)",
-                   "launch": "host calls" if args.no_graph else "CUDA graph of the per-layer C-ABI launches",
+                   "launch": ("host calls" if args.no_graph else "CUDA graph of the per-layer C-ABI launches") +
+                             (f", {mb} micro-batches of {part} images on {mb} streams" if mb > 1 else ""),
+                   "microbatches": mb,
                    "paths": [snn.PATH_NAMES[p] for p in paths]},
         "effective_tops": 2 * workload.dense_macs() * world / (ms_per_step * 1e-3) / 1e12,
         "hbm_floor_ms_per_step": step_floor_hbm_ms,
@@ -414,6 +436,8 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "reuse", "decoded", "decoded_tc"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--microbatch", type=int, default=1,
+                    help="cut the batch into this many parts, each running the layers in order on its own stream")
     ap.add_argument("--no-graph", action="store_true", help="launch every layer from the host instead of a CUDA graph")
     ap.add_argument("--layers", default=None, help="a:b restricts the stack to layers [a, b) (profiling aid)")
     args = ap.parse_args()

@@ -57,12 +57,6 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok;
 }
-// Bounded wait for the phase with the given parity; false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
-    if (mbar_try(bar, parity)) return true;
-  return false;
-}
 // try_wait with a suspend-time hint: the hardware parks the thread until the phase completes
 // or about `ns` nanoseconds have passed, so a waiting thread issues almost no instructions
 // and wakes as soon as the barrier flips.
@@ -76,6 +70,12 @@ __device__ __forceinline__ uint32_t mbar_try_hint(uint32_t bar, uint32_t parity,
       : "r"(bar), "r"(parity), "r"(ns)
       : "memory");
   return ok;
+}
+// Bounded wait for the phase with the given parity; false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
+    if (mbar_try_hint(bar, parity, 1000u)) return true;
+  return false;
 }
 // Bounded wait for a thread whose wait is not on the critical path.  `ns` scales the time the
 // hardware may keep the thread parked per attempt; the attempt limit bounds the whole wait
