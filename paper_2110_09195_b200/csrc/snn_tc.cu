@@ -118,7 +118,7 @@ __device__ __forceinline__ void epilogue_slice(const TcParams& p, uint32_t taddr
 #pragma unroll
     for (int e = 0; e < NC; ++e)
       if (co0 + e < p.K)
-        o[e] = __fmul_rn(F16 ? __uint_as_float(v[e]) : (float)(int)v[e], __ldg(p.alpha + co0 + e));
+        o[e] = __fmul_rn(F16 ? __uint_as_float(v[e]) : small_int_to_float(v[e]), __ldg(p.alpha + co0 + e));
   }
 }
 
@@ -399,10 +399,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
             if (!p.out_i32) {
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                u[i].x = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].x) : (float)(int)u[i].x, al.x));
-                u[i].y = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].y) : (float)(int)u[i].y, al.y));
-                u[i].z = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].z) : (float)(int)u[i].z, al.z));
-                u[i].w = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].w) : (float)(int)u[i].w, al.w));
+                u[i].x = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].x) : small_int_to_float(u[i].x), al.x));
+                u[i].y = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].y) : small_int_to_float(u[i].y), al.y));
+                u[i].z = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].z) : small_int_to_float(u[i].z), al.z));
+                u[i].w = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].w) : small_int_to_float(u[i].w), al.w));
               }
             }
             uint32_t* obase32 = reinterpret_cast<uint32_t*>(p.out) + co;  // int32 and fp32 outputs share the layout
@@ -674,6 +674,7 @@ static TcPlan plan_for(const Geom& g, int act_type, int MT, int stage_kb) {
   p.dHq = make_fastdiv((uint32_t)p.Hq);
   p.Qtot = (long long)g.N * p.Hq * p.Wq;
   if (p.Qtot + 1024 + p.halo >= (1ll << 31)) return pl;  // positions are 32-bit in the kernels
+  if (g.C > kMaxChannelsSmallInt) return pl;             // the drain's int -> float shortcut
   if ((long long)g.N * g.H * g.W >= (1ll << 31)) return pl;
   const long long mtiles = (p.Qtot + 127) / 128;
   const int sms = sm_count();

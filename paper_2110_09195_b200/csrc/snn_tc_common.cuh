@@ -197,6 +197,15 @@ __device__ __forceinline__ void expand_word(uint32_t bits, int channels_left, bo
   }
 }
 
+// int32 -> float for |s| < 2^22 without the conversion unit (which handles only 16 lanes per SM
+// and clock and was the slowest step of the accumulator drain): adding s to the bit pattern of
+// 1.5 * 2^23 gives the float 1.5 * 2^23 + s exactly, and the subtraction is exact too.  The sums of
+// a 3x3 layer are bounded by 9 * c_in, so the launch plans require 9 * c_in < 2^22.
+__device__ __forceinline__ float small_int_to_float(uint32_t s) {
+  return __fadd_rn(__uint_as_float(0x4B400000u + s), -12582912.0f);
+}
+constexpr int kMaxChannelsSmallInt = ((1 << 22) - 1) / 9;
+
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 static inline int env_int(const char* name, int dflt) {

@@ -433,10 +433,10 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
         if (!p.out_i32) {
 #pragma unroll
           for (int r = 0; r < 4; ++r) {
-            w[r].x = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].x) : (float)(int)w[r].x, al[0]));
-            w[r].y = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].y) : (float)(int)w[r].y, al[1]));
-            w[r].z = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].z) : (float)(int)w[r].z, al[2]));
-            w[r].w = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].w) : (float)(int)w[r].w, al[3]));
+            w[r].x = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].x) : small_int_to_float(w[r].x), al[0]));
+            w[r].y = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].y) : small_int_to_float(w[r].y), al[1]));
+            w[r].z = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].z) : small_int_to_float(w[r].z), al[2]));
+            w[r].w = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(w[r].w) : small_int_to_float(w[r].w), al[3]));
           }
         }
         if (vec) {
@@ -645,6 +645,7 @@ CmPlan cm_plan(const Geom& g, int act_type, int Np) {
   p.dHq = make_fastdiv((uint32_t)p.Hq);
   p.Qtot = (long long)g.N * p.Hq * p.Wq;
   if (p.Qtot + 1024 + p.halo >= (1ll << 31)) return pl;  // positions are 32-bit in the kernel
+  if (g.C > kMaxChannelsSmallInt) return pl;             // the drain's int -> float shortcut
   if ((long long)g.N * g.H * g.W >= (1ll << 31) || (long long)g.N * g.Ho * g.Wo >= (1ll << 31)) return pl;
   p.Np = Np;
   p.Rr = Np + p.halo;
