@@ -200,6 +200,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       // already requested, so that the first ones can be requested before the expanded
       // activations exist (the weights are constants of the layer).
       long long w_next = 0;
+      int w_cb = 0, w_sg = 0;
       auto issue_weights = [&](int tile, long long upto) -> bool {
         // requests stages [w_next, upto) of this CTA's stage sequence, stopping when the ring is full
         const int nti = tile % p.n_ntiles;
@@ -207,8 +208,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
         const size_t wtile = (size_t)(n0 / p.NtL) * p.n_cb;
         const int n_in = n0 % p.NtL;
         while (w_next < upto) {
-          const int in_tile = (int)(w_next % stages_per_tile);
-          const int cb = in_tile / stages_per_cb, sg = in_tile - cb * stages_per_cb;
+          const int cb = w_cb, sg = w_sg;  // position inside the tile, kept as counters (no divisions)
+          if (++w_sg == stages_per_cb) {
+            w_sg = 0;
+            if (++w_cb == p.n_cb) w_cb = 0;
+          }
           if (b_issued >= NS && !mbar_wait_backoff(bar_bempty + 8 * b_slot, b_phase, 32)) return false;
           const uint32_t dst = smem_u32(b_smem) + (uint32_t)b_slot * p.stage_bytes;
           const uint8_t* src =
@@ -344,14 +348,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       tc_fence_after();
       const uint32_t d0 = tmem_base + (uint32_t)acc_slot * acc_cols;
       // row of sub-tile mt this lane owns in TMEM -> is it an output, and where does it go
-      auto row_info = [&](int mt, bool* valid, size_t* obase) {
+      // output pixel (n*Ho + y)*Wo + x, or -1 when the row is not an output
+      auto row_pixel = [&](int mt) -> int {
         const uint32_t q = Q0 + (uint32_t)(mt * 128 + rq * 32 + lane);
         const uint32_t rg = fdiv(q, p.dWq);
         const int x = (int)(q - rg * (uint32_t)p.Wq);
         const uint32_t n = fdiv(rg, p.dHq);
         const int y = (int)(rg - n * (uint32_t)p.Hq);
-        *valid = ((long long)q < p.Qtot) && ((int)n < p.N) && (y < p.Ho) && (x < p.Wo);
-        *obase = (((size_t)n * p.Ho + y) * p.Wo + x) * p.K;
+        const bool valid = ((long long)q < p.Qtot) && ((int)n < p.N) && (y < p.Ho) && (x < p.Wo);
+        return valid ? ((int)n * p.Ho + y) * p.Wo + x : -1;
       };
       if (fast) {
         // The warp's slices (sub-tile mt, columns c0..c0+31) form one sequence.  The TMEM load of
@@ -362,15 +367,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
         uint32_t v[32];
         int ro[8];
         if (total > 0) tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(32 * half), v);
+        int mt = 0, ci = 0;  // slice = (sub-tile mt, this warp's ci-th slice of it); no divisions in the loop
 #pragma unroll 1
         for (int sl = 0; sl < total; ++sl) {
-          const int mt = sl / per_mt, c0 = 32 * half + 64 * (sl - mt * per_mt);
-          if (sl - mt * per_mt == 0) {
+          const int c0 = 32 * half + 64 * ci;
+          if (ci == 0) {
             // output pixels of the eight rows this lane stores (row = srow + 4*i), -1 when not an output
-            bool valid;
-            size_t obase;
-            row_info(mt, &valid, &obase);
-            const int mine = valid ? (int)(obase / (size_t)p.K) : -1;  // output pixel (fits: pixels are 32-bit here)
+            const int mine = row_pixel(mt);
 #pragma unroll
             for (int i = 0; i < 8; ++i) ro[i] = __shfl_sync(0xffffffffu, mine, srow + 4 * i);
           }
@@ -383,10 +386,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
             *reinterpret_cast<uint4*>(stage + lane * EPI_PITCH + ((e ^ (lane & 7)) << 4)) =
                 make_uint4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
           __syncwarp();
-          if (sl + 1 < total) {
-            const int nmt = (sl + 1) / per_mt, nc0 = 32 * half + 64 * (sl + 1 - nmt * per_mt);
-            tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(nmt * p.Nt + nc0), v);
-          }
+          const int this_mt = mt;
+          if (++ci == per_mt) { ci = 0; ++mt; }
+          if (sl + 1 < total)
+            tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt + 32 * half + 64 * ci), v);
+          (void)this_mt;
           if (co < p.K) {  // K is a multiple of 4 here, so the four channels exist together
             // loads and conversions first, the (predicated) stores last: no branch sits between
             // the eight independent chains, so their latencies overlap
@@ -415,9 +419,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       } else {
 #pragma unroll 1
         for (int mt = 0; mt < MT; ++mt) {
-          bool valid;
-          size_t obase;
-          row_info(mt, &valid, &obase);
+          const int pix = row_pixel(mt);
+          const bool valid = pix >= 0;
+          const size_t obase = (size_t)(valid ? pix : 0) * (size_t)p.K;
           const uint32_t trow = d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt);
           if ((p.Nt & 31) == 0) {
             for (int c0 = 32 * half; c0 < p.Nt; c0 += 64)

@@ -479,12 +479,21 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
     const int per_cb = 9 * p.kpt;
     const long long n_stages = p.w_resident ? (long long)p.n_wstages : (long long)my_tiles * p.n_wstages;
     uint32_t v[32];
-    // this warp's half of stage g -> registers; returns the number of K steps in it (<= 0: none)
-    auto load_half = [&](long long g) -> int {
-      const int it = (int)(g / p.n_wstages), s = (int)(g - (long long)it * p.n_wstages);
-      const int tile = (int)blockIdx.x + it * (int)gridDim.x;
-      const int ct = tile % p.n_cotiles;
-      const int cb = s / p.spc, si = s - cb * p.spc;
+    // Position of the next stage to load: channel tile of the CTA's current tile, channel block,
+    // stage inside the block; kept as counters, because divisions by run-time values are slow.
+    int ld_ct = (int)blockIdx.x % p.n_cotiles, ld_cb = 0, ld_si = 0;
+    const int ct_step = (int)gridDim.x % p.n_cotiles;  // 0 when the grid is a multiple of the channel tiles
+    // this warp's half of the next stage -> registers; returns the number of K steps in it (<= 0: none)
+    auto load_half = [&]() -> int {
+      const int ct = ld_ct, cb = ld_cb, si = ld_si;
+      if (++ld_si == p.spc) {
+        ld_si = 0;
+        if (++ld_cb == p.n_cb) {
+          ld_cb = 0;
+          ld_ct += ct_step;
+          if (ld_ct >= p.n_cotiles) ld_ct -= p.n_cotiles;
+        }
+      }
       const int first = si * CM_WST + pair * 4;   // first K step of the half inside the channel block
       const int nks = min(4, per_cb - first);
       // a warp reads 512 contiguous bytes per instruction: the two halves of a K step's rows are stored apart
@@ -501,10 +510,10 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
       }
       return nks;
     };
-    int nks = n_stages > 0 ? load_half(0) : 0;
+    int nks = n_stages > 0 ? load_half() : 0;
+    int slot = 0;
+    uint32_t use = 0;  // laps of the ring so far
     for (long long g = 0; g < n_stages; ++g) {
-      const int slot = (int)(g % NW);
-      const long long use = g / NW;
       if (use >= 1) {
         int okw = 1;
         if (lane == 0)
@@ -524,11 +533,12 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
         tmem_st32(tmem_base + p.ring_col0 + (uint32_t)(slot * 8 * CM_WST + pair * 32) + ((uint32_t)(qtr * 32) << 16), v);
       // The store has read its registers once it is issued: the next stage's loads go out now
       // and fly while the store completes and the stage is published.
-      if (g + 1 < n_stages) nks = load_half(g + 1);
+      if (g + 1 < n_stages) nks = load_half();
       if (stored) tmem_st_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_wfull + 8 * slot);
+      if (++slot == NW) { slot = 0; ++use; }
     }
   }
 
