@@ -63,7 +63,7 @@ struct TcParams {
   int Kpad, n_chunks;     // padded channels out; 16-byte chunks along the padded channels in
   int NtL;                // channels per layout tile of the weight operand
   int Hq, Wq;             // rows per image / row pitch of the flattened position space
-  FastDiv dWq, dHq;
+  FastDiv dWq, dHq, dNt;  // exact division by Wq, Hq and the number of channel tiles
   int n_planes;           // 1 (stride 1) or 4 (stride 2)
   int halo;               // largest tap shift in rows
   int Rr;                 // staged rows per plane = 128*MT + halo
@@ -203,10 +203,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
       int w_cb = 0, w_sg = 0;
       auto issue_weights = [&](int tile, long long upto) -> bool {
         // requests stages [w_next, upto) of this CTA's stage sequence, stopping when the ring is full
-        const int nti = tile % p.n_ntiles;
+        const int nti = tile - (int)fdiv((uint32_t)tile, p.dNt) * p.n_ntiles;
         const int n0 = nti * p.Nt;
-        const size_t wtile = (size_t)(n0 / p.NtL) * p.n_cb;
-        const int n_in = n0 % p.NtL;
+        // channel tile -> layout tile of the weight operand (the same thing unless a narrower tile was asked for)
+        const int ltile = p.Nt == p.NtL ? nti : n0 / p.NtL;
+        const size_t wtile = (size_t)ltile * p.n_cb;
+        const int n_in = n0 - ltile * p.NtL;
         while (w_next < upto) {
           const int cb = w_cb, sg = w_sg;  // position inside the tile, kept as counters (no divisions)
           if (++w_sg == stages_per_cb) {
@@ -332,7 +334,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
     int acc_slot = 0;
     uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
-      const int mg = tile / p.n_ntiles, nti = tile - mg * p.n_ntiles;
+      const int mg = (int)fdiv((uint32_t)tile, p.dNt), nti = tile - mg * p.n_ntiles;
       const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
       const int n0 = nti * p.Nt;
       int okw = 1;
@@ -412,7 +414,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
             uint32_t* obase32 = reinterpret_cast<uint32_t*>(p.out) + co;  // int32 and fp32 outputs share the layout
 #pragma unroll
             for (int i = 0; i < 8; ++i)
-              if (ro[i] >= 0) *reinterpret_cast<uint4*>(obase32 + (size_t)ro[i] * (size_t)p.K) = u[i];
+              if (ro[i] >= 0) *reinterpret_cast<uint4*>(obase32 + wide_mul((uint32_t)ro[i], (uint32_t)p.K)) = u[i];
           }
           __syncwarp();
         }
@@ -451,7 +453,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
     volatile int* exp_flag = abort_flag + 1;
     const int nstep = p.cb_chunks / 2;  // pairs of chunks per unit
     for (int tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
-      const int mg = tile / p.n_ntiles;
+      const int mg = (int)fdiv((uint32_t)tile, p.dNt);
       const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
       bool stop = false;
       // input pixel of every staged row, once per tile (the first tile's table was made during set-up)
@@ -495,7 +497,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
                     v[j][k] = make_uint4(0, 0, 0, 0);
                     const int ch = (cb * p.cb_chunks + c0 + k) * 8;  // first channel of the chunk
                     if (pix[j] >= 0 && ch < p.C) {
-                      const __half* src = (const __half*)p.act + (size_t)pix[j] * p.C + ch;
+                      const __half* src = (const __half*)p.act + wide_mul((uint32_t)pix[j], (uint32_t)p.C) + ch;
                       if (p.act_vec) {
                         v[j][k] = __ldg(reinterpret_cast<const uint4*>(src));
                       } else {
@@ -525,7 +527,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
               for (int j = 0; j < EXP_ROWS; ++j) {
                 bits[j][0] = bits[j][1] = bits[j][2] = bits[j][3] = 0;
                 if (pix[j] >= 0 && w0 < p.Cw) {
-                  const uint32_t* src = (const uint32_t*)p.act + (size_t)pix[j] * p.Cw + w0;
+                  const uint32_t* src = (const uint32_t*)p.act + wide_mul((uint32_t)pix[j], (uint32_t)p.Cw) + w0;
                   if (p.act_vec && nstep == 4) {
                     const uint4 t = __ldg(reinterpret_cast<const uint4*>(src));
                     bits[j][0] = t.x; bits[j][1] = t.y; bits[j][2] = t.z; bits[j][3] = t.w;
@@ -688,6 +690,7 @@ static TcPlan plan_for(const Geom& g, int act_type, int MT, int stage_kb) {
   if (forced_nt >= 16 && forced_nt <= 256 && forced_nt % 16 == 0 && p.NtL % forced_nt == 0) Nt = forced_nt;
   p.Nt = Nt;
   p.n_ntiles = Kpad / Nt;
+  p.dNt = make_fastdiv((uint32_t)p.n_ntiles);
   if (MT * Nt > 512) return pl;
   p.MT = MT;
   p.Rr = 128 * MT + p.halo;

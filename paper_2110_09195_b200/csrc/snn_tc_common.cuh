@@ -204,6 +204,9 @@ __device__ __forceinline__ void expand_word(uint32_t bits, int channels_left, bo
 __device__ __forceinline__ float small_int_to_float(uint32_t s) {
   return __fadd_rn(__uint_as_float(0x4B400000u + s), -12582912.0f);
 }
+// 32 x 32 -> 64-bit product in one instruction (element offsets of pixels: both factors are non-negative 32-bit)
+__device__ __forceinline__ size_t wide_mul(uint32_t a, uint32_t b) { return (size_t)a * (size_t)b; }
+
 constexpr int kMaxChannelsSmallInt = ((1 << 22) - 1) / 9;
 
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }

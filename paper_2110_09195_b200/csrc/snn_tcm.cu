@@ -56,7 +56,7 @@ struct CmParams {
   int out_i32, act_vec;
   int N, H, W, C, K, Cw, stride, pad, Ho, Wo;
   int Hq, Wq;             // rows per image / row pitch of the flattened position space
-  FastDiv dWq, dHq;
+  FastDiv dWq, dHq, dCt;  // exact division by Wq, Hq and the number of channel tiles
   int n_planes, halo;
   int Np, Rr;             // positions per tile; staged rows per plane = Np + halo
   int n_mgroups, n_cotiles, total_tiles;
@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
     uint32_t acc_phase = 0;
     auto expand_tile = [&](int it) -> bool {
       const int tile = (int)blockIdx.x + it * (int)gridDim.x;
-      const int mg = tile / p.n_cotiles;
+      const int mg = (int)fdiv((uint32_t)tile, p.dCt);
       const uint32_t Q0 = (uint32_t)mg * (uint32_t)p.Np;
       bool stop = false;
       if (it > 0)  // the first tile's table was made during set-up
@@ -320,7 +320,7 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
                     v[j][k] = make_uint4(0, 0, 0, 0);
                     const int ch = (cb * p.cb_chunks + c0 + k) * 8;
                     if (pix[j] >= 0 && ch < p.C) {
-                      const __half* src = (const __half*)p.act + (size_t)pix[j] * p.C + ch;
+                      const __half* src = (const __half*)p.act + wide_mul((uint32_t)pix[j], (uint32_t)p.C) + ch;
                       if (p.act_vec) {
                         v[j][k] = __ldg(reinterpret_cast<const uint4*>(src));
                       } else {
@@ -349,7 +349,7 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
               for (int j = 0; j < CM_EXP_ROWS; ++j) {
                 bits[j][0] = bits[j][1] = bits[j][2] = bits[j][3] = 0;
                 if (pix[j] >= 0 && w0 < p.Cw) {
-                  const uint32_t* src = (const uint32_t*)p.act + (size_t)pix[j] * p.Cw + w0;
+                  const uint32_t* src = (const uint32_t*)p.act + wide_mul((uint32_t)pix[j], (uint32_t)p.Cw) + w0;
                   if (p.act_vec && nstep == 4) {
                     const uint4 t = __ldg(reinterpret_cast<const uint4*>(src));
                     bits[j][0] = t.x; bits[j][1] = t.y; bits[j][2] = t.z; bits[j][3] = t.w;
@@ -390,7 +390,7 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
     };
     auto drain_tile = [&](int it) -> bool {
       const int tile = (int)blockIdx.x + it * (int)gridDim.x;
-      const int mg = tile / p.n_cotiles, ct = tile - mg * p.n_cotiles;
+      const int mg = (int)fdiv((uint32_t)tile, p.dCt), ct = tile - mg * p.n_cotiles;
       const uint32_t Q0 = (uint32_t)mg * (uint32_t)p.Np;
       const int co4 = ct * 128 + qtr * 32 + cgrp * 4;  // first of the four channels this lane stores
       float al[4] = {0.f, 0.f, 0.f, 0.f};
@@ -442,12 +442,12 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
         if (vec) {
 #pragma unroll
           for (int r = 0; r < 4; ++r)
-            if (pj[r] >= 0 && co4 < p.K) *reinterpret_cast<uint4*>(out32 + (size_t)pj[r] * (size_t)p.K + co4) = w[r];
+            if (pj[r] >= 0 && co4 < p.K) *reinterpret_cast<uint4*>(out32 + wide_mul((uint32_t)pj[r], (uint32_t)p.K) + co4) = w[r];
         } else {
 #pragma unroll
           for (int r = 0; r < 4; ++r) {
             if (pj[r] >= 0) {
-              uint32_t* o = out32 + (size_t)pj[r] * (size_t)p.K + co4;
+              uint32_t* o = out32 + wide_mul((uint32_t)pj[r], (uint32_t)p.K) + co4;
               if (co4 + 0 < p.K) o[0] = w[r].x;
               if (co4 + 1 < p.K) o[1] = w[r].y;
               if (co4 + 2 < p.K) o[2] = w[r].z;
@@ -661,6 +661,7 @@ CmPlan cm_plan(const Geom& g, int act_type, int Np) {
   p.Rr = Np + p.halo;
   const long long mgroups = (p.Qtot + Np - 1) / Np;
   p.n_cotiles = (g.K + 127) / 128;
+  p.dCt = make_fastdiv((uint32_t)p.n_cotiles);
   if (mgroups * p.n_cotiles > 0x7fffffffLL) return pl;
   p.n_mgroups = (int)mgroups;
   p.total_tiles = (int)(mgroups * p.n_cotiles);
