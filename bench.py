@@ -242,9 +242,23 @@ def run_ours(args):
             layers[j].forward(acts[j][m * part:(m + 1) * part], outs[j][m * part:(m + 1) * part], snn.OUT_F32,
                               paths[j], stream)
 
+    n_lanes = max(1, args.streams)
+    lane_streams = [torch.cuda.Stream(dev) for _ in range(n_lanes - 1)]
+
     def launch_layers(idxs, stream):
         """One pass over layers `idxs`: micro-batch 0 on `stream`, the others on streams forked from
         and joined back into it (the pattern stream capture needs)."""
+        if n_lanes > 1 and len(idxs) > 1:
+            # The layers of the benchmark are independent problems (each has its own input), so they
+            # may be issued round-robin on several streams: a layer's start-up then overlaps the
+            # tail of the layer before it.
+            for ls in lane_streams:
+                ls.wait_stream(stream)
+            for k, j in enumerate(idxs):
+                launch_part([j], 0, stream if k % n_lanes == 0 else lane_streams[k % n_lanes - 1])
+            for ls in lane_streams:
+                stream.wait_stream(ls)
+            return
         for ps in part_streams:
             ps.wait_stream(stream)
         launch_part(idxs, 0, stream)
@@ -391,7 +405,7 @@ def run_ours(args):
                    "tau": workload.tau, "l2": "flushed between timed steps (256 MB write)",
                    "launch": ("host calls" if args.no_graph else "CUDA graph of the per-layer C-ABI launches") +
                              (f", {mb} micro-batches of {part} images on {mb} streams" if mb > 1 else ""),
-                   "microbatches": mb,
+                   "microbatches": mb, "streams": n_lanes,
                    "paths": [snn.PATH_NAMES[p] for p in paths]},
         "effective_tops": 2 * workload.dense_macs() * world / (ms_per_step * 1e-3) / 1e12,
         "hbm_floor_ms_per_step": step_floor_hbm_ms,
@@ -438,6 +452,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--microbatch", type=int, default=1,
                     help="cut the batch into this many parts, each running the layers in order on its own stream")
+    ap.add_argument("--streams", type=int, default=1,
+                    help="issue the (independent) layers of a step round-robin on this many streams")
     ap.add_argument("--no-graph", action="store_true", help="launch every layer from the host instead of a CUDA graph")
     ap.add_argument("--layers", default=None, help="a:b restricts the stack to layers [a, b) (profiling aid)")
     args = ap.parse_args()

@@ -76,7 +76,7 @@ cudaError_t microbench(int kind, double* rate);
 // Largest dynamic shared memory a CTA may ask for on sm_100 (227 KB).
 constexpr int kMaxDynSmem = 227 * 1024;
 
-// Raises a kernel's dynamic shared-memory limit to the maximum, once per device.
+// Raises a kernel's dynamic shared-memory limit (and the shared-memory carve-out) to the maximum, once per device.
 template <typename Kernel>
 inline cudaError_t allow_max_smem(Kernel kernel, unsigned long long* done_mask) {
   int dev = 0;
@@ -85,6 +85,9 @@ inline cudaError_t allow_max_smem(Kernel kernel, unsigned long long* done_mask) 
   const unsigned long long bit = 1ull << (dev & 63);
   if (__atomic_load_n(done_mask, __ATOMIC_ACQUIRE) & bit) return cudaSuccess;
   e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  // all of the SM's memory as shared memory, so that two CTAs of half its size fit side by side
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
   if (e == cudaSuccess) __atomic_fetch_or(done_mask, bit, __ATOMIC_RELEASE);
   return e;
 }

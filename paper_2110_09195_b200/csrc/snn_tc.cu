@@ -42,13 +42,16 @@ namespace snn {
 
 namespace {
 
-constexpr int EXP_WARPS = 8, EXP_THREADS = 32 * EXP_WARPS;
-constexpr int TC_THREADS = 320 + EXP_THREADS;  // warp 0 producer, 1 MMA issue, 2-9 epilogue, 10-17 expanders
-constexpr int EPI_WARPS = 8;
+// A CTA has EW epilogue warps and EW expander warps behind the producer and the MMA issuer.
+// EW = 8: one CTA per SM with all of its shared and tensor memory.  EW = 4: a CTA of half the
+// size (at most half of the shared memory, 256 tensor-memory columns, 320 threads), two of which
+// share an SM, so that one's start-up, first loads and last drain run beside the other's MMAs,
+// and the CTAs of the next kernel in the stream set themselves up while this one still runs.
+constexpr int tc_threads(int ew) { return 64 + 64 * ew; }  // warp 0 producer, 1 MMA issue, EW epilogue, EW expanders
 constexpr int EXP_ROWS = 3;                   // rows of a unit one expander thread loads together
 constexpr int NS_MAX = 8;                     // most weight stages in flight
 constexpr int EPI_PITCH = 128;                // bytes per staged output row; 16-byte columns are XOR-swizzled by row
-constexpr int EPI_BYTES = EPI_WARPS * 32 * EPI_PITCH;
+constexpr int epi_bytes(int ew) { return ew * 32 * EPI_PITCH; }
 constexpr size_t kSmemTail = 512;             // barriers, flags, tap offsets
 
 struct TcParams {
@@ -126,8 +129,10 @@ __device__ __forceinline__ void epilogue_slice(const TcParams& p, uint32_t taddr
 
 // ------------------------------------------------------------------ GEMM
 // KPT = MMAs per sub-tile and tap when known at compile time (2 or 4), 0 = read from the parameters
-template <bool F16, int MT, int KPT>
-__global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p) {
+template <bool F16, int MT, int KPT, int EW>
+__global__ void __launch_bounds__(tc_threads(EW), EW == 8 ? 1 : 2) tc_conv_kernel(const TcParams p) {
+  constexpr int EPI_WARPS = EW, EXP_THREADS = 32 * EW;
+  constexpr int NH = EW / 4;  // epilogue warps per TMEM lane quarter; they take the 32-column slices in turn
   extern __shared__ __align__(128) uint8_t smem[];
   // carve-up: [NA activation units][NS weight stages][epilogue tiles][barriers, flags, table]
   uint8_t* a_smem = smem;
@@ -364,7 +369,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
         // The warp's slices (sub-tile mt, columns c0..c0+31) form one sequence.  The TMEM load of
         // slice s+1 is issued as soon as slice s sits in the staging tile, so it flies while
         // slice s is converted and stored, and the store path never waits for a TMEM load.
-        const int per_mt = (p.Nt - 32 * half + 63) / 64;
+        const int per_mt = (p.Nt - 32 * half + 32 * NH - 1) / (32 * NH);
         const int total = MT * per_mt;
         uint32_t v[32];
         int ro[8];
@@ -372,7 +377,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
         int mt = 0, ci = 0;  // slice = (sub-tile mt, this warp's ci-th slice of it); no divisions in the loop
 #pragma unroll 1
         for (int sl = 0; sl < total; ++sl) {
-          const int c0 = 32 * half + 64 * ci;
+          const int c0 = 32 * half + 32 * NH * ci;
           if (ci == 0) {
             // output pixels of the eight rows this lane stores (row = srow + 4*i), -1 when not an output
             const int mine = row_pixel(mt);
@@ -391,7 +396,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
           const int this_mt = mt;
           if (++ci == per_mt) { ci = 0; ++mt; }
           if (sl + 1 < total)
-            tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt + 32 * half + 64 * ci), v);
+            tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt + 32 * half + 32 * NH * ci), v);
           (void)this_mt;
           if (co < p.K) {  // K is a multiple of 4 here, so the four channels exist together
             // loads and conversions first, the (predicated) stores last: no branch sits between
@@ -426,10 +431,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
           const size_t obase = (size_t)(valid ? pix : 0) * (size_t)p.K;
           const uint32_t trow = d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt);
           if ((p.Nt & 31) == 0) {
-            for (int c0 = 32 * half; c0 < p.Nt; c0 += 64)
+            for (int c0 = 32 * half; c0 < p.Nt; c0 += 32 * NH)
               epilogue_slice<F16, 32>(p, trow + (uint32_t)c0, c0, n0, valid, obase);
           } else {
-            for (int c0 = 16 * half; c0 < p.Nt; c0 += 32)
+            for (int c0 = 16 * half; c0 < p.Nt; c0 += 16 * NH)
               epilogue_slice<F16, 16>(p, trow + (uint32_t)c0, c0, n0, valid, obase);
           }
         }
@@ -442,7 +447,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_conv_kernel(const TcParams p
     }
   }
   else {
-    // ------------------------------------------------ expanders (warps 10-17)
+    // ------------------------------------------------ expanders (the last EW warps)
     // Fill activation unit (tile, channel block) of the ring: for every plane, row and 32-channel
     // word, bits -> two 16-byte chunks of +1/-1 bytes (fp16: copy two 8-channel chunks).  A thread
     // takes EXP_ROWS rows at a time and issues their loads together.
@@ -648,17 +653,25 @@ cudaError_t tc_expand_weights(const LayerDev& L, const Geom& g, int act_type, cu
 // ------------------------------------------------------------------ launch plan
 struct TcPlan {
   TcParams p;
+  int ew;
   size_t smem;
   dim3 grid;
   bool ok;
   double score;
 };
 
-constexpr size_t kSmemBudget = 226 * 1024;
+// Shared memory a CTA may plan with: the whole SM's, or half of it for the half-size CTAs
+// (two of them, plus the 1 KB the system keeps per resident CTA, fit the SM's 228 KB).
+static size_t smem_budget(int ew) { return ew == 8 ? (size_t)226 * 1024 : (size_t)112 * 1024; }
 
-// Everything that follows from a choice of sub-tiles per tile (MT) and weight-stage size.
-static TcPlan plan_for(const Geom& g, int act_type, int MT, int stage_kb) {
+// Everything that follows from a choice of sub-tiles per tile (MT), weight-stage size and
+// CTA size (ew = 8: one CTA per SM, ew = 4: two half-size CTAs per SM).
+static TcPlan plan_for(const Geom& g, int act_type, int MT, int stage_kb, int ew) {
+  const size_t kSmemBudget = smem_budget(ew);
+  const int EPI_BYTES = epi_bytes(ew);
+  const int tmem_limit = ew == 8 ? 512 : 256;
   TcPlan pl{};
+  pl.ew = ew;
   TcParams& p = pl.p;
   const bool f16 = act_type == SNN_ACT_F16;
   pl.ok = false;
@@ -688,22 +701,24 @@ static TcPlan plan_for(const Geom& g, int act_type, int MT, int stage_kb) {
   int Nt = p.NtL;
   int forced_nt = env_int("SNN_TC_NT", 0);
   if (forced_nt >= 16 && forced_nt <= 256 && forced_nt % 16 == 0 && p.NtL % forced_nt == 0) Nt = forced_nt;
+  if (ew == 4 && Nt > 128 && p.NtL % 128 == 0) Nt = 128;  // two accumulators in 256 tensor-memory columns
   p.Nt = Nt;
   p.n_ntiles = Kpad / Nt;
   p.dNt = make_fastdiv((uint32_t)p.n_ntiles);
-  if (MT * Nt > 512) return pl;
+  if (MT * Nt > tmem_limit) return pl;
   p.MT = MT;
   p.Rr = 128 * MT + p.halo;
   const long long mgroups = (mtiles + MT - 1) / MT;
   if (mgroups * p.n_ntiles > 0x7fffffffLL || mgroups * p.Rr >= (1ll << 31)) return pl;
   p.n_mgroups = (int)mgroups;
   p.total_tiles = (int)(mgroups * p.n_ntiles);
-  // persistent grid: one CTA per SM, a multiple of the channel tiles so that a CTA keeps its channel tile
-  int grid = sms;
+  // persistent grid: one CTA (two half-size ones) per SM, a multiple of the channel tiles so that a
+  // CTA keeps its channel tile
+  int grid = ew == 8 ? sms : 2 * sms;
   if (grid > p.total_tiles) grid = p.total_tiles;
   if (grid >= p.n_ntiles) grid = grid / p.n_ntiles * p.n_ntiles;
   const int tiles_per_cta = (p.total_tiles + grid - 1) / grid;
-  p.n_acc = (2 * MT * Nt <= 512 && tiles_per_cta > 1) ? 2 : 1;
+  p.n_acc = (2 * MT * Nt <= tmem_limit && tiles_per_cta > 1) ? 2 : 1;
   uint32_t cols = 32;
   while (cols < (uint32_t)(p.n_acc * MT * Nt)) cols *= 2;
   p.tmem_cols = cols;
@@ -761,7 +776,7 @@ static TcPlan plan_for(const Geom& g, int act_type, int MT, int stage_kb) {
   pl.grid = dim3((unsigned)grid);
   // heuristic score: balance of the persistent CTAs x useful share of the staged rows
   const long long rounds = tiles_per_cta;
-  double eff = (double)p.total_tiles / (double)(rounds * grid) * (double)grid / (double)sms;
+  double eff = (double)p.total_tiles / (double)(rounds * grid) * (double)grid / (double)(ew == 8 ? sms : 2 * sms);
   eff *= (double)(128 * MT) / (double)(128 * MT + p.halo);
   if (p.n_acc == 1 && rounds > 1) eff *= 0.8;   // epilogue cannot overlap the next tile's MMAs
   if (p.b_resident) eff *= 1.1;
@@ -770,11 +785,19 @@ static TcPlan plan_for(const Geom& g, int act_type, int MT, int stage_kb) {
   return pl;
 }
 
-// variant: 0 = heuristic; otherwise mt_code (1..3 -> 1,2,4) + 4*stage_code (0..3 -> 48,16,32,64 KB)
-static TcPlan make_plan(const Geom& g, int act_type, int variant) {
+constexpr int kPmVariants = 16;  // position-major variants come first, then the channel-major ones,
+constexpr int kPmHalfVariants = 8;  // then the position-major kernel's half-size CTAs
+
+// variant: 0 = heuristic; 1..15 = mt_code (1..3 -> 1,2,4) + 4*stage_code (0..3 -> 48,16,32,64 KB);
+// half-size CTAs: 0..7 = mt_code' (0,1 -> 1,2) + 2*stage_code' (0..3 -> 8,16,24,32 KB)
+static TcPlan make_plan(const Geom& g, int act_type, int variant, bool half_size = false) {
   TcPlan none{};
   none.ok = false;
   if (g.N < 1) return none;
+  if (half_size) {
+    static const int kbs[4] = {8, 16, 24, 32};
+    return plan_for(g, act_type, 1 + (variant & 1), kbs[(variant >> 1) & 3], 4);
+  }
   int want_mt = 0, want_stage_kb = 0;
   if (variant > 0) {
     static const int mts[4] = {0, 1, 2, 4};
@@ -784,18 +807,16 @@ static TcPlan make_plan(const Geom& g, int act_type, int variant) {
   }
   if (int v = env_int("SNN_TC_MT", 0)) want_mt = v;
   if (int v = env_int("SNN_TC_STAGE_KB", 0)) want_stage_kb = v;
-  if (want_mt == 1 || want_mt == 2 || want_mt == 4) return plan_for(g, act_type, want_mt, want_stage_kb);
+  if (want_mt == 1 || want_mt == 2 || want_mt == 4) return plan_for(g, act_type, want_mt, want_stage_kb, 8);
   TcPlan best = none;
   for (int mt = 1; mt <= 4; mt *= 2) {
-    TcPlan c = plan_for(g, act_type, mt, want_stage_kb);
+    TcPlan c = plan_for(g, act_type, mt, want_stage_kb, 8);
     if (c.ok && (!best.ok || c.score > best.score)) best = c;
   }
   return best;
 }
 
-constexpr int kPmVariants = 16;  // position-major variants come first, the channel-major ones after them
-
-int tc_variant_count() { return kPmVariants + cm_variant_count(); }
+int tc_variant_count() { return kPmVariants + cm_variant_count() + kPmHalfVariants; }
 
 bool tc_supported(const Geom& g, int act_type) {
   if (env_int("SNN_TC_DISABLE", 0)) return false;
@@ -806,6 +827,10 @@ bool tc_supported(const Geom& g, int act_type) {
 
 bool tc_variant_ok(const Geom& g, int act_type, int variant) {
   if (variant < 0 || variant >= tc_variant_count()) return false;
+  if (variant >= kPmVariants + cm_variant_count()) {
+    if (env_int("SNN_TC_NO_HALF", 0)) return false;
+    return make_plan(g, act_type, variant - kPmVariants - cm_variant_count(), true).ok;
+  }
   if (variant >= kPmVariants) return cm_variant_ok(g, act_type, variant - kPmVariants);
   if (variant > 0 && (variant & 3) == 0) return false;  // names no tile size
   return make_plan(g, act_type, variant).ok;
@@ -817,8 +842,10 @@ cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l
     const int forced = env_int("SNN_TC_VARIANT", -1);  // test hook: run one variant regardless of tuning
     if (forced >= 0 && tc_variant_ok(g, act_type, forced)) variant = forced;
   }
-  if (variant >= kPmVariants) return cm_forward(L, g, act_type, l, launched, status_dev, variant - kPmVariants);
-  TcPlan pl = make_plan(g, act_type, variant);
+  const int first_half = kPmVariants + cm_variant_count();
+  if (variant >= kPmVariants && variant < first_half)
+    return cm_forward(L, g, act_type, l, launched, status_dev, variant - kPmVariants);
+  TcPlan pl = variant >= first_half ? make_plan(g, act_type, variant - first_half, true) : make_plan(g, act_type, variant);
   if (!pl.ok) return cudaErrorInvalidConfiguration;
   const bool f16 = act_type == SNN_ACT_F16;
   TcParams& p = pl.p;
@@ -849,28 +876,36 @@ cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l
   cfg.numAttrs = pdl ? 1 : 0;
   cudaError_t e = cudaSuccess;
   cfg.gridDim = pl.grid;
-  cfg.blockDim = dim3(TC_THREADS);
+  cfg.blockDim = dim3((unsigned)tc_threads(pl.ew));
   cfg.dynamicSmemBytes = pl.smem;
-#define SNN_TC_LAUNCH(F, M, KP)                                                                    \
+#define SNN_TC_LAUNCH(F, M, KP, E)                                                                 \
   do {                                                                                             \
     static unsigned long long done = 0;                                                            \
-    e = allow_max_smem(tc_conv_kernel<F, M, KP>, &done);                                           \
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tc_conv_kernel<F, M, KP>, p);               \
+    e = allow_max_smem(tc_conv_kernel<F, M, KP, E>, &done);                                        \
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tc_conv_kernel<F, M, KP, E>, p);            \
   } while (0)
-#define SNN_TC_LAUNCH_K(F, M)                 \
-  do {                                        \
-    if (p.kpt == 4) SNN_TC_LAUNCH(F, M, 4);   \
-    else if (p.kpt == 2) SNN_TC_LAUNCH(F, M, 2); \
-    else SNN_TC_LAUNCH(F, M, 0);              \
+#define SNN_TC_LAUNCH_K(F, M, E)                    \
+  do {                                              \
+    if (p.kpt == 4) SNN_TC_LAUNCH(F, M, 4, E);      \
+    else if (p.kpt == 2) SNN_TC_LAUNCH(F, M, 2, E); \
+    else SNN_TC_LAUNCH(F, M, 0, E);                 \
   } while (0)
-  if (f16) {
-    if (p.MT == 1) SNN_TC_LAUNCH_K(true, 1);
-    else if (p.MT == 2) SNN_TC_LAUNCH_K(true, 2);
-    else SNN_TC_LAUNCH_K(true, 4);
+  if (pl.ew == 4) {
+    if (f16) {
+      if (p.MT == 1) SNN_TC_LAUNCH_K(true, 1, 4);
+      else SNN_TC_LAUNCH_K(true, 2, 4);
+    } else {
+      if (p.MT == 1) SNN_TC_LAUNCH_K(false, 1, 4);
+      else SNN_TC_LAUNCH_K(false, 2, 4);
+    }
+  } else if (f16) {
+    if (p.MT == 1) SNN_TC_LAUNCH_K(true, 1, 8);
+    else if (p.MT == 2) SNN_TC_LAUNCH_K(true, 2, 8);
+    else SNN_TC_LAUNCH_K(true, 4, 8);
   } else {
-    if (p.MT == 1) SNN_TC_LAUNCH_K(false, 1);
-    else if (p.MT == 2) SNN_TC_LAUNCH_K(false, 2);
-    else SNN_TC_LAUNCH_K(false, 4);
+    if (p.MT == 1) SNN_TC_LAUNCH_K(false, 1, 8);
+    else if (p.MT == 2) SNN_TC_LAUNCH_K(false, 2, 8);
+    else SNN_TC_LAUNCH_K(false, 4, 8);
   }
 #undef SNN_TC_LAUNCH_K
 #undef SNN_TC_LAUNCH

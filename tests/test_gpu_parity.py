@@ -258,6 +258,37 @@ def test_channel_major_many_tiles(snn, oracle_mod, monkeypatch):
         check_bin_layer(snn, oracle_mod, shape, 5, n, 93, paths=[snn.PATH_DECODED_TC])
 
 
+HALF_VARIANTS = range(22, 30)  # position-major kernel, two half-size CTAs per SM
+
+
+@pytest.mark.parametrize("c_in,c_out,h,w,stride,n", CM_SHAPES)
+def test_half_size_cta_variants(snn, oracle_mod, monkeypatch, c_in, c_out, h, w, stride, n):
+    """The position-major kernel as CTAs of half an SM's shared and tensor memory (four epilogue and
+    four expander warps), at every tile and weight-stage size the tuner may pick."""
+    shape = wl.LayerShape(c_in, c_out, h, w, stride, 1)
+    for variant in HALF_VARIANTS:
+        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
+        check_bin_layer(snn, oracle_mod, shape, 5, n, 97, paths=[snn.PATH_DECODED_TC])
+
+
+def test_half_size_cta_many_tiles(snn, oracle_mod, monkeypatch):
+    """More tiles than CTAs with two CTAs per SM: both accumulator buffers, ring wrap-around, resident and
+    streamed weights, a channel tile narrower than the weight operand's layout tile."""
+    for variant, shape, n in [(22, wl.LayerShape(128, 128, 28, 28, 1, 1), 40), (25, wl.LayerShape(64, 64, 56, 56, 1, 1), 8),
+                              (24, wl.LayerShape(256, 256, 14, 14, 1, 1), 48), (23, wl.LayerShape(512, 512, 7, 7, 1, 1), 64),
+                              (26, wl.LayerShape(64, 128, 56, 56, 2, 1), 6)]:
+        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
+        check_bin_layer(snn, oracle_mod, shape, 5, n, 99, paths=[snn.PATH_DECODED_TC])
+
+
+def test_half_size_cta_fp16(snn, oracle_mod, monkeypatch):
+    for variant in (22, 23, 26):
+        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
+        for shape, n in [(wl.LayerShape(64, 64, 14, 14, 1, 1), 3), (wl.LayerShape(136, 72, 9, 7, 2, 1), 2)]:
+            ran = check_f16_layer(snn, oracle_mod, shape, 5, n, 95)
+            assert snn.PATH_DECODED_TC in ran
+
+
 def test_channel_major_fp16(snn, oracle_mod, monkeypatch):
     for variant in (16, 17, 18):
         monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
