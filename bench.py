@@ -280,12 +280,33 @@ def run_ours(args):
 
     all_idx = list(range(len(layers)))
     use_graph = not args.no_graph
-    step_graph = capture(all_idx) if use_graph else None
+    group = None
+    if args.group:
+        # The layers of the benchmark are independent problems (each has its own input): the step
+        # is one persistent launch that walks through all of them (snn_conv_group_forward).
+        if mb != 1 or n_lanes != 1 or forced not in (snn.PATH_AUTO, snn.PATH_DECODED_TC):
+            raise SystemExit("--group runs the tensor-core path on one stream without micro-batches")
+        group = snn.SnnConvGroup(layers, [(nb, s.h, s.w) for s in workload.layers])
+
+        def launch_group(stream):
+            group.forward(acts, outs, snn.OUT_F32, stream)
+
+        if use_graph:
+            step_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                launch_group(side)
+                side.synchronize()
+                with torch.cuda.graph(step_graph, stream=side):
+                    launch_group(torch.cuda.current_stream(dev))
+    else:
+        step_graph = capture(all_idx) if use_graph else None
     stream = torch.cuda.current_stream(dev)
 
     def step():
         if use_graph:
             step_graph.replay()
+        elif group is not None:
+            launch_group(stream)
         else:
             launch_layers(all_idx, stream)
 
@@ -312,7 +333,8 @@ def run_ours(args):
         e1.record(stream)
     barrier()
     wall = time.perf_counter() - wall0
-    launches = (snn.kernel_launches() - launches0) if not use_graph else len(layers) * mb * args.steps
+    launches = (snn.kernel_launches() - launches0) if not use_graph else \
+        (1 if group is not None else len(layers) * mb) * args.steps
     step_ms = [e0.elapsed_time(e1) for e0, e1 in ev]
     total_ms = float(sum(step_ms))
 
@@ -405,7 +427,7 @@ def run_ours(args):
                    "tau": workload.tau, "l2": "flushed between timed steps (256 MB write)",
                    "launch": ("host calls" if args.no_graph else "CUDA graph of the per-layer C-ABI launches") +
                              (f", {mb} micro-batches of {part} images on {mb} streams" if mb > 1 else ""),
-                   "microbatches": mb, "streams": n_lanes,
+                   "microbatches": mb, "streams": n_lanes, "grouped": group is not None,
                    "paths": [snn.PATH_NAMES[p] for p in paths]},
         "effective_tops": 2 * workload.dense_macs() * world / (ms_per_step * 1e-3) / 1e12,
         "hbm_floor_ms_per_step": step_floor_hbm_ms,
@@ -454,6 +476,8 @@ def main():
                     help="cut the batch into this many parts, each running the layers in order on its own stream")
     ap.add_argument("--streams", type=int, default=1,
                     help="issue the (independent) layers of a step round-robin on this many streams")
+    ap.add_argument("--group", action="store_true",
+                    help="run the step as one grouped launch of all layers (independent problems)")
     ap.add_argument("--no-graph", action="store_true", help="launch every layer from the host instead of a CUDA graph")
     ap.add_argument("--layers", default=None, help="a:b restricts the stack to layers [a, b) (profiling aid)")
     args = ap.parse_args()

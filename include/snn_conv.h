@@ -139,6 +139,39 @@ SNN_API int64_t snn_kernel_launches(void);
 SNN_API snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate);
 
 /*
+ * A group of independent layer problems run as ONE persistent tensor-core launch.
+ * The paper times whole networks (Sec. 5.3, Table 4: all binary layers of
+ * ResNet-18/34 in one run); each member of a group is still the forward step of
+ * Sec. 3 / Algorithm 1 for one layer, on that layer's own input, and the members
+ * must not depend on each other (no member's output is another member's input
+ * within one call): the CTAs walk through all members without any grid-wide step
+ * in between, so that one member's start-up, first loads and last drain run beside
+ * its neighbours' MMAs.
+ *
+ * snn_conv_group_create: `layers` are `count` (1..SNN_GROUP_MAX) handles of one
+ * activation type on one device; N[i], H[i], W[i] fix the input shape of member i.
+ * The group keeps the handles' device data by reference: the handles must outlive
+ * the group.  It builds its own tiled weight operands (device memory owned by the
+ * group).  Errors: INVALID_ARG (null, count out of range, mixed activation types
+ * or devices, a shape giving no output), UNSUPPORTED (a member the tensor-core
+ * path cannot run; nothing is kept), CUDA, OOM.
+ *
+ * snn_conv_group_forward: act_dev[i] / out_dev[i] are HOST arrays of `count`
+ * DEVICE pointers with the layouts and alignment of snn_conv_forward; outputs of
+ * different members must not overlap.  Asynchronous on cuda_stream; allocates
+ * nothing.  Errors: INVALID_ARG, TIMEOUT (an earlier launch of the group gave up
+ * a bounded wait), CUDA.
+ */
+#define SNN_GROUP_MAX 32
+typedef struct snn_conv_group snn_conv_group_t; /* opaque; owned by the library */
+SNN_API snn_status_t snn_conv_group_create(snn_conv_t* const* layers, int32_t count, const int32_t* N,
+                                           const int32_t* H, const int32_t* W, snn_conv_group_t** out);
+SNN_API snn_status_t snn_conv_group_forward(snn_conv_group_t* g, const void* const* act_dev, void* const* out_dev,
+                                            int32_t out_type, void* cuda_stream);
+/* Frees the group and its device buffers (not the member handles).  NULL is a no-op. */
+SNN_API snn_status_t snn_conv_group_destroy(snn_conv_group_t* g);
+
+/*
  * Forward pass for callers that must not allocate device memory.  (The paper has
  * no counterpart to this entry point; it exists for how the library is embedded.)
  *

@@ -26,6 +26,7 @@ EXPORTED_SYMBOLS = (
     "snn_conv_create", "snn_conv_forward", "snn_conv_forward_host", "snn_conv_tune", "snn_conv_chosen_path",
     "snn_conv_path_supported", "snn_conv_destroy", "snn_last_error", "snn_version", "snn_kernel_launches",
     "snn_microbench", "snn_conv_forward_static",
+    "snn_conv_group_create", "snn_conv_group_forward", "snn_conv_group_destroy",
 )
 
 
@@ -82,6 +83,13 @@ def load_library():
     lib.snn_kernel_launches.argtypes = []
     lib.snn_conv_forward_static.restype = i32
     lib.snn_conv_forward_static.argtypes = [ctypes.POINTER(_Desc), vp, i32, i32, i32, vp, i32, vp]
+    lib.snn_conv_group_create.restype = i32
+    lib.snn_conv_group_create.argtypes = [ctypes.POINTER(vp), i32, ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                          ctypes.POINTER(i32), ctypes.POINTER(vp)]
+    lib.snn_conv_group_forward.restype = i32
+    lib.snn_conv_group_forward.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), i32, vp]
+    lib.snn_conv_group_destroy.restype = i32
+    lib.snn_conv_group_destroy.argtypes = [vp]
     lib.snn_microbench.restype = i32
     lib.snn_microbench.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double)]
     _lib = lib
@@ -244,6 +252,74 @@ class SnnConv:
         if getattr(self, "_h", None) is not None:
             load_library().snn_conv_destroy(self._h)
             self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+class SnnConvGroup:
+    """Several independent layer problems run as one persistent launch (wraps snn_conv_group_t).
+
+    `layers` are SnnConv objects of one activation type on one device, `shapes` their input
+    shapes (N, H, W).  The members must not depend on each other within one call, and the
+    SnnConv objects must outlive the group."""
+
+    def __init__(self, layers, shapes):
+        lib = load_library()
+        n = len(layers)
+        if n != len(shapes) or n < 1:
+            raise SnnError(1, "a group needs one (N, H, W) per layer")
+        self.layers = list(layers)
+        self.shapes = [tuple(int(v) for v in s) for s in shapes]
+        hs = (ctypes.c_void_p * n)(*[l._h for l in self.layers])
+        i32 = ctypes.c_int32
+        ns = (i32 * n)(*[s[0] for s in self.shapes])
+        hh = (i32 * n)(*[s[1] for s in self.shapes])
+        ww = (i32 * n)(*[s[2] for s in self.shapes])
+        g = ctypes.c_void_p()
+        self._g = None
+        _check(lib.snn_conv_group_create(hs, n, ns, hh, ww, ctypes.byref(g)))
+        self._g = g
+        self.device = self.layers[0].device
+
+    def alloc_outs(self, out_type=OUT_F32):
+        return [l.alloc_out(n, h, w, out_type) for l, (n, h, w) in zip(self.layers, self.shapes)]
+
+    def forward(self, acts, outs=None, out_type=OUT_F32, stream=None):
+        """snn_conv_group_forward: acts / outs are lists of CUDA tensors, one per member;
+        asynchronous on `stream` (default: torch's current stream)."""
+        import torch
+        n = len(self.layers)
+        if len(acts) != n:
+            raise SnnError(1, "one activation tensor per member")
+        if outs is None:
+            outs = self.alloc_outs(out_type)
+        want = torch.float32 if out_type == OUT_F32 else torch.int32
+        for l, (nb, h, w), a, o in zip(self.layers, self.shapes, acts, outs):
+            if not a.is_cuda or a.device.index != self.device:
+                raise SnnError(1, f"activations must live on cuda:{self.device}")
+            l._check_act(a)
+            ho, wo = l.out_hw(h, w)
+            if tuple(a.shape[:3]) != (nb, h, w):
+                raise SnnError(1, "activation tensor does not have the shape the group was created for")
+            if (not o.is_cuda or o.device.index != self.device or o.dtype != want or not o.is_contiguous()
+                    or tuple(o.shape) != (nb, ho, wo, l.c_out)):
+                raise SnnError(1, "output tensor has the wrong device, dtype, shape or layout")
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        ap = (ctypes.c_void_p * n)(*[a.data_ptr() for a in acts])
+        op = (ctypes.c_void_p * n)(*[o.data_ptr() for o in outs])
+        _check(load_library().snn_conv_group_forward(self._g, ap, op, int(out_type),
+                                                     ctypes.c_void_p(stream.cuda_stream)))
+        return outs
+
+    def destroy(self):
+        if getattr(self, "_g", None) is not None:
+            load_library().snn_conv_group_destroy(self._g)
+            self._g = None
 
     def __del__(self):
         try:

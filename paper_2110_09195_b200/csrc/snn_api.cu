@@ -437,6 +437,94 @@ snn_status_t snn_conv_tune(snn_conv_t* h, int32_t N, int32_t H, int32_t W, int32
   return SNN_OK;
 }
 
+struct snn_conv_group {
+  int device = 0, count = 0, act_type = 0;
+  GroupDev* G = nullptr;
+  int* status_host = nullptr;  // pinned, written by the kernel on a bounded-wait timeout
+  int* status_dev = nullptr;
+};
+
+snn_status_t snn_conv_group_create(snn_conv_t* const* layers, int32_t count, const int32_t* N, const int32_t* H,
+                                   const int32_t* W, snn_conv_group_t** out) {
+  if (!out) return fail(SNN_ERR_INVALID_ARG, "null output pointer");
+  *out = nullptr;
+  if (!layers || !N || !H || !W) return fail(SNN_ERR_INVALID_ARG, "null argument");
+  if (count < 1 || count > SNN_GROUP_MAX)
+    return fail(SNN_ERR_INVALID_ARG, "a group has 1..%d members, not %d", SNN_GROUP_MAX, count);
+  const LayerDev* Ls[SNN_GROUP_MAX];
+  Geom gs[SNN_GROUP_MAX];
+  for (int i = 0; i < count; ++i) {
+    if (!layers[i]) return fail(SNN_ERR_INVALID_ARG, "member %d is a null handle", i);
+    if (layers[i]->act_type != layers[0]->act_type || layers[i]->device != layers[0]->device)
+      return fail(SNN_ERR_INVALID_ARG, "member %d differs from member 0 in activation type or device", i);
+    if (N[i] < 1 || !make_geom(layers[i], N[i], H[i], W[i], &gs[i]))
+      return fail(SNN_ERR_INVALID_ARG, "member %d: shape N=%d H=%d W=%d gives no output", i, N[i], H[i], W[i]);
+    Ls[i] = &layers[i]->L;
+  }
+  DeviceGuard guard(layers[0]->device);
+  if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", layers[0]->device);
+  snn_conv_group* g = new (std::nothrow) snn_conv_group();
+  if (!g) return fail(SNN_ERR_OOM, "host allocation failed");
+  g->device = layers[0]->device;
+  g->count = count;
+  g->act_type = layers[0]->act_type;
+  cudaError_t e = cudaHostAlloc((void**)&g->status_host, sizeof(int), cudaHostAllocMapped);
+  if (e == cudaSuccess) {
+    *g->status_host = 0;
+    e = cudaHostGetDevicePointer((void**)&g->status_dev, g->status_host, 0);
+  }
+  int launched = 0;
+  if (e == cudaSuccess) e = tcg_create(Ls, gs, count, g->act_type, layers[0]->host_stream, &g->G, &launched);
+  g_launches += launched;
+  if (e != cudaSuccess) {
+    if (g->status_host) cudaFreeHost(g->status_host);
+    delete g;
+    if (e == cudaErrorInvalidConfiguration) {
+      cudaGetLastError();
+      return fail(SNN_ERR_UNSUPPORTED, "the grouped tensor-core kernel cannot run one of these layers at this shape");
+    }
+    return cuda_fail(e, "snn_conv_group_create");
+  }
+  *out = g;
+  return SNN_OK;
+}
+
+snn_status_t snn_conv_group_forward(snn_conv_group_t* g, const void* const* act_dev, void* const* out_dev,
+                                    int32_t out_type, void* cuda_stream) {
+  if (!g || !g->G) return fail(SNN_ERR_INVALID_ARG, "null group");
+  if (!act_dev || !out_dev) return fail(SNN_ERR_INVALID_ARG, "null pointer array");
+  if (out_type != SNN_OUT_F32 && out_type != SNN_OUT_I32) return fail(SNN_ERR_INVALID_ARG, "unknown output type %d", out_type);
+  if (out_type == SNN_OUT_I32 && g->act_type != SNN_ACT_BIN)
+    return fail(SNN_ERR_INVALID_ARG, "int32 output needs binary activations");
+  for (int i = 0; i < g->count; ++i) {
+    if (!act_dev[i] || !out_dev[i]) return fail(SNN_ERR_INVALID_ARG, "member %d: null device pointer", i);
+    if (((uintptr_t)act_dev[i] & 15) || ((uintptr_t)out_dev[i] & 15))
+      return fail(SNN_ERR_INVALID_ARG, "member %d: misaligned device pointer", i);
+  }
+  DeviceGuard guard(g->device);
+  if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", g->device);
+  if (*g->status_host) {
+    const int code = *g->status_host;
+    *g->status_host = 0;
+    return fail(SNN_ERR_TIMEOUT, "an earlier launch of the group gave up a bounded wait (code %d)", code);
+  }
+  int launched = 0;
+  cudaError_t e = tcg_forward(g->G, act_dev, out_dev, out_type == SNN_OUT_I32, (cudaStream_t)cuda_stream, g->status_dev,
+                              &launched);
+  g_launches += launched;
+  if (e != cudaSuccess) return cuda_fail(e, "snn_conv_group_forward");
+  return SNN_OK;
+}
+
+snn_status_t snn_conv_group_destroy(snn_conv_group_t* g) {
+  if (!g) return SNN_OK;
+  DeviceGuard guard(g->device);
+  tcg_destroy(g->G);
+  if (g->status_host) cudaFreeHost(g->status_host);
+  delete g;
+  return SNN_OK;
+}
+
 snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate) {
   if (!rate) return fail(SNN_ERR_INVALID_ARG, "null rate pointer");
   if (kind < 0 || kind > 4) return fail(SNN_ERR_INVALID_ARG, "unknown microbenchmark %d", kind);

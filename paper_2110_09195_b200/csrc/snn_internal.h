@@ -71,6 +71,20 @@ cudaError_t cm_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l
 size_t cm_weight_bytes(const Geom& g, int act_type);
 cudaError_t cm_expand_weights(const LayerDev& L, const Geom& g, int act_type, cudaStream_t s, int* launched);
 
+// Tensor-core weight operand of the position-major layout with a caller-chosen channel block and
+// layout tile, written to `dst` (9 * n_chunks * Kpad * 16 bytes); used by the grouped kernel.
+cudaError_t tc_expand_weights_custom(const uint32_t* wplanes, void* dst, int C, int K, int Cw, int Kpad, int n_chunks,
+                                     int cb_chunks, int NtL, bool f16, cudaStream_t s);
+
+// Several independent problems in one persistent tensor-core launch (snn_tcg.cu).
+struct GroupDev;
+cudaError_t tcg_create(const LayerDev* const* layers, const Geom* geoms, int count, int act_type, cudaStream_t s,
+                       GroupDev** out, int* launched);
+cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, int out_i32, cudaStream_t s,
+                        int* status_dev, int* launched);
+void tcg_destroy(GroupDev* G);
+int tcg_count(const GroupDev* G);
+
 cudaError_t microbench(int kind, double* rate);
 
 // Largest dynamic shared memory a CTA may ask for on sm_100 (227 KB).

@@ -650,6 +650,19 @@ cudaError_t tc_expand_weights(const LayerDev& L, const Geom& g, int act_type, cu
   return cudaGetLastError();
 }
 
+cudaError_t tc_expand_weights_custom(const uint32_t* wplanes, void* dst, int C, int K, int Cw, int Kpad, int n_chunks,
+                                     int cb_chunks, int NtL, bool f16, cudaStream_t s) {
+  const long long total = (long long)9 * n_chunks * Kpad;
+  const unsigned blocks = (unsigned)((total + 255) / 256);
+  if (f16)
+    tc_expand_weights_kernel<true><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks,
+                                                         n_chunks / cb_chunks, NtL);
+  else
+    tc_expand_weights_kernel<false><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks,
+                                                          n_chunks / cb_chunks, NtL);
+  return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ launch plan
 struct TcPlan {
   TcParams p;

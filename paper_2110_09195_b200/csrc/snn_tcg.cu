@@ -1,0 +1,789 @@
+// Several independent sub-bit convolutions in ONE persistent tensor-core launch.
+//
+// Each problem of a group is the forward pass of Sec. 3 / Algorithm 1 for one layer
+// on its own input (decoded +/-1 weights as int8 or fp16 operands, implicit GEMM
+// over a padded, flattened position space, exactly as in the position-major kernel
+// of snn_tc.cu).  The problems do not depend on each other, so one CTA per SM walks
+// through all of them without any grid-wide step in between: while the MMAs of one
+// problem's last tile run, the expander warps already stage the next problem's first
+// activations, the weight producer streams its first stages, and the epilogue warps
+// still drain the tile before.  Start-up, first loads and last drain, which cost a
+// single-layer launch about as much as its MMAs at batch 64, are paid once per group.
+//
+// What makes this possible is a ring geometry that is the same for every problem:
+//   activation units  NA slots of a_slot_bytes   (a problem's unit uses a prefix)
+//   weight stages     NS slots of b_slot_bytes   (a stage = a run of K steps of one
+//                                                 channel block, taps outermost)
+//   accumulators      two buffers of 256 tensor-memory columns
+// so slots, barriers and phases simply carry on from one problem to the next.
+// Tiles of problem l are dealt to the CTAs round-robin starting where problem l-1
+// stopped, which keeps the CTAs' total work within one tile of each other.
+//
+//      warp 0        one thread streams weight stages (cp.async.bulk onto mbarriers)
+//      warp 1        one thread issues tcgen05.mma and commits barriers
+//      warps 2-9     epilogue: TMEM -> registers -> shared-memory transposition ->
+//                    alpha -> 128-byte row stores
+//      warps 10-17   expanders: packed bits -> +1/-1 bytes (or fp16 copied) into the
+//                    activation ring
+// Every wait is bounded; one that runs out raises a status word the host reads, and
+// the CTA still frees its tensor memory and returns.
+#include "snn_tc_common.cuh"
+
+namespace snn {
+
+namespace {
+
+constexpr int G_EW = 8;                       // epilogue warps = expander warps
+constexpr int G_THREADS = 64 + 64 * G_EW;
+constexpr int G_EXP_THREADS = 32 * G_EW;
+constexpr int G_EXP_ROWS = 3;                 // rows of a unit one expander thread loads together
+constexpr int G_EPI_PITCH = 128;
+constexpr int G_EPI_BYTES = G_EW * 32 * G_EPI_PITCH;
+constexpr int G_NA_MAX = 4, G_NS_MAX = 8;
+constexpr uint32_t G_ACC_COLS = 256;          // tensor-memory columns of one accumulator buffer
+constexpr size_t kGTail = 512;
+constexpr size_t kGSmemBudget = 226 * 1024;
+constexpr uint32_t kGASlotMax = 40 * 1024 + 512;   // largest activation unit a problem may stage
+constexpr uint32_t kGBSlot = 16 * 1024;            // bytes of a weight-stage slot
+
+// One problem of a group, as the kernel reads it from global memory.
+struct GLayer {
+  const uint8_t* wt;      // [layout tile][channel block][tap][chunk][NtL][16 B], owned by the group
+  const float* alpha;
+  int N, H, W, C, K, Cw, stride, pad, Ho, Wo;
+  int NtL, Nt;            // channels per layout tile of the weight operand / per tile
+  int Hq, Wq;             // rows per image / row pitch of the flattened position space
+  FastDiv dWq, dHq, dNt;
+  int n_planes, halo, Rr; // 1 or 4 planes; largest tap shift; staged rows per plane = 128*MT + halo
+  int MT;                 // M sub-tiles of 128 positions per tile
+  int cb_chunks, n_cb, kpt;
+  int st_ksteps;          // K steps (MMAs per sub-tile) per weight stage; divides 9*kpt
+  uint32_t stage_bytes;   // = st_ksteps * 2 * Nt * 16
+  int n_ntiles, total_tiles;
+  int tile_off;           // CTA that takes this problem's tile 0
+  long long Qtot;
+};
+
+struct GParams {
+  const GLayer* layers;
+  int n_layers;
+  const void* act[SNN_GROUP_MAX];
+  void* out[SNN_GROUP_MAX];
+  int* status;
+  int out_i32;
+  int NA, NS;
+  uint32_t a_slot_bytes, b_slot_bytes;
+  uint32_t off_b, off_epi, off_pix, off_lay, off_tail;
+};
+
+__device__ __forceinline__ int g_position_to_pixel(const GLayer& L, uint32_t q, int pa, int pb) {
+  if ((long long)q >= L.Qtot) return -1;
+  const uint32_t rg = fdiv(q, L.dWq);
+  const int j = (int)(q - rg * (uint32_t)L.Wq);
+  const uint32_t n = fdiv(rg, L.dHq);
+  const int i = (int)(rg - n * (uint32_t)L.Hq);
+  if ((int)n >= L.N) return -1;
+  const int r = L.stride * i + pa - L.pad, c = L.stride * j + pb - L.pad;
+  if (r < 0 || r >= L.H || c < 0 || c >= L.W) return -1;
+  return ((int)n * L.H + r) * L.W + c;
+}
+
+// first tile of problem L for this CTA (tiles then follow at a stride of the grid)
+__device__ __forceinline__ int g_first_tile(const GLayer& L) {
+  int f = (int)blockIdx.x - L.tile_off;
+  if (f < 0) f += (int)gridDim.x;
+  return f;
+}
+
+// The MMAs of one channel block of one tile: 9 taps x KPT K steps x MT sub-tiles.  The body of
+// a tap is straight-line code; the taps are a loop, because the issuing thread runs alone on
+// its warp and nine unrolled taps no longer fit the instruction cache closest to it.
+// Weight stages are waited for and released as the K-step counter crosses their boundaries.
+template <bool F16, int MT, int KPT>
+__device__ __forceinline__ bool g_issue_block(uint64_t a_unit, const uint32_t* tapu, uint32_t a_step,
+                                              uint64_t b_desc0, uint32_t b_slot_units, uint32_t b_step, uint32_t d0,
+                                              uint32_t nt, uint32_t idesc, uint32_t& acc, int st_ksteps, int NS,
+                                              uint32_t bar_bfull, uint32_t bar_bempty, int& b_slot, uint32_t& b_phase) {
+  int in_stage = 0;
+  uint64_t bd = 0;
+#pragma unroll 1
+  for (int t = 0; t < 9; ++t) {
+    const uint64_t ad_t = a_unit + (uint64_t)tapu[t];
+#pragma unroll
+    for (int k = 0; k < KPT; ++k) {
+      if (in_stage == 0) {
+        if (!mbar_wait(bar_bfull + 8 * b_slot, b_phase)) return false;
+        tc_fence_after();
+        bd = b_desc0 + (uint64_t)((uint32_t)b_slot * b_slot_units);
+      }
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt)
+        mma_ss<F16>(d0 + (uint32_t)mt * nt, ad_t + (uint64_t)((uint32_t)k * a_step + (uint32_t)(mt * 128)), bd, idesc,
+                    acc);
+      acc = 1;
+      bd += b_step;
+      if (++in_stage == st_ksteps) {
+        in_stage = 0;
+        tc_commit(bar_bempty + 8 * b_slot);  // the slot is free once these MMAs have read it
+        if (++b_slot == NS) { b_slot = 0; b_phase ^= 1u; }
+      }
+    }
+  }
+  return true;
+}
+
+}  // namespace
+
+template <bool F16>
+__global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  // carve-up: [NA activation slots][NS weight slots][epilogue tiles][pixel table][problem table][barriers, flags]
+  uint8_t* a_smem = smem;
+  uint8_t* b_smem = smem + p.off_b;
+  uint8_t* epi_smem = smem + p.off_epi;
+  int* pix_tab = reinterpret_cast<int*>(smem + p.off_pix);
+  // The problems' descriptions are read from shared memory where they are needed instead of
+  // being held in registers: the roles are at different problems at the same time, and the
+  // epilogue's registers are all taken by the slices it transposes.
+  const GLayer* lay = reinterpret_cast<const GLayer*>(smem + p.off_lay);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_tail);
+  // barriers: b_full[8] b_empty[8] a_full[4] a_empty[4] acc_full[2] acc_empty[2]
+  const uint32_t bar_bfull = smem_u32(bars), bar_bempty = smem_u32(bars + 8);
+  const uint32_t bar_afull = smem_u32(bars + 16), bar_aempty = smem_u32(bars + 20);
+  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 28);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint32_t* tapu = tmem_slot + 3;  // [9] row offset of every tap inside a unit, kept by the MMA issuer (tmem_slot[2]: expander flag)
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int NS = p.NS, NA = p.NA;
+  const int G = (int)gridDim.x;
+
+  if (tid < 28) {
+    uint32_t count = 1;
+    if (tid >= 26) count = G_EW;                       // acc_empty: one arrival per epilogue warp
+    if (tid >= 16 && tid < 20) count = G_EXP_THREADS;  // a_full: every expander thread arrives
+    mbar_init(smem_u32(bars + tid), count);
+  }
+  if (tid == 32) *abort_flag = 0;
+  {
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(p.layers);
+    uint32_t* dst = reinterpret_cast<uint32_t*>(smem + p.off_lay);
+    const int words = p.n_layers * (int)(sizeof(GLayer) / 4);
+    for (int i = tid; i < words; i += G_THREADS) dst[i] = __ldg(src + i);
+  }
+  if (warp == 2) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  grid_dep_launch();
+
+  if (warp == 0) {
+    // ------------------------------------------------ weight producer (one lane)
+    if (lane == 0) {
+      int b_slot = 0;
+      long long b_issued = 0;
+      uint32_t b_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
+      bool ok = true;
+      for (int l = 0; l < p.n_layers && ok; ++l) {
+        const GLayer& L = lay[l];
+        const int Nt = L.Nt, NtL = L.NtL, n_cb = L.n_cb, n_ntiles = L.n_ntiles, total = L.total_tiles;
+        const int stages_per_cb = 9 * L.kpt / L.st_ksteps;
+        const int chunks_per_stage = 2 * L.st_ksteps;
+        const uint32_t stage_bytes = L.stage_bytes;
+        const uint8_t* wt = L.wt;
+        const size_t cb_bytes = (size_t)9 * L.cb_chunks * NtL * 16;   // one channel block of one layout tile
+        const FastDiv dNt = L.dNt;
+        for (int tile = g_first_tile(L); tile < total && ok; tile += G) {
+          if (*abort_flag) { ok = false; break; }
+          const int nti = tile - (int)fdiv((uint32_t)tile, dNt) * n_ntiles;
+          const int n0 = nti * Nt;
+          const int ltile = Nt == NtL ? nti : n0 / NtL;
+          const int n_in = n0 - ltile * NtL;
+          const uint8_t* src_tile = wt + (size_t)ltile * n_cb * cb_bytes + (size_t)n_in * 16;
+          for (int cb = 0; cb < n_cb && ok; ++cb) {
+            const uint8_t* src = src_tile + (size_t)cb * cb_bytes;
+            for (int sg = 0; sg < stages_per_cb; ++sg) {
+              if (b_issued >= NS && !mbar_wait_backoff(bar_bempty + 8 * b_slot, b_phase, 32)) { ok = false; break; }
+              const uint32_t dst = smem_u32(b_smem) + (uint32_t)b_slot * p.b_slot_bytes;
+              mbar_expect_tx(bar_bfull + 8 * b_slot, stage_bytes);
+              if (Nt == NtL) {
+                bulk_g2s(dst, src, stage_bytes, bar_bfull + 8 * b_slot);  // the stage's chunks are contiguous
+              } else {
+                for (int c = 0; c < chunks_per_stage; ++c)
+                  bulk_g2s(dst + (uint32_t)c * Nt * 16, src + (size_t)c * NtL * 16, (uint32_t)Nt * 16,
+                           bar_bfull + 8 * b_slot);
+              }
+              src += (size_t)chunks_per_stage * NtL * 16;
+              ++b_issued;
+              if (++b_slot == NS) { b_slot = 0; b_phase ^= 1u; }
+            }
+          }
+        }
+      }
+      if (!ok && !*abort_flag) {
+        *abort_flag = 1;
+        raise_status(p.status, 2);
+      }
+      // never leave with copies in flight: wait (bounded) for the last load of every slot
+      for (int s = 0; s < NS; ++s) {
+        long long last = -1;
+        if (b_issued > s) last = s + (b_issued - 1 - s) / NS * NS;
+        if (last >= 0) mbar_wait_backoff(bar_bfull + 8 * s, (uint32_t)((last / NS) & 1), 64);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer (one lane)
+    if (lane == 0) {
+      bool ok = true;
+      int a_slot = 0, b_slot = 0, acc_slot = 0;
+      uint32_t a_phase = 0, b_phase = 0, acc_phase = 1;
+      long long tiles_done = 0;
+      const uint32_t a_slot_units = p.a_slot_bytes >> 4, b_slot_units = p.b_slot_bytes >> 4;
+      for (int l = 0; l < p.n_layers && ok; ++l) {
+        const GLayer& L = lay[l];
+        const int Nt = L.Nt, Rr = L.Rr, n_cb = L.n_cb, MT = L.MT, kpt = L.kpt, total = L.total_tiles;
+        const int st_ksteps = L.st_ksteps;
+        // instruction descriptor: D format, A/B formats, K-major both, N>>3, M>>4
+        const uint32_t idesc = F16 ? ((1u << 4) | ((uint32_t)(Nt >> 3) << 17) | ((128u >> 4) << 24))
+                                   : ((2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(Nt >> 3) << 17) |
+                                      ((128u >> 4) << 24));
+        const uint64_t a_desc0 = make_desc(smem_u32(a_smem), (uint32_t)Rr * 16, 128);
+        const uint64_t b_desc0 = make_desc(smem_u32(b_smem), (uint32_t)Nt * 16, 128);
+        const uint32_t a_step = 2u * (uint32_t)Rr, b_step = 2u * (uint32_t)Nt;  // two chunks per MMA
+        // rows (16-byte units) from a unit's origin to tap t: plane offset + shift inside the plane
+#pragma unroll
+        for (int t = 0; t < 9; ++t) {
+          const int ky = t / 3, kx = t % 3;
+          tapu[t] = L.stride == 1 ? (uint32_t)(ky * L.Wq + kx)
+                                  : (uint32_t)((ky & 1) * 2 + (kx & 1)) * (uint32_t)(L.cb_chunks * Rr) +
+                                        (uint32_t)((ky >> 1) * L.Wq + (kx >> 1));
+        }
+        for (int tile = g_first_tile(L); tile < total && ok; tile += G, ++tiles_done) {
+          if (tiles_done >= 2) {
+            if (!mbar_wait(bar_accempty + 8 * acc_slot, acc_phase)) { ok = false; break; }
+            tc_fence_after();
+          }
+          const uint32_t d0 = tmem_base + (uint32_t)acc_slot * G_ACC_COLS;
+          uint32_t acc = 0;  // 0 only for the first MMA of every sub-tile
+          for (int cb = 0; cb < n_cb && ok; ++cb) {
+            if (!mbar_wait(bar_afull + 8 * a_slot, a_phase)) { ok = false; break; }
+            tc_fence_after();
+            const uint64_t a_unit = a_desc0 + (uint64_t)((uint32_t)a_slot * a_slot_units);
+#define G_ISSUE(M, KP)                                                                                       \
+  ok = g_issue_block<F16, M, KP>(a_unit, tapu, a_step, b_desc0, b_slot_units, b_step, d0, (uint32_t)Nt, idesc, acc, \
+                                 st_ksteps, NS, bar_bfull, bar_bempty, b_slot, b_phase)
+#define G_ISSUE_K(M)                   \
+  do {                                 \
+    if (kpt == 4) G_ISSUE(M, 4);       \
+    else if (kpt == 2) G_ISSUE(M, 2);  \
+    else if (kpt == 3) G_ISSUE(M, 3);  \
+    else G_ISSUE(M, 1);                \
+  } while (0)
+            if (MT == 4) G_ISSUE_K(4);
+            else if (MT == 2) G_ISSUE_K(2);
+            else G_ISSUE_K(1);
+#undef G_ISSUE_K
+#undef G_ISSUE
+            if (!ok) break;
+            tc_commit(bar_aempty + 8 * a_slot);  // the activation unit may be overwritten
+            if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
+          }
+          if (!ok) break;
+          tc_commit(bar_accfull + 8 * acc_slot);  // fires when this tile's MMAs are complete
+          if (++acc_slot == 2) { acc_slot = 0; acc_phase ^= 1u; }
+        }
+      }
+      if (!ok && !*abort_flag) {
+        *abort_flag = 1;
+        raise_status(p.status, 3);
+      }
+    }
+    __syncwarp();
+  } else if (warp < 2 + G_EW) {
+    // ------------------------------------------------ epilogue warps
+    grid_dep_wait();  // an earlier kernel in the stream may still read the output buffers
+    // Warp w reads TMEM lanes 32*(w%4).. (rows of the tile); the two warps of a lane quarter take
+    // the 32-column slices in turn.  A slice goes through a per-warp shared-memory tile so that
+    // each store instruction writes whole 128-byte rows.
+    const int ew = warp - 2;
+    const int rq = warp & 3, half = ew >> 2;
+    uint8_t* stage = epi_smem + (size_t)ew * (32 * G_EPI_PITCH);
+    const int srow = lane >> 3, scol = lane & 7;  // this lane's (row mod 4, 16-byte column) when storing
+    int acc_slot = 0;
+    uint32_t acc_phase = 0;
+    bool live = true;
+    for (int l = 0; l < p.n_layers && live; ++l) {
+      const GLayer& L = lay[l];
+      const int Nt = L.Nt, MT = L.MT, K = L.K;
+      const float* alpha = L.alpha;
+      uint32_t* out32 = reinterpret_cast<uint32_t*>(p.out[l]);  // int32 and fp32 outputs share the layout
+      const bool fast = ((K & 3) == 0) && ((Nt & 31) == 0);
+      for (int tile = g_first_tile(L); tile < L.total_tiles; tile += G) {
+        const int mg = (int)fdiv((uint32_t)tile, L.dNt), nti = tile - mg * L.n_ntiles;
+        const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
+        const int n0 = nti * Nt;
+        int okw = 1;
+        if (lane == 0) okw = (!*abort_flag && mbar_wait_backoff(bar_accfull + 8 * acc_slot, acc_phase, 100)) ? 1 : 0;
+        okw = __shfl_sync(0xffffffffu, okw, 0);
+        if (!okw) {
+          if (lane == 0 && !*abort_flag) {
+            *abort_flag = 1;
+            raise_status(p.status, 4);
+          }
+          live = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t d0 = tmem_base + (uint32_t)acc_slot * G_ACC_COLS;
+        // output pixel (n*Ho + y)*Wo + x of the row of sub-tile mt this lane owns in TMEM, or -1
+        auto row_pixel = [&](int mt) -> int {
+          const uint32_t q = Q0 + (uint32_t)(mt * 128 + rq * 32 + lane);
+          const uint32_t rg = fdiv(q, L.dWq);
+          const int x = (int)(q - rg * (uint32_t)L.Wq);
+          const uint32_t n = fdiv(rg, L.dHq);
+          const int y = (int)(rg - n * (uint32_t)L.Hq);
+          const bool valid = ((long long)q < L.Qtot) && ((int)n < L.N) && (y < L.Ho) && (x < L.Wo);
+          return valid ? ((int)n * L.Ho + y) * L.Wo + x : -1;
+        };
+        if (fast) {
+          // The warp's slices (sub-tile mt, columns c0..c0+31) form one sequence; the TMEM load of
+          // slice s+1 is issued as soon as slice s sits in the staging tile.
+          const int per_mt = (Nt - 32 * half + 63) / 64;
+          const int total_sl = MT * per_mt;
+          uint32_t v[32];
+          int ro[8];
+          if (total_sl > 0) tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(32 * half), v);
+          int mt = 0, ci = 0;
+#pragma unroll 1
+          for (int sl = 0; sl < total_sl; ++sl) {
+            const int c0 = 32 * half + 64 * ci;
+            if (ci == 0) {
+              const int mine = row_pixel(mt);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) ro[i] = __shfl_sync(0xffffffffu, mine, srow + 4 * i);
+            }
+            const int co = n0 + c0 + scol * 4;
+            float4 al = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (!p.out_i32 && co < K) al = __ldg(reinterpret_cast<const float4*>(alpha + co));
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              *reinterpret_cast<uint4*>(stage + lane * G_EPI_PITCH + ((e ^ (lane & 7)) << 4)) =
+                  make_uint4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+            __syncwarp();
+            if (++ci == per_mt) { ci = 0; ++mt; }
+            if (sl + 1 < total_sl)
+              tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * Nt + 32 * half + 64 * ci), v);
+            if (co < K) {  // K is a multiple of 4 here, so the four channels exist together
+              uint4 u[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int row = srow + 4 * i;
+                u[i] = *reinterpret_cast<const uint4*>(stage + row * G_EPI_PITCH + ((scol ^ (row & 7)) << 4));
+              }
+              if (!p.out_i32) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  u[i].x = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].x) : small_int_to_float(u[i].x), al.x));
+                  u[i].y = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].y) : small_int_to_float(u[i].y), al.y));
+                  u[i].z = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].z) : small_int_to_float(u[i].z), al.z));
+                  u[i].w = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].w) : small_int_to_float(u[i].w), al.w));
+                }
+              }
+              uint32_t* obase32 = out32 + co;
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                if (ro[i] >= 0) *reinterpret_cast<uint4*>(obase32 + wide_mul((uint32_t)ro[i], (uint32_t)K)) = u[i];
+            }
+            __syncwarp();
+          }
+        } else {
+          // c_out not a multiple of 4 or a channel tile not a multiple of 32: 16-column slices
+          // straight from registers, element by element
+#pragma unroll 1
+          for (int mt = 0; mt < MT; ++mt) {
+            const int pix = row_pixel(mt);
+            const uint32_t trow = d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * Nt);
+            for (int c0 = 16 * half; c0 < Nt; c0 += 32) {
+              uint32_t v[16];
+              tmem_ld16(trow + (uint32_t)c0, v);
+              tmem_ld_wait();
+              const int co0 = n0 + c0;
+              if (pix < 0 || co0 >= K) continue;
+              uint32_t* o = out32 + wide_mul((uint32_t)pix, (uint32_t)K) + co0;
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                if (co0 + e < K) {
+                  if (p.out_i32) o[e] = v[e];
+                  else
+                    o[e] = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(v[e]) : small_int_to_float(v[e]),
+                                                     __ldg(alpha + co0 + e)));
+                }
+              }
+            }
+          }
+        }
+        // this warp has read its part of the accumulator buffer: hand it back to the MMA issuer
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_accempty + 8 * acc_slot);
+        if (++acc_slot == 2) { acc_slot = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------ expanders (warps 10-17)
+    // Fill activation unit (problem, tile, channel block) of the ring: for every plane, row and
+    // 32-channel word, bits -> two 16-byte chunks of +1/-1 bytes (fp16: copy two 8-channel chunks).
+    grid_dep_wait();  // the activations may come from the previous kernel in the stream
+    const int et = tid - (2 + G_EW) * 32;
+    int a_slot = 0;
+    long long a_done = 0;
+    uint32_t a_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
+    volatile int* exp_flag = abort_flag + 1;
+    bool stop = false;
+    for (int l = 0; l < p.n_layers && !stop; ++l) {
+      const GLayer& L = lay[l];
+      const int Rr = L.Rr, n_planes = L.n_planes, n_cb = L.n_cb, cb_chunks = L.cb_chunks, MT = L.MT;
+      const int C = L.C, Cw = L.Cw, total = L.total_tiles;
+      const FastDiv dNt = L.dNt;
+      const void* act = p.act[l];
+      // vector loads of a row's words need the base pointer and the row pitch aligned to the load
+      bool vec;
+      {
+        const uintptr_t addr = (uintptr_t)act;
+        if (F16) vec = (addr & 15) == 0 && (C & 7) == 0;
+        else if (cb_chunks == 8) vec = (addr & 15) == 0 && (Cw & 3) == 0;
+        else if (cb_chunks == 4) vec = (addr & 7) == 0 && (Cw & 1) == 0;
+        else vec = false;
+      }
+      const int nstep = cb_chunks / 2;  // pairs of chunks per unit
+      for (int tile = g_first_tile(L); tile < total && !stop; tile += G) {
+        const int mg = (int)fdiv((uint32_t)tile, dNt);
+        const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
+        // Input pixel of every staged row, once per tile.  The table is private to the expanders:
+        // the barrier keeps a fast thread from overwriting entries another still reads.
+        asm volatile("bar.sync 3, %0;" ::"n"(G_EXP_THREADS) : "memory");
+        for (int pl = 0; pl < n_planes; ++pl)
+          for (int r = et; r < Rr; r += G_EXP_THREADS)
+            pix_tab[pl * Rr + r] = g_position_to_pixel(L, Q0 + (uint32_t)r, pl >> 1, pl & 1);
+        for (int cb = 0; cb < n_cb; ++cb) {
+          if (a_done >= NA) {
+            // one elected thread polls; the rest wait on a hardware barrier instead of spinning
+            if (et == 0) *exp_flag = (!*abort_flag && mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 64)) ? 1 : 0;
+            asm volatile("bar.sync 3, %0;" ::"n"(G_EXP_THREADS) : "memory");
+            const int okf = *exp_flag;
+            asm volatile("bar.sync 3, %0;" ::"n"(G_EXP_THREADS) : "memory");
+            if (!okf) {
+              if (et == 0 && !*abort_flag) {
+                *abort_flag = 1;
+                raise_status(p.status, 1);
+              }
+              stop = true;
+              break;
+            }
+          }
+          uint8_t* unit = a_smem + (size_t)a_slot * p.a_slot_bytes;
+          for (int pl = 0; pl < n_planes; ++pl) {
+            uint8_t* plane = unit + (size_t)pl * cb_chunks * Rr * 16;
+            for (int rb = 0; rb < Rr; rb += G_EXP_ROWS * G_EXP_THREADS) {
+              int pix[G_EXP_ROWS];  // input pixel of each of this thread's rows; -1 padding, -2 past the unit
+#pragma unroll
+              for (int j = 0; j < G_EXP_ROWS; ++j) {
+                const int r = rb + et + j * G_EXP_THREADS;
+                pix[j] = r < Rr ? pix_tab[pl * Rr + r] : -2;
+              }
+              if (F16) {
+                for (int c0 = 0; c0 < cb_chunks; c0 += 2) {
+                  uint4 v[G_EXP_ROWS][2];
+#pragma unroll
+                  for (int j = 0; j < G_EXP_ROWS; ++j) {
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                      v[j][k] = make_uint4(0, 0, 0, 0);
+                      const int ch = (cb * cb_chunks + c0 + k) * 8;  // first channel of the chunk
+                      if (pix[j] >= 0 && ch < C) {
+                        const __half* src = (const __half*)act + wide_mul((uint32_t)pix[j], (uint32_t)C) + ch;
+                        if (vec) {
+                          v[j][k] = __ldg(reinterpret_cast<const uint4*>(src));
+                        } else {
+                          uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+                          for (int e = 0; e < 8; ++e)
+                            if (ch + e < C) w[e >> 1] |= (uint32_t)__half_as_ushort(src[e]) << (16 * (e & 1));
+                          v[j][k] = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                      }
+                    }
+                  }
+#pragma unroll
+                  for (int j = 0; j < G_EXP_ROWS; ++j) {
+                    const int r = rb + et + j * G_EXP_THREADS;
+                    if (pix[j] != -2) {
+                      *reinterpret_cast<uint4*>(plane + ((size_t)c0 * Rr + r) * 16) = v[j][0];
+                      *reinterpret_cast<uint4*>(plane + ((size_t)(c0 + 1) * Rr + r) * 16) = v[j][1];
+                    }
+                  }
+                }
+              } else {
+                // up to four 32-channel words per row and block, as one vector load when aligned
+                const int w0 = cb * nstep;
+                uint32_t bits[G_EXP_ROWS][4];
+#pragma unroll
+                for (int j = 0; j < G_EXP_ROWS; ++j) {
+                  bits[j][0] = bits[j][1] = bits[j][2] = bits[j][3] = 0;
+                  if (pix[j] >= 0 && w0 < Cw) {
+                    const uint32_t* src = (const uint32_t*)act + wide_mul((uint32_t)pix[j], (uint32_t)Cw) + w0;
+                    if (vec && nstep == 4) {
+                      const uint4 t = __ldg(reinterpret_cast<const uint4*>(src));
+                      bits[j][0] = t.x; bits[j][1] = t.y; bits[j][2] = t.z; bits[j][3] = t.w;
+                    } else if (vec && nstep == 2) {
+                      const uint2 t = __ldg(reinterpret_cast<const uint2*>(src));
+                      bits[j][0] = t.x; bits[j][1] = t.y;
+                    } else {
+#pragma unroll
+                      for (int k = 0; k < 4; ++k)
+                        if (k < nstep && w0 + k < Cw) bits[j][k] = __ldg(src + k);
+                    }
+                  }
+                }
+#pragma unroll
+                for (int j = 0; j < G_EXP_ROWS; ++j) {
+                  const int r = rb + et + j * G_EXP_THREADS;
+                  if (pix[j] != -2) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                      if (k < nstep) {
+                        uint4 lo, hi;
+                        expand_word(bits[j][k], C - (w0 + k) * 32, pix[j] >= 0 && w0 + k < Cw, lo, hi);
+                        *reinterpret_cast<uint4*>(plane + ((size_t)(2 * k) * Rr + r) * 16) = lo;
+                        *reinterpret_cast<uint4*>(plane + ((size_t)(2 * k + 1) * Rr + r) * 16) = hi;
+                      }
+                    }
+                  }
+                }
+              }
+            }
+          }
+          fence_proxy_async();  // generic-proxy writes -> visible to the tensor core's reads
+          mbar_arrive(bar_afull + 8 * a_slot);
+          ++a_done;
+          if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side
+struct GroupDev {
+  int count = 0, act_type = 0;
+  GLayer* layers_dev = nullptr;   // [count]
+  uint8_t* weights = nullptr;     // the group's own weight operands, one after the other
+  GParams p{};                    // everything but the per-call pointers
+  size_t smem = 0;
+  int grid = 0;
+};
+
+namespace {
+
+// Tile shape, channel blocks and weight stages of one problem under the group's fixed slot sizes.
+bool g_plan_layer(const Geom& g, bool f16, GLayer* L, int* n_chunks_out, int* Kpad_out) {
+  const int cpc = f16 ? 8 : 16;
+  const int raw = round_up(g.C, 2 * cpc) / cpc;  // 16-byte chunks along the channels, even
+  GLayer& o = *L;
+  o.N = g.N; o.H = g.H; o.W = g.W; o.C = g.C; o.K = g.K; o.Cw = g.Cw;
+  o.stride = g.stride; o.pad = g.pad; o.Ho = g.Ho; o.Wo = g.Wo;
+  if (g.stride == 1) {
+    o.Hq = g.H + g.pad; o.Wq = g.W + g.pad; o.n_planes = 1; o.halo = 2 * o.Wq + 2;
+  } else {
+    o.Hq = g.Ho + 1; o.Wq = g.Wo + 1; o.n_planes = 4; o.halo = o.Wq + 1;
+  }
+  o.dWq = make_fastdiv((uint32_t)o.Wq);
+  o.dHq = make_fastdiv((uint32_t)o.Hq);
+  o.Qtot = (long long)g.N * o.Hq * o.Wq;
+  if (g.N < 1) return false;
+  if (o.Qtot + 1024 + o.halo >= (1ll << 31)) return false;  // positions are 32-bit in the kernel
+  if (g.C > kMaxChannelsSmallInt) return false;             // the drain's int -> float shortcut
+  if ((long long)g.N * g.H * g.W >= (1ll << 31) || (long long)g.N * g.Ho * g.Wo >= (1ll << 31)) return false;
+  o.NtL = g.K <= 256 ? round_up(g.K, 16) : 128;
+  o.Nt = o.NtL;
+  const int Kpad = round_up(g.K, o.NtL);
+  o.n_ntiles = Kpad / o.Nt;
+  o.dNt = make_fastdiv((uint32_t)o.n_ntiles);
+  // channel block: the largest of 8/6/4/2 chunks that divides the channels and whose unit fits a slot
+  int d = 0;
+  for (int c = 8; c >= 2; c -= 2) {
+    if (raw % c) continue;
+    if ((size_t)o.n_planes * c * (128 + o.halo) * 16 <= kGASlotMax) { d = c; break; }
+  }
+  if (!d) return false;
+  o.cb_chunks = d;
+  o.n_cb = raw / d;
+  o.kpt = d / 2;
+  int MT = 1;
+  for (int m = 4; m >= 2; m /= 2)
+    if ((size_t)o.n_planes * d * (128 * m + o.halo) * 16 <= kGASlotMax && m * o.Nt <= (int)G_ACC_COLS) { MT = m; break; }
+  const long long mtiles = (o.Qtot + 127) / 128;
+  while (MT > 1 && mtiles < MT) MT /= 2;  // a tiny problem does not need the larger tile
+  o.MT = MT;
+  o.Rr = 128 * MT + o.halo;
+  if ((uint32_t)o.Rr * 16 >= (1u << 18)) return false;  // leading-offset field of the descriptor
+  const long long mgroups = (mtiles + MT - 1) / MT;
+  if (mgroups * o.n_ntiles > 0x7fffffffLL || mgroups * o.Rr >= (1ll << 31)) return false;
+  o.total_tiles = (int)(mgroups * o.n_ntiles);
+  // weight stage: the longest run of K steps that divides a channel block's 9*kpt and fits a slot
+  const int ks_bytes = 2 * o.Nt * 16;
+  int st = 0;
+  for (int s = 9 * o.kpt; s >= 1; --s)
+    if ((9 * o.kpt) % s == 0 && (size_t)s * ks_bytes <= kGBSlot) { st = s; break; }
+  if (!st) return false;
+  o.st_ksteps = st;
+  o.stage_bytes = (uint32_t)(st * ks_bytes);
+  *n_chunks_out = raw;
+  *Kpad_out = Kpad;
+  return true;
+}
+
+}  // namespace
+
+cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int act_type, cudaStream_t s,
+                       GroupDev** out, int* launched) {
+  *out = nullptr;
+  if (count < 1 || count > SNN_GROUP_MAX) return cudaErrorInvalidConfiguration;
+  const bool f16 = act_type == SNN_ACT_F16;
+  GLayer host[SNN_GROUP_MAX];
+  int n_chunks[SNN_GROUP_MAX], Kpad[SNN_GROUP_MAX];
+  size_t w_off[SNN_GROUP_MAX], w_total = 0;
+  size_t a_slot = 0, pix_bytes = 0;
+  long long tiles = 0;
+  for (int i = 0; i < count; ++i) {
+    if (!g_plan_layer(gs[i], f16, &host[i], &n_chunks[i], &Kpad[i])) return cudaErrorInvalidConfiguration;
+    const size_t unit = (size_t)host[i].n_planes * host[i].cb_chunks * host[i].Rr * 16;
+    if (unit > a_slot) a_slot = unit;
+    const size_t pb = (size_t)host[i].n_planes * host[i].Rr * 4;
+    if (pb > pix_bytes) pix_bytes = pb;
+    w_off[i] = w_total;
+    w_total += ((size_t)9 * n_chunks[i] * Kpad[i] * 16 + 255) & ~(size_t)255;
+    tiles += host[i].total_tiles;
+  }
+  a_slot = (a_slot + 127) & ~(size_t)127;
+  pix_bytes = (pix_bytes + 127) & ~(size_t)127;
+  const size_t lay_bytes = ((size_t)count * sizeof(GLayer) + 127) & ~(size_t)127;
+  const size_t fixed = (size_t)G_EPI_BYTES + pix_bytes + lay_bytes + kGTail;
+  int na = 3, ns = 0;
+  for (; na >= 2; --na) {
+    if ((size_t)na * a_slot + fixed + 3 * (size_t)kGBSlot > kGSmemBudget) continue;
+    ns = (int)((kGSmemBudget - fixed - (size_t)na * a_slot) / kGBSlot);
+    break;
+  }
+  if (na < 2 || ns < 3) return cudaErrorInvalidConfiguration;
+  if (ns > G_NS_MAX) ns = G_NS_MAX;
+  const int sms = sm_count();
+  const int grid = tiles < sms ? (int)tiles : sms;
+  int off = 0;
+  for (int i = 0; i < count; ++i) {
+    host[i].tile_off = off;
+    off = (int)(((long long)off + host[i].total_tiles) % grid);
+  }
+  GroupDev* G = new GroupDev();
+  G->count = count;
+  G->act_type = act_type;
+  G->grid = grid;
+  cudaError_t e = cudaMalloc(&G->weights, w_total);
+  if (e == cudaSuccess) e = cudaMalloc(&G->layers_dev, sizeof(GLayer) * count);
+  for (int i = 0; i < count && e == cudaSuccess; ++i) {
+    host[i].wt = G->weights + w_off[i];
+    host[i].alpha = Ls[i]->alpha;
+    e = tc_expand_weights_custom(Ls[i]->wplanes, G->weights + w_off[i], gs[i].C, gs[i].K, gs[i].Cw, Kpad[i],
+                                 n_chunks[i], host[i].cb_chunks, host[i].NtL, f16, s);
+    if (e == cudaSuccess) *launched += 1;
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(G->layers_dev, host, sizeof(GLayer) * count, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);  // `host` lives on this stack
+  if (e != cudaSuccess) {
+    tcg_destroy(G);
+    return e;
+  }
+  GParams& p = G->p;
+  p.layers = G->layers_dev;
+  p.n_layers = count;
+  p.NA = na;
+  p.NS = ns;
+  p.a_slot_bytes = (uint32_t)a_slot;
+  p.b_slot_bytes = kGBSlot;
+  p.off_b = (uint32_t)((size_t)na * a_slot);
+  p.off_epi = p.off_b + (uint32_t)ns * kGBSlot;
+  p.off_pix = p.off_epi + G_EPI_BYTES;
+  p.off_lay = p.off_pix + (uint32_t)pix_bytes;
+  p.off_tail = p.off_lay + (uint32_t)lay_bytes;
+  G->smem = (size_t)p.off_tail + kGTail;
+  if (G->smem > (size_t)kMaxDynSmem || G->smem >= (1u << 18)) {
+    tcg_destroy(G);
+    return cudaErrorInvalidConfiguration;
+  }
+  *out = G;
+  return cudaSuccess;
+}
+
+void tcg_destroy(GroupDev* G) {
+  if (!G) return;
+  cudaFree(G->weights);
+  cudaFree(G->layers_dev);
+  delete G;
+}
+
+int tcg_count(const GroupDev* G) { return G->count; }
+
+cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, int out_i32, cudaStream_t s,
+                        int* status_dev, int* launched) {
+  GParams p = G->p;
+  for (int i = 0; i < G->count; ++i) {
+    p.act[i] = act[i];
+    p.out[i] = out[i];
+  }
+  p.out_i32 = out_i32;
+  p.status = status_dev;
+  // Launched as a programmatic dependent of its predecessor in the stream: set-up overlaps that
+  // kernel's tail; the warps that read activations or write outputs wait on the device for it.
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)G->grid);
+  cfg.blockDim = dim3(G_THREADS);
+  cfg.dynamicSmemBytes = G->smem;
+  cudaError_t e;
+  if (G->act_type == SNN_ACT_F16) {
+    static unsigned long long done = 0;
+    e = allow_max_smem(tcg_conv_kernel<true>, &done);
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<true>, p);
+  } else {
+    static unsigned long long done = 0;
+    e = allow_max_smem(tcg_conv_kernel<false>, &done);
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<false>, p);
+  }
+  if (e != cudaSuccess) return e;
+  *launched += 1;
+  return cudaGetLastError();
+}
+
+}  // namespace snn

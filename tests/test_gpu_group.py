@@ -1,0 +1,159 @@
+"""Parity of the grouped launch (snn_conv_group_*: several independent layer problems
+in one persistent tensor-core kernel) with the CPU oracle, member by member and
+element by element.  Bar as for single layers: int32 sums bit-exact, fp32 outputs
+equal (1e-6 relative), fp16-activation variant within 2e-2 of max(|ref|, alpha*sqrt(9*c_in))."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+REL_F32 = 1e-6
+REL_F16 = 2e-2
+
+
+@pytest.fixture(scope="module")
+def snn():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2110_09195_b200 import build
+    build.build()
+    import paper_2110_09195_b200 as m
+    m.load_library()
+    return m
+
+
+def _guarded(shape, dtype, guard=64):
+    n = int(np.prod(shape))
+    flat = torch.full((n + 2 * guard,), -12345 if dtype == torch.int32 else -12345.0, dtype=dtype, device="cuda:0")
+    return flat, flat[guard:guard + n].view(*shape)
+
+
+def _intact(flat, n, guard=64):
+    return bool((flat[:guard] == -12345).all()) and bool((flat[guard + n:] == -12345).all())
+
+
+def check_bin_group(snn, oracle_mod, members, tau, seed, repeats=1):
+    """members: list of (LayerShape, batch).  Every member gets its own parameters and input."""
+    layers, acts, refs = [], [], []
+    for i, (shape, n) in enumerate(members):
+        p = wl.draw_layer_params(shape, tau, seed + i)
+        packed = wl.pack_activation_bits(wl.draw_activation_bits(shape, n, seed + i))
+        refs.append(oracle_mod.conv_bin(p.codebook, tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out, shape.stride,
+                                        shape.pad, packed))
+        layers.append(snn.SnnConv(shape.c_in, shape.c_out, tau, p.codebook, p.idx_packed, p.alpha, shape.stride,
+                                  shape.pad, snn.ACT_BIN))
+        acts.append(torch.from_numpy(packed.view(np.int32)).cuda())
+    group = snn.SnnConvGroup(layers, [(n, s.h, s.w) for s, n in members])
+    for _ in range(repeats):
+        gs = [_guarded(r[0].shape, torch.int32) for r in refs]
+        gy = [_guarded(r[1].shape, torch.float32) for r in refs]
+        group.forward(acts, [g[1] for g in gs], snn.OUT_I32)
+        group.forward(acts, [g[1] for g in gy], snn.OUT_F32)
+        torch.cuda.synchronize()
+        for i, (s_ref, y_ref) in enumerate(refs):
+            s, y = gs[i][1].cpu().numpy(), gy[i][1].cpu().numpy()
+            assert _intact(gs[i][0], s_ref.size) and _intact(gy[i][0], y_ref.size), f"member {i}: canary overwritten"
+            bad = np.argwhere(s != s_ref)
+            assert bad.size == 0, f"member {i} {members[i][0]}: {len(bad)} int32 mismatches, first at {bad[0]}: " \
+                                  f"{s[tuple(bad[0])]} vs {s_ref[tuple(bad[0])]}"
+            assert (np.abs(y - y_ref) <= REL_F32 * np.abs(y_ref)).all(), f"member {i}"
+            assert (y == y_ref).all(), f"member {i}"
+    group.destroy()
+    for l in layers:
+        l.destroy()
+
+
+def test_group_of_one_small(snn, oracle_mod):
+    check_bin_group(snn, oracle_mod, [(wl.LayerShape(16, 16, 32, 32, 1, 1), 1)], 5, 11)
+
+
+def test_group_ragged_members(snn, oracle_mod):
+    """Ragged channels in and out, stride 2 (four parity planes), no padding, one-pixel maps,
+    several channel blocks: every member shape the kernel treats differently, in one launch."""
+    members = [
+        (wl.LayerShape(33, 7, 9, 11, 1, 1), 3),
+        (wl.LayerShape(70, 37, 13, 6, 2, 1), 2),
+        (wl.LayerShape(5, 3, 7, 6, 2, 0), 2),
+        (wl.LayerShape(64, 64, 5, 8, 1, 0), 2),
+        (wl.LayerShape(16, 16, 1, 1, 1, 1), 5),
+        (wl.LayerShape(96, 130, 3, 17, 1, 1), 1),
+        (wl.LayerShape(300, 20, 6, 5, 1, 1), 2),
+        (wl.LayerShape(1056, 48, 9, 8, 2, 1), 1),
+        (wl.LayerShape(200, 300, 7, 5, 1, 1), 2),
+    ]
+    check_bin_group(snn, oracle_mod, members, 5, 21)
+
+
+@pytest.mark.parametrize("net,cfg", [("resnet20", 1), ("resnet18", 2)])
+def test_group_stack_small_batch(snn, oracle_mod, net, cfg):
+    """The whole stack as one group (all layers, in order), batch 2."""
+    wk = wl.get_workload(net)
+    check_bin_group(snn, oracle_mod, [(s, 2) for s in wk.layers], wk.tau, 31 + cfg, repeats=2)
+
+
+def test_group_many_tiles_per_cta(snn, oracle_mod):
+    """More tiles than twice the CTAs in several members: every ring (activation units, weight
+    stages, accumulator buffers) wraps around many times and carries over between members."""
+    members = [
+        (wl.LayerShape(64, 64, 56, 56, 1, 1), 24),
+        (wl.LayerShape(128, 128, 28, 28, 1, 1), 40),
+        (wl.LayerShape(64, 128, 56, 56, 2, 1), 12),
+        (wl.LayerShape(256, 256, 14, 14, 1, 1), 48),
+        (wl.LayerShape(512, 512, 7, 7, 1, 1), 64),
+        (wl.LayerShape(256, 512, 14, 14, 2, 1), 16),
+    ]
+    check_bin_group(snn, oracle_mod, members, 5, 41)
+
+
+def test_group_fp16(snn, oracle_mod):
+    members = [(wl.LayerShape(64, 64, 14, 14, 1, 1), 3), (wl.LayerShape(136, 72, 9, 7, 2, 1), 2),
+               (wl.LayerShape(33, 7, 6, 5, 2, 1), 2), (wl.LayerShape(256, 256, 7, 7, 1, 1), 2)]
+    layers, acts, refs, alphas = [], [], [], []
+    for i, (shape, n) in enumerate(members):
+        p = wl.draw_layer_params(shape, 5, 51 + i)
+        a = wl.draw_activation_f16(shape, n, 51 + i)
+        refs.append(oracle_mod.conv_f16(p.codebook, 5, p.idx_packed, p.alpha, shape.c_in, shape.c_out, shape.stride,
+                                        shape.pad, a))
+        alphas.append(p.alpha)
+        layers.append(snn.SnnConv(shape.c_in, shape.c_out, 5, p.codebook, p.idx_packed, p.alpha, shape.stride,
+                                  shape.pad, snn.ACT_F16))
+        acts.append(torch.from_numpy(a).cuda())
+    group = snn.SnnConvGroup(layers, [(n, s.h, s.w) for s, n in members])
+    outs = group.forward(acts)
+    torch.cuda.synchronize()
+    for i, ((shape, n), y_ref) in enumerate(zip(members, refs)):
+        y = outs[i].cpu().numpy().astype(np.float64)
+        sigma = alphas[i].astype(np.float64) * np.sqrt(9.0 * shape.c_in)
+        bound = REL_F16 * np.maximum(np.abs(y_ref.astype(np.float64)), sigma[None, None, None, :])
+        err = np.abs(y - y_ref.astype(np.float64))
+        assert (err <= bound).all(), f"member {i}: max err/bound {np.max(err / bound)}"
+        assert np.linalg.norm(err) <= 1e-4 * np.linalg.norm(y_ref)
+    group.destroy()
+    for l in layers:
+        l.destroy()
+
+
+def test_group_argument_errors(snn):
+    shape = wl.LayerShape(16, 16, 8, 8)
+    p = wl.draw_layer_params(shape, 5, 3)
+    a = snn.SnnConv(16, 16, 5, p.codebook, p.idx_packed, p.alpha)
+    b = snn.SnnConv(16, 16, 5, p.codebook, p.idx_packed, p.alpha, act_type=snn.ACT_F16)
+    with pytest.raises(snn.SnnError) as ei:
+        snn.SnnConvGroup([a, b], [(1, 8, 8), (1, 8, 8)])       # mixed activation types
+    assert ei.value.status == 1
+    with pytest.raises(snn.SnnError) as ei:
+        snn.SnnConvGroup([a], [(0, 8, 8)])                     # empty member
+    assert ei.value.status == 1
+    with pytest.raises(snn.SnnError) as ei:
+        snn.SnnConvGroup([a] * 33, [(1, 8, 8)] * 33)           # more members than a group holds
+    assert ei.value.status == 1
+    g = snn.SnnConvGroup([a], [(1, 8, 8)])
+    with pytest.raises(snn.SnnError) as ei:
+        g.forward([torch.zeros((2, 8, 8, 1), dtype=torch.int32, device="cuda")])   # not the group's shape
+    assert ei.value.status == 1
+    g.destroy()
+    a.destroy()
+    b.destroy()
