@@ -44,7 +44,7 @@ constexpr uint32_t G_ACC_COLS = 256;          // tensor-memory columns of one ac
 constexpr size_t kGTail = 512;
 constexpr size_t kGSmemBudget = 226 * 1024;
 constexpr uint32_t kGASlotMax = 40 * 1024 + 512;   // largest activation unit a problem may stage
-constexpr uint32_t kGBSlot = 16 * 1024;            // bytes of a weight-stage slot
+constexpr uint32_t kGBSlot = 32 * 1024;            // bytes of a weight-stage slot
 
 // One problem of a group, as the kernel reads it from global memory.
 struct GLayer {
@@ -103,7 +103,8 @@ template <bool F16, int MT, int KPT>
 __device__ __forceinline__ bool g_issue_block(uint64_t a_unit, const uint32_t* tapu, uint32_t a_step,
                                               uint64_t b_desc0, uint32_t b_slot_units, uint32_t b_step, uint32_t d0,
                                               uint32_t nt, uint32_t idesc, uint32_t& acc, int st_ksteps, int NS,
-                                              uint32_t bar_bfull, uint32_t bar_bempty, int& b_slot, uint32_t& b_phase) {
+                                              uint32_t bar_bfull, uint32_t bar_bempty, int& b_slot, uint32_t& b_phase,
+                                              bool leader) {
   int in_stage = 0;
   uint64_t bd = 0;
 #pragma unroll 1
@@ -116,15 +117,17 @@ __device__ __forceinline__ bool g_issue_block(uint64_t a_unit, const uint32_t* t
         tc_fence_after();
         bd = b_desc0 + (uint64_t)((uint32_t)b_slot * b_slot_units);
       }
+      if (leader) {
 #pragma unroll
-      for (int mt = 0; mt < MT; ++mt)
-        mma_ss<F16>(d0 + (uint32_t)mt * nt, ad_t + (uint64_t)((uint32_t)k * a_step + (uint32_t)(mt * 128)), bd, idesc,
-                    acc);
+        for (int mt = 0; mt < MT; ++mt)
+          mma_ss<F16>(d0 + (uint32_t)mt * nt, ad_t + (uint64_t)((uint32_t)k * a_step + (uint32_t)(mt * 128)), bd,
+                      idesc, acc);
+      }
       acc = 1;
       bd += b_step;
       if (++in_stage == st_ksteps) {
         in_stage = 0;
-        tc_commit(bar_bempty + 8 * b_slot);  // the slot is free once these MMAs have read it
+        if (leader) tc_commit(bar_bempty + 8 * b_slot);  // the slot is free once these MMAs have read it
         if (++b_slot == NS) { b_slot = 0; b_phase ^= 1u; }
       }
     }
@@ -241,8 +244,13 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------------------------ MMA issuer (one lane)
-    if (lane == 0) {
+    // ------------------------------------------------ MMA issuer
+    // The whole warp walks the loops and waits together, so that every address and descriptor
+    // is a warp-uniform value; one elected lane issues the MMAs and the commits.
+    {
+      uint32_t elected;
+      asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(elected));
+      const bool leader = elected != 0;
       bool ok = true;
       int a_slot = 0, b_slot = 0, acc_slot = 0;
       uint32_t a_phase = 0, b_phase = 0, acc_phase = 1;
@@ -260,13 +268,15 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         const uint64_t b_desc0 = make_desc(smem_u32(b_smem), (uint32_t)Nt * 16, 128);
         const uint32_t a_step = 2u * (uint32_t)Rr, b_step = 2u * (uint32_t)Nt;  // two chunks per MMA
         // rows (16-byte units) from a unit's origin to tap t: plane offset + shift inside the plane
-#pragma unroll
-        for (int t = 0; t < 9; ++t) {
+        __syncwarp();
+        if (lane < 9) {
+          const int t = lane;
           const int ky = t / 3, kx = t % 3;
           tapu[t] = L.stride == 1 ? (uint32_t)(ky * L.Wq + kx)
                                   : (uint32_t)((ky & 1) * 2 + (kx & 1)) * (uint32_t)(L.cb_chunks * Rr) +
                                         (uint32_t)((ky >> 1) * L.Wq + (kx >> 1));
         }
+        __syncwarp();
         for (int tile = g_first_tile(L); tile < total && ok; tile += G, ++tiles_done) {
           if (tiles_done >= 2) {
             if (!mbar_wait(bar_accempty + 8 * acc_slot, acc_phase)) { ok = false; break; }
@@ -280,7 +290,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
             const uint64_t a_unit = a_desc0 + (uint64_t)((uint32_t)a_slot * a_slot_units);
 #define G_ISSUE(M, KP)                                                                                       \
   ok = g_issue_block<F16, M, KP>(a_unit, tapu, a_step, b_desc0, b_slot_units, b_step, d0, (uint32_t)Nt, idesc, acc, \
-                                 st_ksteps, NS, bar_bfull, bar_bempty, b_slot, b_phase)
+                                 st_ksteps, NS, bar_bfull, bar_bempty, b_slot, b_phase, leader)
 #define G_ISSUE_K(M)                   \
   do {                                 \
     if (kpt == 4) G_ISSUE(M, 4);       \
@@ -294,15 +304,15 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 #undef G_ISSUE_K
 #undef G_ISSUE
             if (!ok) break;
-            tc_commit(bar_aempty + 8 * a_slot);  // the activation unit may be overwritten
+            if (leader) tc_commit(bar_aempty + 8 * a_slot);  // the activation unit may be overwritten
             if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
           }
           if (!ok) break;
-          tc_commit(bar_accfull + 8 * acc_slot);  // fires when this tile's MMAs are complete
+          if (leader) tc_commit(bar_accfull + 8 * acc_slot);  // fires when this tile's MMAs are complete
           if (++acc_slot == 2) { acc_slot = 0; acc_phase ^= 1u; }
         }
       }
-      if (!ok && !*abort_flag) {
+      if (!ok && leader && !*abort_flag) {
         *abort_flag = 1;
         raise_status(p.status, 3);
       }
