@@ -172,6 +172,23 @@ def run_reference(args):
     return 0
 
 
+# DRAM traffic per launch of the dominant kernel from an ncu capture (profiles/), valid only while
+# the kernel's sources are the ones that were profiled: {kernel: (workload, batch, bytes, sha256 of sources)}
+_TRAFFIC = {}
+
+
+def _profiled_traffic(kernel_name, nb, workload):
+    import hashlib
+    rec = _TRAFFIC.get(kernel_name)
+    if rec is None or rec[0] != workload.name or rec[1] != nb:
+        return None
+    h = hashlib.sha256()
+    for f in ("snn_tcg.cu", "snn_tc_common.cuh"):
+        with open(os.path.join(ROOT, "paper_2110_09195_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return rec[2] if h.hexdigest() == rec[3] else None
+
+
 def _workload_name(workload):
     return f"{workload.name}_stack_n{workload.batch}_tau{workload.tau}_{workload.act}"
 
@@ -281,12 +298,13 @@ def run_ours(args):
     all_idx = list(range(len(layers)))
     use_graph = not args.no_graph
     group = None
-    if args.group:
+    grouped = not args.per_layer and mb == 1 and n_lanes == 1 and forced in (snn.PATH_AUTO, snn.PATH_DECODED_TC)
+    seq_graph = None
+    if grouped:
         # The layers of the benchmark are independent problems (each has its own input): the step
         # is one persistent launch that walks through all of them (snn_conv_group_forward).
-        if mb != 1 or n_lanes != 1 or forced not in (snn.PATH_AUTO, snn.PATH_DECODED_TC):
-            raise SystemExit("--group runs the tensor-core path on one stream without micro-batches")
         group = snn.SnnConvGroup(layers, [(nb, s.h, s.w) for s in workload.layers])
+        seq_graph = capture(all_idx) if use_graph else None   # the same step as per-layer launches, timed beside it
 
         def launch_group(stream):
             group.forward(acts, outs, snn.OUT_F32, stream)
@@ -338,6 +356,25 @@ def run_ours(args):
     step_ms = [e0.elapsed_time(e1) for e0, e1 in ev]
     total_ms = float(sum(step_ms))
 
+    # the same step as one launch per layer, back to back on one stream (what a caller of
+    # snn_conv_forward gets), timed the same way over fewer steps
+    seq_ms = None
+    if group is not None:
+        k = max(3, min(30, args.steps))
+        ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(k)]
+        for i in range(k + 3):
+            flush.zero_()
+            if i >= 3:
+                ev2[i - 3][0].record(stream)
+            if seq_graph is not None:
+                seq_graph.replay()
+            else:
+                launch_layers(all_idx, stream)
+            if i >= 3:
+                ev2[i - 3][1].record(stream)
+        torch.cuda.synchronize(dev)
+        seq_ms = float(sum(a.elapsed_time(b) for a, b in ev2)) / k
+
     # per-layer device time (same launch configuration, L2 flushed before every layer; the
     # flush also keeps the GPU busy while the host enqueues, so no host latency is timed)
     reps = max(3, min(20, args.steps))
@@ -388,6 +425,19 @@ def run_ours(args):
     dom = max(by_path, key=lambda k: by_path[k]["ms"])
     d = by_path[dom]
     sec = d["ms"] * 1e-3
+    kernel_name = snn.PATH_NAMES[dom]
+    if group is not None:
+        # one kernel does the whole step: its launch duration is the step time measured in the timed region
+        dom = snn.PATH_DECODED_TC
+        d = {"ms": ms_per_step, "macs": workload.dense_macs(), "bytes": workload.algorithmic_bytes(), "launches": 1}
+        sec = ms_per_step * 1e-3
+        kernel_name = "tcg_conv_kernel (grouped decoded_tc)"
+    elif len(by_path) == 1 and mb == 1 and n_lanes == 1:
+        # every launch of the step is this path's kernel, back to back: use the time of the timed region
+        # (the per-layer figures in layer_ms are taken one layer at a time after a flush and add the
+        # event clock's 2 us granularity to every layer)
+        d = dict(d, ms=ms_per_step)
+        sec = ms_per_step * 1e-3
     hbm_frac = d["bytes"] / sec / 1e9 / peaks["hbm_gbs"]
     alu_rates = {}
     if dom == snn.PATH_DECODED_TC:
@@ -413,8 +463,12 @@ def run_ours(args):
                     "frac": hbm_frac}
     else:
         roofline = pipe
-    roofline.update({"traffic": None, "kernel": snn.PATH_NAMES[dom], "launches_per_step": d["launches"],
-                     "share_of_step": d["ms"] / max(sum(layer_ms), 1e-9), "peak_source": peaks["source"],
+    roofline.update({"traffic": _profiled_traffic(kernel_name, nb, workload), "kernel": kernel_name,
+                     "launches_per_step": d["launches"],
+                     "share_of_step": 1.0 if group is not None else d["ms"] / max(sum(layer_ms), 1e-9),
+                     "peak_source": peaks["source"],
+                     "algorithmic_bytes_per_launch": d["bytes"] / d["launches"],
+                     "algorithmic_ops_per_launch": 2 * d["macs"] / d["launches"],
                      "hbm_frac": hbm_frac, "pipe_frac": pipe["frac"], **alu_rates})
     # whole-step roofline: sum over layers of max(HBM floor, pipe floor at the path's peak)
     step_floor_hbm_ms = workload.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e3
@@ -425,7 +479,10 @@ def run_ours(args):
         "dtype": "int32" if workload.act == "bin" else "f16", "data": "synthetic",
         "config": {"workload": _workload_name(workload), "layers": len(layers), "batch_per_gpu": nb,
                    "tau": workload.tau, "l2": "flushed between timed steps (256 MB write)",
-                   "launch": ("host calls" if args.no_graph else "CUDA graph of the per-layer C-ABI launches") +
+                   "launch": ("one grouped launch of all layers (snn_conv_group_forward), " if group is not None else "") +
+                             ("host calls" if args.no_graph else
+                              "replayed as a CUDA graph" if group is not None else
+                              "CUDA graph of the per-layer C-ABI launches") +
                              (f", {mb} micro-batches of {part} images on {mb} streams" if mb > 1 else ""),
                    "microbatches": mb, "streams": n_lanes, "grouped": group is not None,
                    "paths": [snn.PATH_NAMES[p] for p in paths]},
@@ -433,6 +490,9 @@ def run_ours(args):
         "hbm_floor_ms_per_step": step_floor_hbm_ms,
         "step_frac_of_hbm_floor": step_floor_hbm_ms / ms_per_step,
         "layer_ms": [round(v, 5) for v in layer_ms],
+        "per_layer_launches": None if seq_ms is None else {
+            "ms_per_step": seq_ms, "value": nb / (seq_ms * 1e-3), "unit": UNIT + " per GPU",
+            "what": "the same step as one snn_conv_forward launch per layer, back to back on one stream"},
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms},
@@ -476,8 +536,8 @@ def main():
                     help="cut the batch into this many parts, each running the layers in order on its own stream")
     ap.add_argument("--streams", type=int, default=1,
                     help="issue the (independent) layers of a step round-robin on this many streams")
-    ap.add_argument("--group", action="store_true",
-                    help="run the step as one grouped launch of all layers (independent problems)")
+    ap.add_argument("--per-layer", action="store_true",
+                    help="run the step as one launch per layer instead of one grouped launch of all layers")
     ap.add_argument("--no-graph", action="store_true", help="launch every layer from the host instead of a CUDA graph")
     ap.add_argument("--layers", default=None, help="a:b restricts the stack to layers [a, b) (profiling aid)")
     args = ap.parse_args()
