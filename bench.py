@@ -243,7 +243,7 @@ def run_ours(args):
         acts.append(a.to(dev))
         outs.append(layer.alloc_out(nb, shape.h, shape.w))
         host_outs.append(layer.alloc_out(nb, shape.h, shape.w, pin=True))
-        if forced == snn.PATH_AUTO:
+        if forced == snn.PATH_AUTO and not args.group_only:
             layer.tune(nb // mb, shape.h, shape.w)
         paths.append(layer.chosen_path(nb // mb, shape.h, shape.w) if forced == snn.PATH_AUTO else forced)
         layers.append(layer)
@@ -304,7 +304,8 @@ def run_ours(args):
         # The layers of the benchmark are independent problems (each has its own input): the step
         # is one persistent launch that walks through all of them (snn_conv_group_forward).
         group = snn.SnnConvGroup(layers, [(nb, s.h, s.w) for s in workload.layers])
-        seq_graph = capture(all_idx) if use_graph else None   # the same step as per-layer launches, timed beside it
+        # the same step as per-layer launches, timed beside it
+        seq_graph = capture(all_idx) if use_graph and not args.group_only else None
 
         def launch_group(stream):
             group.forward(acts, outs, snn.OUT_F32, stream)
@@ -359,7 +360,7 @@ def run_ours(args):
     # the same step as one launch per layer, back to back on one stream (what a caller of
     # snn_conv_forward gets), timed the same way over fewer steps
     seq_ms = None
-    if group is not None:
+    if group is not None and not args.group_only:
         k = max(3, min(30, args.steps))
         ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(k)]
         for i in range(k + 3):
@@ -377,9 +378,9 @@ def run_ours(args):
 
     # per-layer device time (same launch configuration, L2 flushed before every layer; the
     # flush also keeps the GPU busy while the host enqueues, so no host latency is timed)
-    reps = max(3, min(20, args.steps))
+    reps = 0 if args.group_only else max(3, min(20, args.steps))
     layer_ms = [0.0] * len(layers)
-    layer_graphs = [capture([j]) for j in all_idx] if use_graph else None
+    layer_graphs = [capture([j]) for j in all_idx] if use_graph and reps else None
     for _ in range(reps):
         for j in all_idx:
             flush.zero_()
@@ -536,6 +537,8 @@ def main():
                     help="cut the batch into this many parts, each running the layers in order on its own stream")
     ap.add_argument("--streams", type=int, default=1,
                     help="issue the (independent) layers of a step round-robin on this many streams")
+    ap.add_argument("--group-only", action="store_true",
+                    help="time only the grouped launch: no tuning, no per-layer timings (profiling aid)")
     ap.add_argument("--per-layer", action="store_true",
                     help="run the step as one launch per layer instead of one grouped launch of all layers")
     ap.add_argument("--no-graph", action="store_true", help="launch every layer from the host instead of a CUDA graph")

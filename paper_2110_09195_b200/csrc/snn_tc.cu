@@ -258,8 +258,12 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 8 ? 1 : 2) tc_conv_kerne
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------------------------ MMA issuer (one lane)
-    if (lane == 0) {
+    // ------------------------------------------------ MMA issuer
+    // The whole warp walks the loops and waits together, so that every address and descriptor is
+    // a warp-uniform value (no per-MMA moves into uniform registers); one elected lane issues the
+    // MMAs and the commits.
+    {
+      const bool leader = elect_one();
       // instruction descriptor: D format, A/B formats, K-major both, N>>3, M>>4
       const uint32_t idesc = F16 ? ((1u << 4) | ((uint32_t)(p.Nt >> 3) << 17) | ((128u >> 4) << 24))
                                  : ((2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.Nt >> 3) << 17) |
@@ -301,25 +305,27 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 8 ? 1 : 2) tc_conv_kerne
 #pragma unroll
               for (int k = 0; k < (KPT ? KPT : 4); ++k) {
                 if (KPT || k < kpt) {
+                  if (leader) {
 #pragma unroll
-                  for (int mt = 0; mt < MT; ++mt)
-                    mma_ss<F16>(d0 + (uint32_t)mt * nt, ad + (uint64_t)(mt * 128), bd, idesc, acc);
+                    for (int mt = 0; mt < MT; ++mt)
+                      mma_ss<F16>(d0 + (uint32_t)mt * nt, ad + (uint64_t)(mt * 128), bd, idesc, acc);
+                  }
                   acc = 1;
                   ad += a_step;
                   bd += b_step;
                 }
               }
             }
-            if (!p.b_resident) tc_commit(bar_bempty + 8 * b_slot);  // free once these MMAs have read it
+            if (!p.b_resident && leader) tc_commit(bar_bempty + 8 * b_slot);  // free once these MMAs have read it
             if (++b_slot == NS) { b_slot = 0; b_phase ^= 1u; }
           }
-          tc_commit(bar_aempty + 8 * a_slot);  // the activation unit may be overwritten
+          if (leader) tc_commit(bar_aempty + 8 * a_slot);  // the activation unit may be overwritten
           if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
         }
-        tc_commit(bar_accfull + 8 * acc_slot);  // fires when this tile's MMAs are complete
+        if (leader) tc_commit(bar_accfull + 8 * acc_slot);  // fires when this tile's MMAs are complete
         if (++acc_slot == p.n_acc) { acc_slot = 0; acc_phase ^= 1u; }
       }
-      if (!ok) {
+      if (!ok && leader) {
         *abort_flag = 1;
         raise_status(p.status, 3);
       }

@@ -101,6 +101,13 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// One lane of a fully active warp (the same one every time); the others get false.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t elected;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(elected));
+  return elected != 0;
+}
+
 // Programmatic dependent launch: a kernel launched with the serialization attribute may start
 // while its predecessor in the stream still runs; grid_dep_wait() blocks until the predecessor has
 // completed and its writes are visible (a no-op for an ordinary launch), grid_dep_launch() lets the

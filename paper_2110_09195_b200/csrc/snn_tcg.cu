@@ -248,9 +248,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     // The whole warp walks the loops and waits together, so that every address and descriptor
     // is a warp-uniform value; one elected lane issues the MMAs and the commits.
     {
-      uint32_t elected;
-      asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(elected));
-      const bool leader = elected != 0;
+      const bool leader = elect_one();
       bool ok = true;
       int a_slot = 0, b_slot = 0, acc_slot = 0;
       uint32_t a_phase = 0, b_phase = 0, acc_phase = 1;

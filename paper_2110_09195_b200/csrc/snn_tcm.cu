@@ -192,8 +192,11 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
   const int my_tiles = (p.total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
 
   if (warp == 1) {
-    // ------------------------------------------------ MMA issuer (one lane)
-    if (lane == 0) {
+    // ------------------------------------------------ MMA issuer
+    // The whole warp walks the loops and waits together, so that every address and descriptor is
+    // a warp-uniform value; one elected lane issues the MMAs and the commits.
+    {
+      const bool leader = elect_one();
       const uint32_t idesc = F16 ? ((1u << 4) | ((uint32_t)(p.Np >> 3) << 17) | ((128u >> 4) << 24))
                                  : ((2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.Np >> 3) << 17) |
                                     ((128u >> 4) << 24));
@@ -236,21 +239,22 @@ __global__ void __launch_bounds__(CM_THREADS, 1) cm_conv_kernel(const CmParams p
                 }
                 wbase = ring + (uint32_t)(w_slot * (8 * CM_WST));
               }
-              mma_ts<F16>(d0, wbase + (uint32_t)((j % CM_WST) * 8), bt + (uint32_t)k * a_step, b_hi, idesc, acc);
+              if (leader)
+                mma_ts<F16>(d0, wbase + (uint32_t)((j % CM_WST) * 8), bt + (uint32_t)k * a_step, b_hi, idesc, acc);
               acc = 1;
               if (j % CM_WST == CM_WST - 1 || j == 9 * KPT - 1) {
-                if (!p.w_resident) tc_commit(bar_wempty + 8 * w_slot);  // the ring stage may be overwritten
+                if (!p.w_resident && leader) tc_commit(bar_wempty + 8 * w_slot);  // the ring stage may be overwritten
                 if (++w_slot == NW) { w_slot = 0; w_phase ^= 1u; }
               }
             }
           }
-          tc_commit(bar_aempty + 8 * a_slot);
+          if (leader) tc_commit(bar_aempty + 8 * a_slot);
           if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
         }
-        tc_commit(bar_accfull + 8 * acc_slot);
+        if (leader) tc_commit(bar_accfull + 8 * acc_slot);
         if (++acc_slot == p.n_acc) { acc_slot = 0; acc_phase ^= 1u; }
       }
-      if (!ok) {
+      if (!ok && leader) {
         *abort_flag = 1;
         raise_status(p.status, 3);
       }
