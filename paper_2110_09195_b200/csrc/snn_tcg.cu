@@ -629,7 +629,9 @@ bool g_plan_layer(const Geom& g, bool f16, GLayer* L, int* n_chunks_out, int* Kp
   if (o.Qtot + 1024 + o.halo >= (1ll << 31)) return false;  // positions are 32-bit in the kernel
   if (g.C > kMaxChannelsSmallInt) return false;             // the drain's int -> float shortcut
   if ((long long)g.N * g.H * g.W >= (1ll << 31) || (long long)g.N * g.Ho * g.Wo >= (1ll << 31)) return false;
-  o.NtL = g.K <= 256 ? round_up(g.K, 16) : 128;
+  // layout tile of the weight operand = channels per tile: all of them up to 256; beyond that 256
+  // when that pads little (fewer channel tiles re-expand the same activations), else 128
+  o.NtL = g.K <= 256 ? round_up(g.K, 16) : (round_up(g.K, 256) - g.K < 64 ? 256 : 128);
   o.Nt = o.NtL;
   const int Kpad = round_up(g.K, o.NtL);
   o.n_ntiles = Kpad / o.Nt;
