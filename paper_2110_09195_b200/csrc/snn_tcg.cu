@@ -34,7 +34,9 @@ namespace snn {
 namespace {
 
 constexpr int G_EW = 8;                       // epilogue warps = expander warps
-constexpr int G_THREADS = 64 + 64 * G_EW;
+// Warps 13 and 17 stay idle: a warp's scheduler is warp % 4, and the MMA-issuing warp (1) then
+// shares its scheduler with two epilogue warps only instead of two epilogue and two expander warps.
+constexpr int G_THREADS = 64 + 64 * G_EW + 64;
 constexpr int G_EXP_THREADS = 32 * G_EW;
 constexpr int G_EXP_ROWS = 3;                 // rows of a unit one expander thread loads together
 constexpr int G_EPI_PITCH = 128;
@@ -447,12 +449,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         if (++acc_slot == 2) { acc_slot = 0; acc_phase ^= 1u; }
       }
     }
-  } else {
-    // ------------------------------------------------ expanders (warps 10-17)
+  } else if (warp != 13 && warp != 17) {
+    // ------------------------------------------------ expanders (warps 10-12, 14-16, 18, 19)
     // Fill activation unit (problem, tile, channel block) of the ring: for every plane, row and
     // 32-channel word, bits -> two 16-byte chunks of +1/-1 bytes (fp16: copy two 8-channel chunks).
     grid_dep_wait();  // the activations may come from the previous kernel in the stream
-    const int et = tid - (2 + G_EW) * 32;
+    const int et = (warp - 10 - (warp > 13) - (warp > 17)) * 32 + lane;  // rank among the expander threads
     int a_slot = 0;
     long long a_done = 0;
     uint32_t a_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
