@@ -176,8 +176,8 @@ def run_reference(args):
 # the kernel's sources are the ones that were profiled: {kernel: (workload, batch, bytes, sha256 of sources)}
 _TRAFFIC = {
     # profiles/dram_traffic_resnet18_stack_n64_grouped.txt: mean of the two timed launches
-    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 351402368,
-                                             "7fb4a602e3743c3212870728dfb3ccfb5a32ff1cc62aaa6a9abd674279ef12bb"),
+    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 349305983,
+                                             "0e08eb199b958cbe311673880df7b3b68f769f8ee9da08d0c1c1cc31798e4451"),
 }
 
 
