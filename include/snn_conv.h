@@ -53,7 +53,14 @@ typedef enum {
 } snn_status_t;
 
 enum { SNN_ACT_BIN = 0, SNN_ACT_F16 = 1 };
-enum { SNN_OUT_F32 = 0, SNN_OUT_I32 = 1 }; /* I32 only with SNN_ACT_BIN */
+enum {
+  SNN_OUT_F32 = 0,
+  SNN_OUT_I32 = 1,  /* only with SNN_ACT_BIN */
+  SNN_OUT_BITS = 2  /* only with SNN_ACT_BIN and snn_conv_group_forward: the signs of Y, packed as the next
+                       layer's binary input (Algorithm 1: layer i consumes sign(a^{i-1})):
+                       uint32 [N][Ho][Wo][ceil(c_out/32)], bit co%32 of word co/32 = 1 iff Y >= 0
+                       (so S = 0 gives +1), unused high bits 0 */
+};
 enum {
   SNN_PATH_AUTO = 0,       /* tuned choice if snn_conv_tune ran for the shape, else a heuristic */
   SNN_PATH_REUSE = 1,      /* codebook-reuse: per-channel partial maps + index-driven accumulate (Sec. 4.5) */
@@ -158,9 +165,10 @@ SNN_API snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate);
  *
  * snn_conv_group_forward: act_dev[i] / out_dev[i] are HOST arrays of `count`
  * DEVICE pointers with the layouts and alignment of snn_conv_forward; outputs of
- * different members must not overlap.  Asynchronous on cuda_stream; allocates
- * nothing.  Errors: INVALID_ARG, TIMEOUT (an earlier launch of the group gave up
- * a bounded wait), CUDA.
+ * different members must not overlap.  out_type SNN_OUT_BITS writes the packed
+ * signs instead (1 bit per output instead of 32; out_dev[i] 16-byte aligned as
+ * well).  Asynchronous on cuda_stream; allocates nothing.  Errors: INVALID_ARG,
+ * TIMEOUT (an earlier launch of the group gave up a bounded wait), CUDA.
  */
 #define SNN_GROUP_MAX 32
 typedef struct snn_conv_group snn_conv_group_t; /* opaque; owned by the library */

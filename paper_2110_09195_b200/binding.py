@@ -13,7 +13,7 @@ from pathlib import Path
 import numpy as np
 
 ACT_BIN, ACT_F16 = 0, 1
-OUT_F32, OUT_I32 = 0, 1
+OUT_F32, OUT_I32, OUT_BITS = 0, 1, 2
 PATH_AUTO, PATH_REUSE, PATH_DECODED, PATH_DECODED_TC = 0, 1, 2, 3
 PATH_NAMES = {PATH_AUTO: "auto", PATH_REUSE: "reuse", PATH_DECODED: "decoded", PATH_DECODED_TC: "decoded_tc"}
 _STATUS = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "CUDA", 4: "OOM", 5: "TIMEOUT"}
@@ -209,8 +209,9 @@ class SnnConv:
         else:
             ho, wo = self.out_hw(h, w)
             want = torch.float32 if out_type == OUT_F32 else torch.int32
+            last = (self.c_out + 31) // 32 if out_type == OUT_BITS else self.c_out
             if (not out.is_cuda or out.device.index != self.device or out.dtype != want or not out.is_contiguous()
-                    or tuple(out.shape) != (n, ho, wo, self.c_out)):
+                    or tuple(out.shape) != (n, ho, wo, last)):
                 raise SnnError(1, "output tensor has the wrong device, dtype, shape or layout")
         if stream is None:
             stream = torch.cuda.current_stream(self.device)
@@ -286,6 +287,10 @@ class SnnConvGroup:
         self.device = self.layers[0].device
 
     def alloc_outs(self, out_type=OUT_F32):
+        import torch
+        if out_type == OUT_BITS:   # packed signs: the next layer's binary activation layout
+            return [torch.empty((n, *l.out_hw(h, w), (l.c_out + 31) // 32), dtype=torch.int32,
+                                device=f"cuda:{self.device}") for l, (n, h, w) in zip(self.layers, self.shapes)]
         return [l.alloc_out(n, h, w, out_type) for l, (n, h, w) in zip(self.layers, self.shapes)]
 
     def forward(self, acts, outs=None, out_type=OUT_F32, stream=None):
@@ -299,6 +304,7 @@ class SnnConvGroup:
             outs = self.alloc_outs(out_type)
         want = torch.float32 if out_type == OUT_F32 else torch.int32
         for l, (nb, h, w), a, o in zip(self.layers, self.shapes, acts, outs):
+            last = (l.c_out + 31) // 32 if out_type == OUT_BITS else l.c_out
             if not a.is_cuda or a.device.index != self.device:
                 raise SnnError(1, f"activations must live on cuda:{self.device}")
             l._check_act(a)
@@ -306,7 +312,7 @@ class SnnConvGroup:
             if tuple(a.shape[:3]) != (nb, h, w):
                 raise SnnError(1, "activation tensor does not have the shape the group was created for")
             if (not o.is_cuda or o.device.index != self.device or o.dtype != want or not o.is_contiguous()
-                    or tuple(o.shape) != (nb, ho, wo, l.c_out)):
+                    or tuple(o.shape) != (nb, ho, wo, last)):
                 raise SnnError(1, "output tensor has the wrong device, dtype, shape or layout")
         if stream is None:
             stream = torch.cuda.current_stream(self.device)

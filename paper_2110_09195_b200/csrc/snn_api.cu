@@ -143,6 +143,8 @@ snn_status_t run_path(snn_conv* h, int path, const Geom& g, const Launch& l, int
 snn_status_t check_forward_args(snn_conv* h, const void* act, int N, int H, int W, void* out, int out_type, int path,
                                 Geom* g, int* chosen) {
   if (!h) return fail(SNN_ERR_INVALID_ARG, "null handle");
+  if (out_type == SNN_OUT_BITS)
+    return fail(SNN_ERR_UNSUPPORTED, "packed-sign output is produced by snn_conv_group_forward (a group of one serves a single layer)");
   if (out_type != SNN_OUT_F32 && out_type != SNN_OUT_I32) return fail(SNN_ERR_INVALID_ARG, "bad out_type %d", out_type);
   if (out_type == SNN_OUT_I32 && h->act_type != SNN_ACT_BIN)
     return fail(SNN_ERR_INVALID_ARG, "int32 output needs binary activations");
@@ -493,9 +495,10 @@ snn_status_t snn_conv_group_forward(snn_conv_group_t* g, const void* const* act_
                                     int32_t out_type, void* cuda_stream) {
   if (!g || !g->G) return fail(SNN_ERR_INVALID_ARG, "null group");
   if (!act_dev || !out_dev) return fail(SNN_ERR_INVALID_ARG, "null pointer array");
-  if (out_type != SNN_OUT_F32 && out_type != SNN_OUT_I32) return fail(SNN_ERR_INVALID_ARG, "unknown output type %d", out_type);
-  if (out_type == SNN_OUT_I32 && g->act_type != SNN_ACT_BIN)
-    return fail(SNN_ERR_INVALID_ARG, "int32 output needs binary activations");
+  if (out_type != SNN_OUT_F32 && out_type != SNN_OUT_I32 && out_type != SNN_OUT_BITS)
+    return fail(SNN_ERR_INVALID_ARG, "unknown output type %d", out_type);
+  if (out_type != SNN_OUT_F32 && g->act_type != SNN_ACT_BIN)
+    return fail(SNN_ERR_INVALID_ARG, "int32 and packed-sign outputs need binary activations");
   for (int i = 0; i < g->count; ++i) {
     if (!act_dev[i] || !out_dev[i]) return fail(SNN_ERR_INVALID_ARG, "member %d: null device pointer", i);
     if (((uintptr_t)act_dev[i] & 15) || ((uintptr_t)out_dev[i] & 15))
@@ -509,7 +512,7 @@ snn_status_t snn_conv_group_forward(snn_conv_group_t* g, const void* const* act_
     return fail(SNN_ERR_TIMEOUT, "an earlier launch of the group gave up a bounded wait (code %d)", code);
   }
   int launched = 0;
-  cudaError_t e = tcg_forward(g->G, act_dev, out_dev, out_type == SNN_OUT_I32, (cudaStream_t)cuda_stream, g->status_dev,
+  cudaError_t e = tcg_forward(g->G, act_dev, out_dev, out_type, (cudaStream_t)cuda_stream, g->status_dev,
                               &launched);
   g_launches += launched;
   if (e != cudaSuccess) return cuda_fail(e, "snn_conv_group_forward");

@@ -72,7 +72,7 @@ struct GParams {
   const void* act[SNN_GROUP_MAX];
   void* out[SNN_GROUP_MAX];
   int* status;
-  int out_i32;
+  int out_i32;            // 0: fp32 alpha*S, 1: int32 S, 2: packed signs of alpha*S
   int NA, NS;
   uint32_t a_slot_bytes, b_slot_bytes;
   uint32_t off_b, off_epi, off_pix, off_lay, off_tail;
@@ -364,7 +364,64 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           const bool valid = ((long long)q < L.Qtot) && ((int)n < L.N) && (y < L.Ho) && (x < L.Wo);
           return valid ? ((int)n * L.Ho + y) * L.Wo + x : -1;
         };
-        if (fast) {
+        if (p.out_i32 == 2) {
+          // Packed signs of the scaled output (Algorithm 1: the next layer consumes sign(a)): a thread
+          // owns one position and the 32 (or 16) consecutive channels of a slice, i.e. one word (or
+          // half-word) of the next layer's binary input.  No transposition, one small store per slice.
+          const int Kw = (K + 31) >> 5;
+          if ((Nt & 31) == 0) {
+            const int per_mt = (Nt - 32 * half + 63) / 64;
+#pragma unroll 1
+            for (int mt = 0; mt < MT; ++mt) {
+              const int pix = row_pixel(mt);
+#pragma unroll 1
+              for (int ci = 0; ci < per_mt; ++ci) {
+                const int c0 = 32 * half + 64 * ci, co0 = n0 + c0;
+                uint32_t v[32];
+                __syncwarp();  // the load is a warp-wide instruction: no lane may still be in the store below
+                tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * Nt + c0), v);
+                tmem_ld_wait();
+                if (pix >= 0 && co0 < K) {
+                  uint32_t word = 0;
+#pragma unroll
+                  for (int e = 0; e < 32; ++e) {
+                    const float a = co0 + e < K ? __ldg(alpha + co0 + e) : -1.f;  // a missing channel gives bit 0 ...
+                    const float s = co0 + e < K ? small_int_to_float(v[e]) : 1.f;  // ... through 1 * -1 < 0
+                    word |= (__fmul_rn(s, a) >= 0.f ? 1u : 0u) << e;
+                  }
+                  out32[wide_mul((uint32_t)pix, (uint32_t)Kw) + (uint32_t)(co0 >> 5)] = word;
+                }
+              }
+            }
+          } else {
+            // one channel tile whose width is an odd multiple of 16: half-words; the slice that ends
+            // the tile also clears the half-word behind it, so that every word is written in full
+            uint16_t* out16 = reinterpret_cast<uint16_t*>(out32);
+#pragma unroll 1
+            for (int mt = 0; mt < MT; ++mt) {
+              const int pix = row_pixel(mt);
+              for (int c0 = 16 * half; c0 < Nt; c0 += 32) {
+                uint32_t v[16];
+                __syncwarp();
+                tmem_ld16(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * Nt + c0), v);
+                tmem_ld_wait();
+                const int co0 = n0 + c0;
+                if (pix >= 0) {
+                  uint32_t hw = 0;
+#pragma unroll
+                  for (int e = 0; e < 16; ++e) {
+                    const float a = co0 + e < K ? __ldg(alpha + co0 + e) : -1.f;
+                    const float s = co0 + e < K ? small_int_to_float(v[e]) : 1.f;
+                    hw |= (__fmul_rn(s, a) >= 0.f ? 1u : 0u) << e;
+                  }
+                  const size_t at = wide_mul((uint32_t)pix, (uint32_t)(2 * Kw)) + (uint32_t)(co0 >> 4);
+                  if ((co0 >> 4) < 2 * Kw) out16[at] = (uint16_t)hw;
+                  if (c0 + 16 >= Nt && (co0 >> 4) + 1 < 2 * Kw) out16[at + 1] = 0;
+                }
+              }
+            }
+          }
+        } else if (fast) {
           // The warp's slices (sub-tile mt, columns c0..c0+31) form one sequence; the TMEM load of
           // slice s+1 is issued as soon as slice s sits in the staging tile.
           const int per_mt = (Nt - 32 * half + 63) / 64;

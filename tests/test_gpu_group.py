@@ -157,3 +157,81 @@ def test_group_argument_errors(snn):
     g.destroy()
     a.destroy()
     b.destroy()
+
+
+def _pack_signs(y):
+    """Oracle-side packing of sign(Y) (Y >= 0 -> bit 1) along c_out into little-endian uint32 words."""
+    bits = (y >= 0)
+    n, h, w, k = bits.shape
+    kw = (k + 31) // 32
+    pad = np.zeros((n, h, w, kw * 32), dtype=np.uint64)
+    pad[..., :k] = bits
+    weights = (np.uint64(1) << np.arange(32, dtype=np.uint64))
+    return (pad.reshape(n, h, w, kw, 32) * weights).sum(axis=-1).astype(np.uint32)
+
+
+def test_group_packed_sign_outputs(snn, oracle_mod):
+    """SNN_OUT_BITS: the signs of alpha*S packed as the next layer's input, bit-exact against the
+    oracle's outputs; channel counts that are not multiples of 32 or 16, several channel tiles,
+    negative scales and exact zeros (an all-zero... S = 0 must give bit 1)."""
+    members = [
+        (wl.LayerShape(33, 7, 9, 11, 1, 1), 3),
+        (wl.LayerShape(70, 37, 13, 6, 2, 1), 2),
+        (wl.LayerShape(64, 48, 5, 8, 1, 0), 2),
+        (wl.LayerShape(96, 130, 3, 17, 1, 1), 1),
+        (wl.LayerShape(40, 300, 6, 5, 1, 1), 2),
+        (wl.LayerShape(64, 64, 20, 20, 1, 1), 4),
+        (wl.LayerShape(128, 256, 12, 12, 2, 1), 3),
+        (wl.LayerShape(64, 512, 7, 7, 1, 1), 3),
+        (wl.LayerShape(2, 40, 6, 6, 1, 1), 2),     # tiny c_in: many sums are exactly 0
+    ]
+    layers, acts, refs = [], [], []
+    for i, (shape, n) in enumerate(members):
+        p = wl.draw_layer_params(shape, 5, 61 + i)
+        alpha = p.alpha.copy()
+        alpha[::3] *= -1.0                         # negative scales flip the sign
+        packed = wl.pack_activation_bits(wl.draw_activation_bits(shape, n, 61 + i))
+        _, y_ref = oracle_mod.conv_bin(p.codebook, 5, p.idx_packed, alpha, shape.c_in, shape.c_out, shape.stride,
+                                       shape.pad, packed)
+        refs.append(_pack_signs(y_ref))
+        layers.append(snn.SnnConv(shape.c_in, shape.c_out, 5, p.codebook, p.idx_packed, alpha, shape.stride,
+                                  shape.pad, snn.ACT_BIN))
+        acts.append(torch.from_numpy(packed.view(np.int32)).cuda())
+    group = snn.SnnConvGroup(layers, [(n, s.h, s.w) for s, n in members])
+    guarded = [_guarded(r.shape, torch.int32) for r in refs]
+    group.forward(acts, [g[1] for g in guarded], snn.OUT_BITS)
+    torch.cuda.synchronize()
+    for i, ref in enumerate(refs):
+        got = guarded[i][1].cpu().numpy().view(np.uint32)
+        assert _intact(guarded[i][0], ref.size), f"member {i}: canary overwritten"
+        bad = np.argwhere(got != ref)
+        assert bad.size == 0, f"member {i} {members[i][0]}: {len(bad)} words differ, first at {bad[0]}: " \
+                              f"{got[tuple(bad[0])]:#x} vs {ref[tuple(bad[0])]:#x}"
+    group.destroy()
+    for l in layers:
+        l.destroy()
+
+
+def test_chained_layers_through_packed_signs(snn, oracle_mod):
+    """Two layers chained on the GPU (layer 1 writes packed signs, layer 2 reads them as its binary
+    input) against the same chain through the oracle."""
+    s1, s2, n = wl.LayerShape(64, 96, 14, 14, 1, 1), wl.LayerShape(96, 128, 14, 14, 2, 1), 3
+    p1, p2 = wl.draw_layer_params(s1, 5, 71), wl.draw_layer_params(s2, 5, 72)
+    packed = wl.pack_activation_bits(wl.draw_activation_bits(s1, n, 71))
+    _, y1 = oracle_mod.conv_bin(p1.codebook, 5, p1.idx_packed, p1.alpha, 64, 96, 1, 1, packed)
+    mid_ref = _pack_signs(y1)
+    s_ref, y_ref = oracle_mod.conv_bin(p2.codebook, 5, p2.idx_packed, p2.alpha, 96, 128, 2, 1, mid_ref)
+    l1 = snn.SnnConv(64, 96, 5, p1.codebook, p1.idx_packed, p1.alpha, 1, 1, snn.ACT_BIN)
+    l2 = snn.SnnConv(96, 128, 5, p2.codebook, p2.idx_packed, p2.alpha, 2, 1, snn.ACT_BIN)
+    g1 = snn.SnnConvGroup([l1], [(n, 14, 14)])
+    mid = g1.forward([torch.from_numpy(packed.view(np.int32)).cuda()], out_type=snn.OUT_BITS)[0]
+    out = l2.forward(mid, out_type=snn.OUT_F32)
+    torch.cuda.synchronize()
+    assert (mid.cpu().numpy().view(np.uint32) == mid_ref).all()
+    assert (out.cpu().numpy() == y_ref).all()
+    with pytest.raises(snn.SnnError) as ei:       # the single-layer entry point does not produce packed signs
+        l1.forward(torch.from_numpy(packed.view(np.int32)).cuda(), out=mid, out_type=snn.OUT_BITS)
+    assert ei.value.status == 2
+    g1.destroy()
+    l1.destroy()
+    l2.destroy()
