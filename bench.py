@@ -397,6 +397,22 @@ def run_ours(args):
             e1.record(stream)
             e1.synchronize()
             layer_ms[j] += e0.elapsed_time(e1) / reps
+    # the same grouped step writing packed signs (1 bit per output: the next layer's input) instead of fp32
+    bits_ms = None
+    if group is not None and workload.act == "bin":
+        bit_outs = group.alloc_outs(snn.OUT_BITS)
+        k = max(3, min(30, args.steps))
+        ev3 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(k)]
+        for i in range(k + 3):
+            flush.zero_()
+            if i >= 3:
+                ev3[i - 3][0].record(stream)
+            group.forward(acts, bit_outs, snn.OUT_BITS, stream)
+            if i >= 3:
+                ev3[i - 3][1].record(stream)
+        torch.cuda.synchronize(dev)
+        bits_ms = float(sum(a.elapsed_time(b) for a, b in ev3)) / k
+        del bit_outs
     clocks = sampler.stop()
 
     # end to end through the host-buffer entry point: H2D of the inputs and D2H of the results inside the timing
@@ -412,6 +428,26 @@ def run_ours(args):
     e2e_ms = (time.perf_counter() - t0) / e2e_steps * 1e3
     h2d = sum(a.numel() * a.element_size() for a in host_acts)
     d2h = sum(o.numel() * o.element_size() for o in host_outs)
+
+    # Write-only HBM rate, measured here: the path writes 29 bytes for every byte it reads (fp32 outputs
+    # against packed inputs), and a fill runs well below the copy rate that MEASURED_PEAKS.json holds
+    # (a copy's traffic is half reads).  Reported beside the roofline as context.
+    write_gbs = None
+    try:
+        big = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+        best = None
+        for _ in range(6):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            big.fill_(1)
+            e1.record(stream)
+            e1.synchronize()
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None or ms < best else best
+        write_gbs = big.numel() / (best * 1e-3) / 1e9
+        del big
+    except Exception:
+        write_gbs = None
 
     # max over ranks of the device-timed totals; every rank ran a batch of its own (weak scaling)
     total_ms, e2e_ms = replicas.max_over_ranks([total_ms, e2e_ms], world, dev)
@@ -473,6 +509,8 @@ def run_ours(args):
                      "share_of_step": 1.0 if group is not None else d["ms"] / max(sum(layer_ms), 1e-9),
                      "peak_source": peaks["source"],
                      "algorithmic_bytes_per_launch": d["bytes"] / d["launches"],
+                     "hbm_write_only_gbs": write_gbs,
+                     "frac_of_write_only_rate": None if not write_gbs else d["bytes"] / sec / 1e9 / write_gbs,
                      "algorithmic_ops_per_launch": 2 * d["macs"] / d["launches"],
                      "hbm_frac": hbm_frac, "pipe_frac": pipe["frac"], **alu_rates})
     # whole-step roofline: sum over layers of max(HBM floor, pipe floor at the path's peak)
@@ -498,6 +536,10 @@ def run_ours(args):
         "per_layer_launches": None if seq_ms is None else {
             "ms_per_step": seq_ms, "value": nb / (seq_ms * 1e-3), "unit": UNIT + " per GPU",
             "what": "the same step as one snn_conv_forward launch per layer, back to back on one stream"},
+        "packed_sign_outputs": None if bits_ms is None else {
+            "ms_per_step": bits_ms, "value": nb / (bits_ms * 1e-3), "unit": UNIT + " per GPU",
+            "what": "the grouped step with SNN_OUT_BITS (signs of the outputs packed as the next layer's input) "
+                    "instead of fp32 outputs; host launches, not a graph"},
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms},

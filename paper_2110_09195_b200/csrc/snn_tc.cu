@@ -416,10 +416,8 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 8 ? 1 : 2) tc_conv_kerne
             if (!p.out_i32) {
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                u[i].x = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].x) : small_int_to_float(u[i].x), al.x));
-                u[i].y = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].y) : small_int_to_float(u[i].y), al.y));
-                u[i].z = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].z) : small_int_to_float(u[i].z), al.z));
-                u[i].w = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(u[i].w) : small_int_to_float(u[i].w), al.w));
+                scale_pair<F16>(u[i].x, u[i].y, al.x, al.y);
+                scale_pair<F16>(u[i].z, u[i].w, al.z, al.w);
               }
             }
             uint32_t* obase32 = reinterpret_cast<uint32_t*>(p.out) + co;  // int32 and fp32 outputs share the layout

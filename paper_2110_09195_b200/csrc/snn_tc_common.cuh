@@ -211,6 +211,25 @@ __device__ __forceinline__ void expand_word(uint32_t bits, int channels_left, bo
 __device__ __forceinline__ float small_int_to_float(uint32_t s) {
   return __fadd_rn(__uint_as_float(0x4B400000u + s), -12582912.0f);
 }
+// Two accumulators -> two scaled outputs with the packed fp32 instructions (one add and one
+// multiply for the pair; each lane rounds exactly as the scalar instruction does):
+// F16 = false: a, b hold int32 sums (|s| < 2^22) and become (float)s * alpha; F16 = true: they
+// hold fp32 sums and become sum * alpha.
+template <bool F16>
+__device__ __forceinline__ void scale_pair(uint32_t& a, uint32_t& b, float ax, float ay) {
+  unsigned long long v, m;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(m) : "f"(ax), "f"(ay));
+  if (F16) {
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "r"(a), "r"(b));
+  } else {
+    unsigned long long c;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "r"(0x4B400000u + a), "r"(0x4B400000u + b));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(c) : "f"(-12582912.0f));
+    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(v) : "l"(c));
+  }
+  asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(v) : "l"(m));
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+}
 // 32 x 32 -> 64-bit product in one instruction (element offsets of pixels: both factors are non-negative 32-bit)
 __device__ __forceinline__ size_t wide_mul(uint32_t a, uint32_t b) { return (size_t)a * (size_t)b; }
 
