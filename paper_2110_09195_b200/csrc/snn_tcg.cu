@@ -537,9 +537,13 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         // Input pixel of every staged row, once per tile.  The table is private to the expanders:
         // the barrier keeps a fast thread from overwriting entries another still reads.
         asm volatile("bar.sync 3, %0;" ::"n"(G_EXP_THREADS) : "memory");
-        for (int pl = 0; pl < n_planes; ++pl)
-          for (int r = et; r < Rr; r += G_EXP_THREADS)
-            pix_tab[pl * Rr + r] = g_position_to_pixel(L, Q0 + (uint32_t)r, pl >> 1, pl & 1);
+        // (plane, row) pairs form one index space f = plane*Rr + row, dealt to the threads at a stride of
+        // the expander count, here and below: a thread reads back only entries it wrote itself
+        const int all_rows = n_planes * Rr;
+        for (int f = et; f < all_rows; f += G_EXP_THREADS) {
+          const int pl = (f >= Rr) + (f >= 2 * Rr) + (f >= 3 * Rr);
+          pix_tab[f] = g_position_to_pixel(L, Q0 + (uint32_t)(f - pl * Rr), pl >> 1, pl & 1);
+        }
         for (int cb = 0; cb < n_cb; ++cb) {
           if (a_done >= NA) {
             // one elected thread polls; the rest wait on a hardware barrier instead of spinning
@@ -557,14 +561,18 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
             }
           }
           uint8_t* unit = a_smem + (size_t)a_slot * p.a_slot_bytes;
-          for (int pl = 0; pl < n_planes; ++pl) {
-            uint8_t* plane = unit + (size_t)pl * cb_chunks * Rr * 16;
-            for (int rb = 0; rb < Rr; rb += G_EXP_ROWS * G_EXP_THREADS) {
+          // A thread has rows of several planes in flight together: a stride-2 unit (four short
+          // planes) costs one round trip to memory instead of four.
+          {
+            for (int rb = 0; rb < all_rows; rb += G_EXP_ROWS * G_EXP_THREADS) {
               int pix[G_EXP_ROWS];  // input pixel of each of this thread's rows; -1 padding, -2 past the unit
+              uint8_t* dst[G_EXP_ROWS];  // where the row starts in its plane (chunk 0)
 #pragma unroll
               for (int j = 0; j < G_EXP_ROWS; ++j) {
-                const int r = rb + et + j * G_EXP_THREADS;
-                pix[j] = r < Rr ? pix_tab[pl * Rr + r] : -2;
+                const int f = rb + et + j * G_EXP_THREADS;
+                pix[j] = f < all_rows ? pix_tab[f] : -2;
+                const int pl = (f >= Rr) + (f >= 2 * Rr) + (f >= 3 * Rr);
+                dst[j] = unit + ((size_t)pl * cb_chunks * Rr + (size_t)(f - pl * Rr)) * 16;
               }
               if (F16) {
                 for (int c0 = 0; c0 < cb_chunks; c0 += 2) {
@@ -591,10 +599,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
                   }
 #pragma unroll
                   for (int j = 0; j < G_EXP_ROWS; ++j) {
-                    const int r = rb + et + j * G_EXP_THREADS;
                     if (pix[j] != -2) {
-                      *reinterpret_cast<uint4*>(plane + ((size_t)c0 * Rr + r) * 16) = v[j][0];
-                      *reinterpret_cast<uint4*>(plane + ((size_t)(c0 + 1) * Rr + r) * 16) = v[j][1];
+                      *reinterpret_cast<uint4*>(dst[j] + (size_t)c0 * Rr * 16) = v[j][0];
+                      *reinterpret_cast<uint4*>(dst[j] + (size_t)(c0 + 1) * Rr * 16) = v[j][1];
                     }
                   }
                 }
@@ -622,15 +629,14 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
                 }
 #pragma unroll
                 for (int j = 0; j < G_EXP_ROWS; ++j) {
-                  const int r = rb + et + j * G_EXP_THREADS;
                   if (pix[j] != -2) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                       if (k < nstep) {
                         uint4 lo, hi;
                         expand_word(bits[j][k], C - (w0 + k) * 32, pix[j] >= 0 && w0 + k < Cw, lo, hi);
-                        *reinterpret_cast<uint4*>(plane + ((size_t)(2 * k) * Rr + r) * 16) = lo;
-                        *reinterpret_cast<uint4*>(plane + ((size_t)(2 * k + 1) * Rr + r) * 16) = hi;
+                        *reinterpret_cast<uint4*>(dst[j] + (size_t)(2 * k) * Rr * 16) = lo;
+                        *reinterpret_cast<uint4*>(dst[j] + (size_t)(2 * k + 1) * Rr * 16) = hi;
                       }
                     }
                   }
