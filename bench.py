@@ -176,8 +176,8 @@ def run_reference(args):
 # the kernel's sources are the ones that were profiled: {kernel: (workload, batch, bytes, sha256 of sources)}
 _TRAFFIC = {
     # profiles/dram_traffic_resnet18_stack_n64_grouped.txt: mean of the two timed launches
-    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 348289024,
-                                             "d78e18098601ca57e65a79537185c13c31664b4332ce9867457277a0c96f18f1"),
+    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 349819776,
+                                             "7006c0db14225a5fdd0875976e9318067d0df48328fb67dc8bc6d44e5f121e33"),
 }
 
 

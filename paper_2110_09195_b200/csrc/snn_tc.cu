@@ -179,9 +179,12 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 8 ? 1 : 2) tc_conv_kerne
     // the wait for the previous kernel.  A thread reads back only entries it wrote itself.
     const int et0 = tid - (2 + EPI_WARPS) * 32;
     const uint32_t Q00 = (uint32_t)((int)blockIdx.x / p.n_ntiles) * (uint32_t)(128 * MT);
-    for (int pl = 0; pl < p.n_planes; ++pl)
-      for (int r = et0; r < p.Rr; r += EXP_THREADS)
-        pix_tab[pl * p.Rr + r] = position_to_pixel(p, Q00 + (uint32_t)r, pl >> 1, pl & 1);
+    // (plane, row) pairs form one index space f = plane*Rr + row, dealt to the threads at a stride of
+    // the expander count, here and in the expanders' loops
+    for (int f = et0; f < p.n_planes * p.Rr; f += EXP_THREADS) {
+      const int pl = (f >= p.Rr) + (f >= 2 * p.Rr) + (f >= 3 * p.Rr);
+      pix_tab[f] = position_to_pixel(p, Q00 + (uint32_t)(f - pl * p.Rr), pl >> 1, pl & 1);
+    }
   }
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   tc_fence_before();
@@ -467,9 +470,10 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 8 ? 1 : 2) tc_conv_kerne
       bool stop = false;
       // input pixel of every staged row, once per tile (the first tile's table was made during set-up)
       if (tile != (int)blockIdx.x)
-        for (int pl = 0; pl < p.n_planes; ++pl)
-          for (int r = et; r < p.Rr; r += EXP_THREADS)
-            pix_tab[pl * p.Rr + r] = position_to_pixel(p, Q0 + (uint32_t)r, pl >> 1, pl & 1);
+        for (int f = et; f < p.n_planes * p.Rr; f += EXP_THREADS) {
+          const int pl = (f >= p.Rr) + (f >= 2 * p.Rr) + (f >= 3 * p.Rr);
+          pix_tab[f] = position_to_pixel(p, Q0 + (uint32_t)(f - pl * p.Rr), pl >> 1, pl & 1);
+        }
       for (int cb = 0; cb < p.n_cb; ++cb) {
         if (a_done >= NA) {
           // one elected thread polls; the rest wait on a hardware barrier instead of spinning
@@ -487,14 +491,19 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 8 ? 1 : 2) tc_conv_kerne
           }
         }
         uint8_t* unit = a_smem + (size_t)a_slot * p.a_unit_bytes;
-        for (int pl = 0; pl < p.n_planes; ++pl) {
-          uint8_t* plane = unit + (size_t)pl * p.cb_chunks * p.Rr * 16;
-          for (int rb = 0; rb < p.Rr; rb += EXP_ROWS * EXP_THREADS) {
+        // A thread has rows of several planes in flight together: a stride-2 unit (four short
+        // planes) costs one round trip to memory instead of four.
+        const int all_rows = p.n_planes * p.Rr;
+        {
+          for (int rb = 0; rb < all_rows; rb += EXP_ROWS * EXP_THREADS) {
             int pix[EXP_ROWS];  // input pixel of each of this thread's rows; -1 padding, -2 past the unit
+            uint8_t* dst[EXP_ROWS];  // where the row starts in its plane (chunk 0)
 #pragma unroll
             for (int j = 0; j < EXP_ROWS; ++j) {
-              const int r = rb + et + j * EXP_THREADS;
-              pix[j] = r < p.Rr ? pix_tab[pl * p.Rr + r] : -2;
+              const int f = rb + et + j * EXP_THREADS;
+              pix[j] = f < all_rows ? pix_tab[f] : -2;
+              const int pl = (f >= p.Rr) + (f >= 2 * p.Rr) + (f >= 3 * p.Rr);
+              dst[j] = unit + ((size_t)pl * p.cb_chunks * p.Rr + (size_t)(f - pl * p.Rr)) * 16;
             }
             if (F16) {
               for (int c0 = 0; c0 < p.cb_chunks; c0 += 2) {
@@ -521,10 +530,9 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 8 ? 1 : 2) tc_conv_kerne
                 }
 #pragma unroll
                 for (int j = 0; j < EXP_ROWS; ++j) {
-                  const int r = rb + et + j * EXP_THREADS;
                   if (pix[j] != -2) {
-                    *reinterpret_cast<uint4*>(plane + ((size_t)c0 * p.Rr + r) * 16) = v[j][0];
-                    *reinterpret_cast<uint4*>(plane + ((size_t)(c0 + 1) * p.Rr + r) * 16) = v[j][1];
+                    *reinterpret_cast<uint4*>(dst[j] + (size_t)c0 * p.Rr * 16) = v[j][0];
+                    *reinterpret_cast<uint4*>(dst[j] + (size_t)(c0 + 1) * p.Rr * 16) = v[j][1];
                   }
                 }
               }
@@ -552,15 +560,14 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 8 ? 1 : 2) tc_conv_kerne
               }
 #pragma unroll
               for (int j = 0; j < EXP_ROWS; ++j) {
-                const int r = rb + et + j * EXP_THREADS;
                 if (pix[j] != -2) {
 #pragma unroll
                   for (int k = 0; k < 4; ++k) {
                     if (k < nstep) {
                       uint4 lo, hi;
                       expand_word(bits[j][k], p.C - (w0 + k) * 32, pix[j] >= 0 && w0 + k < p.Cw, lo, hi);
-                      *reinterpret_cast<uint4*>(plane + ((size_t)(2 * k) * p.Rr + r) * 16) = lo;
-                      *reinterpret_cast<uint4*>(plane + ((size_t)(2 * k + 1) * p.Rr + r) * 16) = hi;
+                      *reinterpret_cast<uint4*>(dst[j] + (size_t)(2 * k) * p.Rr * 16) = lo;
+                      *reinterpret_cast<uint4*>(dst[j] + (size_t)(2 * k + 1) * p.Rr * 16) = hi;
                     }
                   }
                 }
