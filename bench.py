@@ -52,7 +52,7 @@ def _peaks():
 class ClockSampler:
     """Samples SM clock and clock-event reasons through NVML while the timed region runs."""
 
-    def __init__(self, device_index: int, period_s: float = 0.05):
+    def __init__(self, device_index: int, period_s: float = 0.005):
         self.idx, self.period = device_index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
@@ -519,7 +519,10 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int32" if workload.act == "bin" else "f16", "data": "synthetic",
+        # the type the dominant path computes in: int8 operands (+/-1) with int32 accumulation on the tensor
+        # cores, fp16 operands with fp32 accumulation in the fp16-activation variant, int32 on the ALU paths
+        "dtype": ("f16" if workload.act != "bin" else "int8" if dom == snn.PATH_DECODED_TC else "int32"),
+        "data": "synthetic",
         "config": {"workload": _workload_name(workload), "layers": len(layers), "batch_per_gpu": nb,
                    "tau": workload.tau, "l2": "flushed between timed steps (256 MB write)",
                    "launch": ("one grouped launch of all layers (snn_conv_group_forward), " if group is not None else "") +
