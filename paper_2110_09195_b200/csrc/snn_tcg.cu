@@ -16,8 +16,9 @@
 //                                                 channel block, taps outermost)
 //   accumulators      two buffers of 256 tensor-memory columns
 // so slots, barriers and phases simply carry on from one problem to the next.
-// Tiles of problem l are dealt to the CTAs round-robin starting where problem l-1
-// stopped, which keeps the CTAs' total work within one tile of each other.
+// Tiles of a problem are dealt to the CTAs round-robin; which CTAs get a problem's odd
+// tiles is decided on the host from the time the CTAs have been given so far, so that the
+// CTAs end close together.
 //
 //      warp 0        one thread streams weight stages (cp.async.bulk onto mbarriers)
 //      warp 1        one thread issues tcgen05.mma and commits barriers
@@ -27,6 +28,9 @@
 //                    activation ring
 // Every wait is bounded; one that runs out raises a status word the host reads, and
 // the CTA still frees its tensor memory and returns.
+#include <algorithm>
+#include <vector>
+
 #include "snn_tc_common.cuh"
 
 namespace snn {
@@ -62,7 +66,7 @@ struct GLayer {
   int st_ksteps;          // K steps (MMAs per sub-tile) per weight stage; divides 9*kpt
   uint32_t stage_bytes;   // = st_ksteps * 2 * Nt * 16
   int n_ntiles, total_tiles;
-  int tile_off;           // CTA that takes this problem's tile 0
+  const uint16_t* rank;   // [grid] CTA b takes this problem's tiles rank[b], rank[b] + grid, ...
   long long Qtot;
 };
 
@@ -92,9 +96,7 @@ __device__ __forceinline__ int g_position_to_pixel(const GLayer& L, uint32_t q, 
 
 // first tile of problem L for this CTA (tiles then follow at a stride of the grid)
 __device__ __forceinline__ int g_first_tile(const GLayer& L) {
-  int f = (int)blockIdx.x - L.tile_off;
-  if (f < 0) f += (int)gridDim.x;
-  return f;
+  return (int)__ldg(L.rank + blockIdx.x);
 }
 
 // The MMAs of one channel block of one tile: 9 taps x KPT K steps x MT sub-tiles.  The body of
@@ -666,6 +668,7 @@ struct GroupDev {
   int count = 0, act_type = 0;
   GLayer* layers_dev = nullptr;   // [count]
   uint8_t* weights = nullptr;     // the group's own weight operands, one after the other
+  uint16_t* ranks = nullptr;      // [count][grid] tile assignment, see tcg_create
   GParams p{};                    // everything but the per-call pointers
   size_t smem = 0;
   int grid = 0;
@@ -769,10 +772,29 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   if (ns > G_NS_MAX) ns = G_NS_MAX;
   const int sms = sm_count();
   const int grid = tiles < sms ? (int)tiles : sms;
-  int off = 0;
-  for (int i = 0; i < count; ++i) {
-    host[i].tile_off = off;
-    off = (int)(((long long)off + host[i].total_tiles) % grid);
+  // Which CTAs take a problem's odd tiles.  Every CTA gets floor(tiles / grid) tiles of a problem
+  // and the first (tiles % grid) CTAs in the problem's rank order get one more; the rank order is
+  // by the time the CTAs have been given so far, least first, so that the CTAs end close
+  // together although a tile of one problem may take six times as long as a tile of another.
+  // Time of a tile: the larger of its MMAs (73 cycles each up to 128 channels wide, 128 cycles at
+  // 256) and of its fp32 output at the write rate an SM gets (13 bytes per cycle).
+  std::vector<uint16_t> ranks((size_t)count * grid);
+  {
+    std::vector<double> busy(grid, 0.0);
+    std::vector<int> order(grid);
+    for (int i = 0; i < count; ++i) {
+      const GLayer& o = host[i];
+      const double mma = (double)o.MT * o.n_cb * 9 * o.kpt * (o.Nt > 146 ? o.Nt / 2 : 73);
+      const double wr = 128.0 * o.MT * (o.Nt < o.K ? o.Nt : o.K) * 4 / 13.0;
+      const double cost = (mma > wr ? mma : wr) + 300.0;
+      for (int b = 0; b < grid; ++b) order[b] = b;
+      std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return busy[a] < busy[b]; });
+      const int base = o.total_tiles / grid, rem = o.total_tiles % grid;
+      for (int r = 0; r < grid; ++r) {
+        ranks[(size_t)i * grid + order[r]] = (uint16_t)r;
+        busy[order[r]] += cost * (base + (r < rem ? 1 : 0));
+      }
+    }
   }
   GroupDev* G = new GroupDev();
   G->count = count;
@@ -780,7 +802,11 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   G->grid = grid;
   cudaError_t e = cudaMalloc(&G->weights, w_total);
   if (e == cudaSuccess) e = cudaMalloc(&G->layers_dev, sizeof(GLayer) * count);
+  if (e == cudaSuccess) e = cudaMalloc(&G->ranks, ranks.size() * sizeof(uint16_t));
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(G->ranks, ranks.data(), ranks.size() * sizeof(uint16_t), cudaMemcpyHostToDevice, s);
   for (int i = 0; i < count && e == cudaSuccess; ++i) {
+    host[i].rank = G->ranks + (size_t)i * grid;
     host[i].wt = G->weights + w_off[i];
     host[i].alpha = Ls[i]->alpha;
     e = tc_expand_weights_custom(Ls[i]->wplanes, G->weights + w_off[i], gs[i].C, gs[i].K, gs[i].Cw, Kpad[i],
@@ -788,7 +814,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
     if (e == cudaSuccess) *launched += 1;
   }
   if (e == cudaSuccess) e = cudaMemcpyAsync(G->layers_dev, host, sizeof(GLayer) * count, cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaStreamSynchronize(s);  // `host` lives on this stack
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);  // `host` and `ranks` live on this stack
   if (e != cudaSuccess) {
     tcg_destroy(G);
     return e;
@@ -818,6 +844,7 @@ void tcg_destroy(GroupDev* G) {
   if (!G) return;
   cudaFree(G->weights);
   cudaFree(G->layers_dev);
+  cudaFree(G->ranks);
   delete G;
 }
 
