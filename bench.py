@@ -176,8 +176,8 @@ def run_reference(args):
 # the kernel's sources are the ones that were profiled: {kernel: (workload, batch, bytes, sha256 of sources)}
 _TRAFFIC = {
     # profiles/dram_traffic_resnet18_stack_n64_grouped.txt: mean of the two timed launches
-    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 349819776,
-                                             "7006c0db14225a5fdd0875976e9318067d0df48328fb67dc8bc6d44e5f121e33"),
+    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 348673920,
+                                             "80d6d8912c9655fdbe80994caa5981401e87a84a753fdb5afa04400ddc026db3"),
 }
 
 
