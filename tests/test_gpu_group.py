@@ -212,6 +212,32 @@ def test_group_packed_sign_outputs(snn, oracle_mod):
         l.destroy()
 
 
+def test_group_packed_signs_many_tiles_and_repeatable(snn, oracle_mod):
+    """Packed-sign output with more tiles than CTAs (both accumulator buffers, ring wrap-around),
+    twice in a row into fresh buffers: bit-exact against the oracle and identical between runs."""
+    members = [(wl.LayerShape(64, 64, 56, 56, 1, 1), 12), (wl.LayerShape(128, 128, 28, 28, 1, 1), 24),
+               (wl.LayerShape(256, 512, 14, 14, 2, 1), 16)]
+    layers, acts, refs = [], [], []
+    for i, (shape, n) in enumerate(members):
+        p = wl.draw_layer_params(shape, 5, 81 + i)
+        packed = wl.pack_activation_bits(wl.draw_activation_bits(shape, n, 81 + i))
+        _, y_ref = oracle_mod.conv_bin(p.codebook, 5, p.idx_packed, p.alpha, shape.c_in, shape.c_out, shape.stride,
+                                       shape.pad, packed)
+        refs.append(_pack_signs(y_ref))
+        layers.append(snn.SnnConv(shape.c_in, shape.c_out, 5, p.codebook, p.idx_packed, p.alpha, shape.stride,
+                                  shape.pad, snn.ACT_BIN))
+        acts.append(torch.from_numpy(packed.view(np.int32)).cuda())
+    group = snn.SnnConvGroup(layers, [(n, s.h, s.w) for s, n in members])
+    first = [o.cpu().numpy().view(np.uint32) for o in group.forward(acts, out_type=snn.OUT_BITS)]
+    second = [o.cpu().numpy().view(np.uint32) for o in group.forward(acts, out_type=snn.OUT_BITS)]
+    for i, ref in enumerate(refs):
+        assert (first[i] == ref).all(), f"member {i}"
+        assert (second[i] == first[i]).all(), f"member {i}: second run differs"
+    group.destroy()
+    for l in layers:
+        l.destroy()
+
+
 def test_chained_layers_through_packed_signs(snn, oracle_mod):
     """Two layers chained on the GPU (layer 1 writes packed signs, layer 2 reads them as its binary
     input) against the same chain through the oracle."""
