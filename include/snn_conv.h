@@ -56,7 +56,7 @@ enum { SNN_ACT_BIN = 0, SNN_ACT_F16 = 1 };
 enum {
   SNN_OUT_F32 = 0,
   SNN_OUT_I32 = 1,  /* only with SNN_ACT_BIN */
-  SNN_OUT_BITS = 2  /* only with SNN_ACT_BIN and snn_conv_group_forward: the signs of Y, packed as the next
+  SNN_OUT_BITS = 2  /* only with SNN_ACT_BIN and the tensor-core path: the signs of Y, packed as the next
                        layer's binary input (Algorithm 1: layer i consumes sign(a^{i-1})):
                        uint32 [N][Ho][Wo][ceil(c_out/32)], bit co%32 of word co/32 = 1 iff Y >= 0
                        (so S = 0 gives +1), unused high bits 0 */
@@ -94,9 +94,10 @@ SNN_API snn_status_t snn_conv_create(const snn_conv_desc_t* desc, snn_conv_t** o
  * out_dev 16-byte aligned; they are neither kept nor freed.  The call is
  * asynchronous on cuda_stream (a cudaStream_t, NULL = default stream) and does
  * not allocate.  N may be 0 (nothing is launched).
- * Errors: INVALID_ARG (null, H/W giving no output, I32 output with fp16
+ * Errors: INVALID_ARG (null, H/W giving no output, I32 or BITS output with fp16
  * activations, unknown path), UNSUPPORTED (the named path cannot run this
- * layer; AUTO never returns it), CUDA.
+ * layer; AUTO never returns it, except for SNN_OUT_BITS on a layer the
+ * tensor-core path cannot run), CUDA.
  */
 SNN_API snn_status_t snn_conv_forward(snn_conv_t* h, const void* act_dev, int32_t N, int32_t H, int32_t W,
                               void* out_dev, int32_t out_type, int32_t path, void* cuda_stream);

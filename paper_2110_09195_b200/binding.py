@@ -189,11 +189,12 @@ class SnnConv:
         import torch
         ho, wo = self.out_hw(h, w)
         dt = torch.float32 if out_type == OUT_F32 else torch.int32
+        last = (self.c_out + 31) // 32 if out_type == OUT_BITS else self.c_out   # packed signs: 32 channels a word
         if device is None:
             device = f"cuda:{self.device}"
         if pin:
-            return torch.empty((n, ho, wo, self.c_out), dtype=dt, pin_memory=True)
-        return torch.empty((n, ho, wo, self.c_out), dtype=dt, device=device)
+            return torch.empty((n, ho, wo, last), dtype=dt, pin_memory=True)
+        return torch.empty((n, ho, wo, last), dtype=dt, device=device)
 
     # -- the C entry points -------------------------------------------------
     def forward(self, act, out=None, out_type=OUT_F32, path=PATH_AUTO, stream=None):

@@ -143,11 +143,10 @@ snn_status_t run_path(snn_conv* h, int path, const Geom& g, const Launch& l, int
 snn_status_t check_forward_args(snn_conv* h, const void* act, int N, int H, int W, void* out, int out_type, int path,
                                 Geom* g, int* chosen) {
   if (!h) return fail(SNN_ERR_INVALID_ARG, "null handle");
-  if (out_type == SNN_OUT_BITS)
-    return fail(SNN_ERR_UNSUPPORTED, "packed-sign output is produced by snn_conv_group_forward (a group of one serves a single layer)");
-  if (out_type != SNN_OUT_F32 && out_type != SNN_OUT_I32) return fail(SNN_ERR_INVALID_ARG, "bad out_type %d", out_type);
-  if (out_type == SNN_OUT_I32 && h->act_type != SNN_ACT_BIN)
-    return fail(SNN_ERR_INVALID_ARG, "int32 output needs binary activations");
+  if (out_type != SNN_OUT_F32 && out_type != SNN_OUT_I32 && out_type != SNN_OUT_BITS)
+    return fail(SNN_ERR_INVALID_ARG, "bad out_type %d", out_type);
+  if (out_type != SNN_OUT_F32 && h->act_type != SNN_ACT_BIN)
+    return fail(SNN_ERR_INVALID_ARG, "int32 and packed-sign outputs need binary activations");
   if (path < SNN_PATH_AUTO || path > SNN_PATH_DECODED_TC) return fail(SNN_ERR_INVALID_ARG, "unknown path %d", path);
   if (!make_geom(h, N, H, W, g))
     return fail(SNN_ERR_INVALID_ARG, "shape N=%d H=%d W=%d gives no output (pad %d) or is too large", N, H, W, h->pad);
@@ -155,7 +154,14 @@ snn_status_t check_forward_args(snn_conv* h, const void* act, int N, int H, int 
   if (((uintptr_t)act & 15) || ((uintptr_t)out & 15))
     return fail(SNN_ERR_INVALID_ARG, "activation / output pointers must be 16-byte aligned");
   int pth = path;
-  if (pth == SNN_PATH_AUTO) pth = auto_path(h, *g);
+  if (out_type == SNN_OUT_BITS) {
+    // only the tensor-core path writes packed signs
+    if (pth != SNN_PATH_AUTO && pth != SNN_PATH_DECODED_TC)
+      return fail(SNN_ERR_UNSUPPORTED, "packed-sign output is written by the tensor-core path only, not by path %d", pth);
+    pth = SNN_PATH_DECODED_TC;
+    if (!path_ok(h, pth, *g))
+      return fail(SNN_ERR_UNSUPPORTED, "packed-sign output needs the tensor-core path, which cannot run this layer");
+  } else if (pth == SNN_PATH_AUTO) pth = auto_path(h, *g);
   else if (!path_ok(h, pth, *g))
     return fail(SNN_ERR_UNSUPPORTED, "path %d does not support this layer (act_type %d, C=%d K=%d)", pth, h->act_type,
                 h->C, h->K);
@@ -302,7 +308,7 @@ snn_status_t snn_conv_forward(snn_conv_t* h, const void* act_dev, int32_t N, int
     *h->tc_status_host = 0;
     return fail(SNN_ERR_TIMEOUT, "an earlier tensor-core launch gave up a bounded wait (code %d)", code);
   }
-  Launch l{act_dev, out_dev, out_type == SNN_OUT_I32, (cudaStream_t)cuda_stream};
+  Launch l{act_dev, out_dev, out_type, (cudaStream_t)cuda_stream};
   return run_path(h, chosen, g, l);
 }
 
@@ -315,7 +321,8 @@ snn_status_t snn_conv_forward_host(snn_conv_t* h, const void* act_host, int32_t 
   if (!act_host || !out_host) return fail(SNN_ERR_INVALID_ARG, "null host pointer");
   DeviceGuard guard(h->device);
   if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", h->device);
-  const size_t ib = act_bytes(h, g), ob = out_bytes(g);
+  const size_t ib = act_bytes(h, g);
+  const size_t ob = out_type == SNN_OUT_BITS ? (size_t)g.N * g.Ho * g.Wo * ((g.K + 31) / 32) * 4 : out_bytes(g);
   cudaError_t e = cudaSuccess;
   if (ib > h->stage_in_bytes) {
     cudaFree(h->stage_in);

@@ -36,7 +36,7 @@ struct LayerDev {
 struct Launch {
   const void* act;
   void* out;
-  int out_i32;   // 1: write int32 S, 0: write fp32 alpha*S
+  int out_i32;   // 0: write fp32 alpha*S, 1: write int32 S, 2: packed signs of alpha*S (tensor-core path only)
   cudaStream_t stream;
 };
 

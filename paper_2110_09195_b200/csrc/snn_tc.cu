@@ -60,7 +60,7 @@ struct TcParams {
   const float* alpha;
   void* out;
   int* status;            // mapped host word, set on a timed-out wait
-  int out_i32;
+  int out_i32;            // 0: fp32 alpha*S, 1: int32 S, 2: packed signs of alpha*S
   int act_vec;            // the activation rows may be read with 8/16-byte loads
   int N, H, W, C, K, Cw, stride, pad, Ho, Wo;
   int Kpad, n_chunks;     // padded channels out; 16-byte chunks along the padded channels in
@@ -374,7 +374,65 @@ __global__ void __launch_bounds__(tc_threads(EW), EW == 8 ? 1 : 2) tc_conv_kerne
         const bool valid = ((long long)q < p.Qtot) && ((int)n < p.N) && (y < p.Ho) && (x < p.Wo);
         return valid ? ((int)n * p.Ho + y) * p.Wo + x : -1;
       };
-      if (fast) {
+      if (p.out_i32 == 2) {
+        // Packed signs of the scaled output (Algorithm 1: the next layer consumes sign(a)): a thread
+        // owns one position and the 32 (or 16) consecutive channels of a slice, i.e. one word (or
+        // half-word) of the next layer's binary input.  No transposition, one small store per slice.
+        const int Kw = (p.K + 31) >> 5;
+        uint32_t* out32 = reinterpret_cast<uint32_t*>(p.out);
+        if ((p.Nt & 31) == 0) {
+          const int per_mt = (p.Nt - 32 * half + 32 * NH - 1) / (32 * NH);
+#pragma unroll 1
+          for (int mt = 0; mt < MT; ++mt) {
+            const int pix = row_pixel(mt);
+#pragma unroll 1
+            for (int ci = 0; ci < per_mt; ++ci) {
+              const int c0 = 32 * half + 32 * NH * ci, co0 = n0 + c0;
+              uint32_t v[32];
+              __syncwarp();  // the load is a warp-wide instruction: no lane may still be in the store below
+              tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt + c0), v);
+              tmem_ld_wait();
+              if (pix >= 0 && co0 < p.K) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                  const float a = co0 + e < p.K ? __ldg(p.alpha + co0 + e) : -1.f;  // a missing channel gives bit 0 ...
+                  const float s = co0 + e < p.K ? small_int_to_float(v[e]) : 1.f;   // ... through 1 * -1 < 0
+                  word |= (__fmul_rn(s, a) >= 0.f ? 1u : 0u) << e;
+                }
+                out32[wide_mul((uint32_t)pix, (uint32_t)Kw) + (uint32_t)(co0 >> 5)] = word;
+              }
+            }
+          }
+        } else {
+          // one channel tile whose width is an odd multiple of 16: half-words; the slice that ends
+          // the tile also clears the half-word behind it, so that every word is written in full
+          uint16_t* out16 = reinterpret_cast<uint16_t*>(p.out);
+#pragma unroll 1
+          for (int mt = 0; mt < MT; ++mt) {
+            const int pix = row_pixel(mt);
+            for (int c0 = 16 * half; c0 < p.Nt; c0 += 16 * NH) {
+              uint32_t v[16];
+              __syncwarp();
+              tmem_ld16(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * p.Nt + c0), v);
+              tmem_ld_wait();
+              const int co0 = n0 + c0;
+              if (pix >= 0) {
+                uint32_t hw = 0;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                  const float a = co0 + e < p.K ? __ldg(p.alpha + co0 + e) : -1.f;
+                  const float s = co0 + e < p.K ? small_int_to_float(v[e]) : 1.f;
+                  hw |= (__fmul_rn(s, a) >= 0.f ? 1u : 0u) << e;
+                }
+                const size_t at = wide_mul((uint32_t)pix, (uint32_t)(2 * Kw)) + (uint32_t)(co0 >> 4);
+                if ((co0 >> 4) < 2 * Kw) out16[at] = (uint16_t)hw;
+                if (c0 + 16 >= p.Nt && (co0 >> 4) + 1 < 2 * Kw) out16[at + 1] = 0;
+              }
+            }
+          }
+        }
+      } else if (fast) {
         // The warp's slices (sub-tile mt, columns c0..c0+31) form one sequence.  The TMEM load of
         // slice s+1 is issued as soon as slice s sits in the staging tile, so it flies while
         // slice s is converted and stored, and the store path never waits for a TMEM load.
@@ -867,6 +925,7 @@ cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l
     if (forced >= 0 && tc_variant_ok(g, act_type, forced)) variant = forced;
   }
   const int first_half = kPmVariants + cm_variant_count();
+  if (l.out_i32 == 2 && variant >= kPmVariants && variant < first_half) variant = 0;  // packed signs: this kernel only
   if (variant >= kPmVariants && variant < first_half)
     return cm_forward(L, g, act_type, l, launched, status_dev, variant - kPmVariants);
   TcPlan pl = variant >= first_half ? make_plan(g, act_type, variant - first_half, true) : make_plan(g, act_type, variant);

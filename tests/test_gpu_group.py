@@ -255,9 +255,50 @@ def test_chained_layers_through_packed_signs(snn, oracle_mod):
     torch.cuda.synchronize()
     assert (mid.cpu().numpy().view(np.uint32) == mid_ref).all()
     assert (out.cpu().numpy() == y_ref).all()
-    with pytest.raises(snn.SnnError) as ei:       # the single-layer entry point does not produce packed signs
-        l1.forward(torch.from_numpy(packed.view(np.int32)).cuda(), out=mid, out_type=snn.OUT_BITS)
+    # the same chain through the single-layer entry point
+    mid1 = l1.forward(torch.from_numpy(packed.view(np.int32)).cuda(), out_type=snn.OUT_BITS)
+    out1 = l2.forward(mid1, out_type=snn.OUT_I32)
+    torch.cuda.synchronize()
+    assert (mid1.cpu().numpy().view(np.uint32) == mid_ref).all()
+    assert (out1.cpu().numpy() == s_ref).all()
+    with pytest.raises(snn.SnnError) as ei:       # only the tensor-core path writes packed signs
+        l1.forward(torch.from_numpy(packed.view(np.int32)).cuda(), out_type=snn.OUT_BITS, path=snn.PATH_DECODED)
     assert ei.value.status == 2
     g1.destroy()
     l1.destroy()
     l2.destroy()
+
+
+@pytest.mark.parametrize("c_in,c_out,h,w,stride,pad,n", [
+    (33, 7, 9, 11, 1, 1, 3), (70, 37, 13, 6, 2, 1, 2), (64, 48, 5, 8, 1, 0, 2), (96, 130, 3, 17, 1, 1, 1),
+    (40, 300, 6, 5, 1, 1, 2), (64, 64, 56, 56, 1, 1, 6), (128, 256, 12, 12, 2, 1, 3), (512, 512, 7, 7, 1, 1, 8),
+])
+def test_single_layer_packed_sign_outputs(snn, oracle_mod, monkeypatch, c_in, c_out, h, w, stride, pad, n):
+    """SNN_OUT_BITS through snn_conv_forward (tensor-core path: tuned or heuristic full-size tiles, and
+    the half-size CTAs), through snn_conv_forward_host, and after tuning (a tuned channel-major tile
+    must not be used for it): bit-exact against the oracle's outputs."""
+    shape = wl.LayerShape(c_in, c_out, h, w, stride, pad)
+    p = wl.draw_layer_params(shape, 5, 91)
+    alpha = p.alpha.copy()
+    alpha[1::4] *= -1.0
+    packed = wl.pack_activation_bits(wl.draw_activation_bits(shape, n, 91))
+    _, y_ref = oracle_mod.conv_bin(p.codebook, 5, p.idx_packed, alpha, c_in, c_out, stride, pad, packed)
+    ref = _pack_signs(y_ref)
+    layer = snn.SnnConv(c_in, c_out, 5, p.codebook, p.idx_packed, alpha, stride, pad, snn.ACT_BIN)
+    act = torch.from_numpy(packed.view(np.int32)).cuda()
+    for variant in (None, 22, 25, 17):
+        if variant is None:
+            monkeypatch.delenv("SNN_TC_VARIANT", raising=False)
+        else:
+            monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
+        flat, out = _guarded(ref.shape, torch.int32)
+        layer.forward(act, out, snn.OUT_BITS)
+        torch.cuda.synchronize()
+        assert _intact(flat, ref.size), f"variant {variant}: canary overwritten"
+        assert (out.cpu().numpy().view(np.uint32) == ref).all(), f"variant {variant}"
+    monkeypatch.delenv("SNN_TC_VARIANT", raising=False)
+    host = layer.forward_host(torch.from_numpy(packed.view(np.int32)).pin_memory(), out_type=snn.OUT_BITS)
+    assert (host.numpy().view(np.uint32) == ref).all()
+    layer.tune(n, h, w)
+    assert (layer.forward(act, out_type=snn.OUT_BITS).cpu().numpy().view(np.uint32) == ref).all()
+    layer.destroy()
