@@ -413,6 +413,38 @@ def run_ours(args):
         torch.cuda.synchronize(dev)
         bits_ms = float(sum(a.elapsed_time(b) for a, b in ev3)) / k
         del bit_outs
+    # The stack as a true chain: layer i writes packed signs that layer i+1 reads as its binary input
+    # (no batch-norm or shortcut in between: the path has none), one snn_conv_forward launch per layer.
+    chain_ms = None
+    shapes = workload.layers
+    chains = all(a.c_out == b.c_in and ((a.h + 2 * a.pad - 3) // a.stride + 1) == b.h for a, b in zip(shapes, shapes[1:]))
+    if workload.act == "bin" and chains and not args.group_only and forced in (snn.PATH_AUTO, snn.PATH_DECODED_TC):
+        bufs = [layers[j].alloc_out(nb, shapes[j].h, shapes[j].w, snn.OUT_BITS) for j in all_idx]
+
+        def launch_chain(s):
+            x = acts[0]
+            for j in all_idx:
+                layers[j].forward(x, bufs[j], snn.OUT_BITS, snn.PATH_DECODED_TC, s)
+                x = bufs[j]
+
+        gchain = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            launch_chain(side)
+            side.synchronize()
+            with torch.cuda.graph(gchain, stream=side):
+                launch_chain(torch.cuda.current_stream(dev))
+        k = max(3, min(30, args.steps))
+        ev4 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(k)]
+        for i in range(k + 3):
+            flush.zero_()
+            if i >= 3:
+                ev4[i - 3][0].record(stream)
+            gchain.replay()
+            if i >= 3:
+                ev4[i - 3][1].record(stream)
+        torch.cuda.synchronize(dev)
+        chain_ms = float(sum(a.elapsed_time(b) for a, b in ev4)) / k
+        del bufs, gchain
     clocks = sampler.stop()
 
     # end to end through the host-buffer entry point: H2D of the inputs and D2H of the results inside the timing
@@ -543,6 +575,10 @@ def run_ours(args):
             "ms_per_step": bits_ms, "value": nb / (bits_ms * 1e-3), "unit": UNIT + " per GPU",
             "what": "the grouped step with SNN_OUT_BITS (signs of the outputs packed as the next layer's input) "
                     "instead of fp32 outputs; host launches, not a graph"},
+        "chained_packed_signs": None if chain_ms is None else {
+            "ms_per_step": chain_ms, "value": nb / (chain_ms * 1e-3), "unit": UNIT + " per GPU",
+            "what": "the layers as a dependent chain: each layer's packed signs (SNN_OUT_BITS) are the next "
+                    "layer's input, one snn_conv_forward launch per layer, CUDA graph"},
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms},
