@@ -110,7 +110,8 @@ def test_group_many_tiles_per_cta(snn, oracle_mod):
 
 def test_group_fp16(snn, oracle_mod):
     members = [(wl.LayerShape(64, 64, 14, 14, 1, 1), 3), (wl.LayerShape(136, 72, 9, 7, 2, 1), 2),
-               (wl.LayerShape(33, 7, 6, 5, 2, 1), 2), (wl.LayerShape(256, 256, 7, 7, 1, 1), 2)]
+               (wl.LayerShape(33, 7, 6, 5, 2, 1), 2), (wl.LayerShape(256, 256, 7, 7, 1, 1), 2),
+               (wl.LayerShape(64, 64, 56, 56, 1, 1), 10), (wl.LayerShape(128, 256, 28, 28, 2, 1), 24)]  # many tiles per CTA
     layers, acts, refs, alphas = [], [], [], []
     for i, (shape, n) in enumerate(members):
         p = wl.draw_layer_params(shape, 5, 51 + i)
