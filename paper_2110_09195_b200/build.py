@@ -37,6 +37,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     objdir = PKG / "_build"
     objdir.mkdir(exist_ok=True)
     extra = ["-Xptxas", "-v"] if verbose else []
+    extra += os.environ.get("SNN_NVCC_FLAGS", "").split()   # e.g. -DSNN_TRACE (per-role wait counters)
 
     def compile_one(src: str) -> Path:
         obj = objdir / (src + ".o")

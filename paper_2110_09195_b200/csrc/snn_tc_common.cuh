@@ -71,8 +71,21 @@ __device__ __forceinline__ uint32_t mbar_try_hint(uint32_t bar, uint32_t parity,
       : "memory");
   return ok;
 }
+// non-blocking test of the phase: a wait that is already over costs one short instruction
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
 // Bounded wait for the phase with the given parity; false when the limit ran out.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_test(bar, parity)) return true;
   for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
     if (mbar_try_hint(bar, parity, 1000u)) return true;
   return false;
@@ -90,6 +103,15 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
+// Shared -> global bulk copy in this thread's bulk group (16-byte aligned addresses, size a multiple of 16).
+__device__ __forceinline__ void bulk_s2g(const void* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all of this thread's bulk groups have read their shared-memory source
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// all of this thread's bulk groups are complete (their writes done)
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void raise_status(int* status, int code) {
   *reinterpret_cast<volatile int*>(status) = code;
   __threadfence_system();
@@ -144,6 +166,28 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t
   }
 }
 
+// Block-scaled 4-bit MMA (e2m1 operands, one ue8m0 scale per 32 elements along K, fp32 accumulators):
+// D[128 x N] (+)= A[128 x 64] * B[N x 64]^T.  +1, -1 and 0 are exact e2m1 values, unit scales leave the
+// products alone and every partial sum of a 3x3 layer is an integer far below 2^24, so the fp32
+// accumulators hold the exact sums.  sfa / sfb are tensor-memory addresses of the scale factors.
+__device__ __forceinline__ void mma_ss_fp4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t accumulate, uint32_t sfa, uint32_t sfb) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+      : "memory");
+}
+// One 32-bit value into 32 consecutive tensor-memory columns of this warp's 32 lanes.
+__device__ __forceinline__ void tmem_fill32(uint32_t taddr, uint32_t v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,"
+      "%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};" ::"r"(taddr),
+      "r"(v)
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -160,6 +204,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
         "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
         "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+// 16 lanes x 32 columns in the 256-bit shape: with r = lane / 4 and q = lane % 4, register 4j + 2s + e holds
+// row (r + 8s) of the 16, column 8j + 2q + e  (j = 0..3, s = 0..1, e = 0..1).
+__device__ __forceinline__ void tmem_ld16x256(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(taddr)
       : "memory");
 }
@@ -202,6 +256,28 @@ __device__ __forceinline__ void expand_word(uint32_t bits, int channels_left, bo
       hi.w &= nibble_to_mask(vm >> 28);
     }
   }
+}
+
+// 32 activation bits -> 32 e2m1 nibbles (16 bytes): +1.0 is 0x2, -1.0 is 0xA; channel c of the word sits in
+// nibble c (byte c/2, low nibble first).  A byte is looked up from its two bits with a byte permute whose
+// table holds the four nibble pairs; the selectors of 16 channels are made by spreading the bit pairs to
+// nibble positions.  Bits of channels that do not exist may be anything: their weights are zero.
+__device__ __forceinline__ uint32_t spread_pairs16(uint32_t x) {
+  x = (x | (x << 8)) & 0x00ff00ffu;
+  x = (x | (x << 4)) & 0x0f0f0f0fu;
+  x = (x | (x << 2)) & 0x33333333u;
+  return x;
+}
+__device__ __forceinline__ uint4 expand_word_fp4(uint32_t bits, bool present) {
+  if (!present) return make_uint4(0, 0, 0, 0);
+  const uint32_t lut = 0x222aa2aau;  // byte i = nibble pair of the 2-bit value i
+  const uint32_t s0 = spread_pairs16(bits & 0xffffu), s1 = spread_pairs16(bits >> 16);
+  uint4 r;
+  asm("prmt.b32 %0, %1, %1, %2;" : "=r"(r.x) : "r"(lut), "r"(s0));
+  asm("prmt.b32 %0, %1, %1, %2;" : "=r"(r.y) : "r"(lut), "r"(s0 >> 16));
+  asm("prmt.b32 %0, %1, %1, %2;" : "=r"(r.z) : "r"(lut), "r"(s1));
+  asm("prmt.b32 %0, %1, %1, %2;" : "=r"(r.w) : "r"(lut), "r"(s1 >> 16));
+  return r;
 }
 
 // int32 -> float for |s| < 2^22 without the conversion unit (which handles only 16 lanes per SM

@@ -29,6 +29,7 @@
 // Every wait is bounded; one that runs out raises a status word the host reads, and
 // the CTA still frees its tensor memory and returns.
 #include <algorithm>
+#include <cstdio>
 #include <vector>
 
 #include "snn_tc_common.cuh"
@@ -37,6 +38,10 @@ namespace snn {
 
 namespace {
 
+// Operand modes of the kernel.  Binary activations run on 4-bit e2m1 operands (+1 / -1 / 0 are exact, the
+// block scales are all 1, fp32 accumulators hold the exact integer sums): an MMA then covers 64 input
+// channels in the time an int8 MMA covers 32.  The int8 mode is the same contraction with int32 accumulators.
+enum { M_I8 = 0, M_F16 = 1, M_FP4 = 2 };
 constexpr int G_EW = 8;                       // epilogue warps = expander warps
 // Warps 13 and 17 stay idle: a warp's scheduler is warp % 4, and the MMA-issuing warp (1) then
 // shares its scheduler with two epilogue warps only instead of two epilogue and two expander warps.
@@ -47,6 +52,8 @@ constexpr int G_EPI_PITCH = 128;
 constexpr int G_EPI_BYTES = G_EW * 32 * G_EPI_PITCH;
 constexpr int G_NA_MAX = 4, G_NS_MAX = 8;
 constexpr uint32_t G_ACC_COLS = 256;          // tensor-memory columns of one accumulator buffer
+constexpr uint32_t G_ACC_COLS_FP4 = 240;      // 4-bit mode: columns 480..511 hold the (unit) block scales
+constexpr uint32_t G_SCALE_COL = 480;
 constexpr size_t kGTail = 512;
 constexpr size_t kGSmemBudget = 226 * 1024;
 constexpr uint32_t kGASlotMax = 40 * 1024 + 512;   // largest activation unit a problem may stage
@@ -63,8 +70,8 @@ struct GLayer {
   int n_planes, halo, Rr; // 1 or 4 planes; largest tap shift; staged rows per plane = 128*MT + halo
   int MT;                 // M sub-tiles of 128 positions per tile
   int cb_chunks, n_cb, kpt;
-  int st_ksteps;          // K steps (MMAs per sub-tile) per weight stage; divides 9*kpt
-  uint32_t stage_bytes;   // = st_ksteps * 2 * Nt * 16
+  int st_taps;            // taps per weight stage (the last stage of a channel block holds 9 % st_taps, if not 0)
+  uint32_t tap_bytes;     // weights of one tap of one channel block and channel tile = kpt * 2 * Nt * 16
   int n_ntiles, total_tiles;
   const uint16_t* rank;   // [grid] CTA b takes this problem's tiles rank[b], rank[b] + grid, ...
   long long Qtot;
@@ -77,10 +84,30 @@ struct GParams {
   void* out[SNN_GROUP_MAX];
   int* status;
   int out_i32;            // 0: fp32 alpha*S, 1: int32 S, 2: packed signs of alpha*S
+  uint32_t acc_cols;      // tensor-memory columns of one accumulator buffer
   int NA, NS;
   uint32_t a_slot_bytes, b_slot_bytes;
   uint32_t off_b, off_epi, off_pix, off_lay, off_tail;
 };
+
+// Profiling aid (build with -DSNN_TRACE): every role's reporting lane adds up the cycles it spends in its
+// waits; the host prints the averages over the CTAs after each launch.  No effect on an ordinary build.
+#ifdef SNN_TRACE
+__device__ long long g_trace[256 * 16];
+#define TR_WAIT(var, expr) ([&]() { const long long _t = clock64(); const bool _r = (expr); var += clock64() - _t; return _r; }())
+#define TR_BEGIN(t) const long long t = clock64()
+#define TR_END(var, t) var += clock64() - t
+#define TR_REPORT(role, total, w0, w1, w2)                         \
+  do {                                                             \
+    long long* _o = g_trace + (size_t)blockIdx.x * 16 + (role)*4;  \
+    _o[0] = (total); _o[1] = (w0); _o[2] = (w1); _o[3] = (w2);     \
+  } while (0)
+#else
+#define TR_WAIT(var, expr) (expr)
+#define TR_BEGIN(t) do { } while (0)
+#define TR_END(var, t) do { } while (0)
+#define TR_REPORT(role, total, w0, w1, w2) do { } while (0)
+#endif
 
 __device__ __forceinline__ int g_position_to_pixel(const GLayer& L, uint32_t q, int pa, int pb) {
   if ((long long)q >= L.Qtot) return -1;
@@ -94,6 +121,14 @@ __device__ __forceinline__ int g_position_to_pixel(const GLayer& L, uint32_t q, 
   return ((int)n * L.H + r) * L.W + c;
 }
 
+// one accumulator value (fp32, or int32 below 2^22 in magnitude) times the channel's scale: one rounding
+template <bool FACC>
+__device__ __forceinline__ uint32_t g_scale(uint32_t v, float a) {
+  return __float_as_uint(__fmul_rn(FACC ? __uint_as_float(v) : small_int_to_float(v), a));
+}
+// an fp32 accumulator that holds an integer, as that integer
+__device__ __forceinline__ uint32_t g_to_int(uint32_t v) { return (uint32_t)__float2int_rn(__uint_as_float(v)); }
+
 // first tile of problem L for this CTA (tiles then follow at a stride of the grid)
 __device__ __forceinline__ int g_first_tile(const GLayer& L) {
   return (int)__ldg(L.rank + blockIdx.x);
@@ -103,46 +138,57 @@ __device__ __forceinline__ int g_first_tile(const GLayer& L) {
 // a tap is straight-line code; the taps are a loop, because the issuing thread runs alone on
 // its warp and nine unrolled taps no longer fit the instruction cache closest to it.
 // Weight stages are waited for and released as the K-step counter crosses their boundaries.
-template <bool F16, int MT, int KPT>
-__device__ __forceinline__ bool g_issue_block(uint64_t a_unit, const uint32_t* tapu, uint32_t a_step,
+template <int MODE, int MT, int KPT>
+__device__ __forceinline__ bool g_issue_block(uint64_t a_unit, uint32_t wq, uint32_t plane_units, bool s2, uint32_t a_step,
                                               uint64_t b_desc0, uint32_t b_slot_units, uint32_t b_step, uint32_t d0,
-                                              uint32_t nt, uint32_t idesc, uint32_t& acc, int st_ksteps, int NS,
+                                              uint32_t nt, uint32_t idesc, uint32_t& acc, int st_taps, int NS,
                                               uint32_t bar_bfull, uint32_t bar_bempty, int& b_slot, uint32_t& b_phase,
-                                              bool leader) {
-  int in_stage = 0;
-  uint64_t bd = 0;
+                                              bool leader, uint32_t sf, long long& tr_b) {
+  uint32_t ky = 0, kx = 0;
+  int t = 0;
 #pragma unroll 1
-  for (int t = 0; t < 9; ++t) {
-    const uint64_t ad_t = a_unit + (uint64_t)tapu[t];
-#pragma unroll
-    for (int k = 0; k < KPT; ++k) {
-      if (in_stage == 0) {
-        if (!mbar_wait(bar_bfull + 8 * b_slot, b_phase)) return false;
-        tc_fence_after();
-        bd = b_desc0 + (uint64_t)((uint32_t)b_slot * b_slot_units);
-      }
+  while (t < 9) {
+    // a weight stage holds whole taps: one wait, then nothing but MMAs until its last tap
+    if (!TR_WAIT(tr_b, mbar_wait(bar_bfull + 8 * b_slot, b_phase))) return false;
+    tc_fence_after();
+    uint64_t bd = b_desc0 + (uint64_t)((uint32_t)b_slot * b_slot_units);
+    const int t_end = t + st_taps < 9 ? t + st_taps : 9;
+#pragma unroll 1
+    for (; t < t_end; ++t) {
+      // rows (16-byte units) from a unit's origin to tap (ky, kx): a shift inside the plane, plus, for stride 2,
+      // the offset of the tap's parity plane
+      const uint32_t tap = s2 ? ((ky & 1u) * 2u + (kx & 1u)) * plane_units + (ky >> 1) * wq + (kx >> 1) : ky * wq + kx;
+      if (++kx == 3) { kx = 0; ++ky; }
+      const uint64_t ad_t = a_unit + (uint64_t)tap;
       if (leader) {
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-          mma_ss<F16>(d0 + (uint32_t)mt * nt, ad_t + (uint64_t)((uint32_t)k * a_step + (uint32_t)(mt * 128)), bd,
-                      idesc, acc);
+        for (int k = 0; k < KPT; ++k) {
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            const uint64_t ad = ad_t + (uint64_t)((uint32_t)k * a_step + (uint32_t)(mt * 128));
+            const uint64_t bdk = bd + (uint64_t)((uint32_t)k * b_step);
+            const uint32_t accum = k == 0 ? acc : 1u;
+            if (MODE == M_FP4) mma_ss_fp4(d0 + (uint32_t)mt * nt, ad, bdk, idesc, accum, sf, sf + 16);
+            else mma_ss<MODE == M_F16>(d0 + (uint32_t)mt * nt, ad, bdk, idesc, accum);
+          }
+        }
       }
       acc = 1;
-      bd += b_step;
-      if (++in_stage == st_ksteps) {
-        in_stage = 0;
-        if (leader) tc_commit(bar_bempty + 8 * b_slot);  // the slot is free once these MMAs have read it
-        if (++b_slot == NS) { b_slot = 0; b_phase ^= 1u; }
-      }
+      bd += (uint64_t)((uint32_t)KPT * b_step);
     }
+    if (leader) tc_commit(bar_bempty + 8 * b_slot);  // the slot is free once these MMAs have read it
+    if (++b_slot == NS) { b_slot = 0; b_phase ^= 1u; }
   }
   return true;
 }
 
 }  // namespace
 
-template <bool F16>
+template <int MODE>
 __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p) {
+  constexpr bool F16 = MODE == M_F16;   // fp16 activations (copied, not expanded)
+  constexpr bool FP4 = MODE == M_FP4;   // binary activations as e2m1 nibbles
+  constexpr bool FACC = MODE != M_I8;   // fp32 accumulators
   extern __shared__ __align__(128) uint8_t smem[];
   // carve-up: [NA activation slots][NS weight slots][epilogue tiles][pixel table][problem table][barriers, flags]
   uint8_t* a_smem = smem;
@@ -160,7 +206,6 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
   const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 28);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  uint32_t* tapu = tmem_slot + 3;  // [9] row offset of every tap inside a unit, kept by the MMA issuer (tmem_slot[2]: expander flag)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int NS = p.NS, NA = p.NA;
@@ -191,6 +236,14 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   grid_dep_launch();
+  if (FP4) {
+    // unit block scales: every byte of the scale columns is the ue8m0 code of 1.0, in all 128 lanes
+    // (warps 2..5 cover the four lane quarters), whatever part of them an MMA reads
+    if (warp >= 2 && warp < 6) tmem_fill32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + G_SCALE_COL, 0x7f7f7f7fu);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+  }
 
   if (warp == 0) {
     // ------------------------------------------------ weight producer (one lane)
@@ -199,12 +252,14 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       long long b_issued = 0;
       uint32_t b_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
       bool ok = true;
+      long long tr_w0 = 0, tr_t0 = clock64();
+      (void)tr_w0; (void)tr_t0;
       for (int l = 0; l < p.n_layers && ok; ++l) {
         const GLayer& L = lay[l];
         const int Nt = L.Nt, NtL = L.NtL, n_cb = L.n_cb, n_ntiles = L.n_ntiles, total = L.total_tiles;
-        const int stages_per_cb = 9 * L.kpt / L.st_ksteps;
-        const int chunks_per_stage = 2 * L.st_ksteps;
-        const uint32_t stage_bytes = L.stage_bytes;
+        const int st_taps = L.st_taps, stages_per_cb = (9 + st_taps - 1) / st_taps;
+        const int chunks_per_tap = 2 * L.kpt;
+        const uint32_t tap_bytes = L.tap_bytes;
         const uint8_t* wt = L.wt;
         const size_t cb_bytes = (size_t)9 * L.cb_chunks * NtL * 16;   // one channel block of one layout tile
         const FastDiv dNt = L.dNt;
@@ -218,7 +273,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           for (int cb = 0; cb < n_cb && ok; ++cb) {
             const uint8_t* src = src_tile + (size_t)cb * cb_bytes;
             for (int sg = 0; sg < stages_per_cb; ++sg) {
-              if (b_issued >= NS && !mbar_wait_backoff(bar_bempty + 8 * b_slot, b_phase, 32)) { ok = false; break; }
+              const int ntaps = 9 - sg * st_taps < st_taps ? 9 - sg * st_taps : st_taps;
+              const uint32_t stage_bytes = (uint32_t)ntaps * tap_bytes;
+              const int chunks_per_stage = ntaps * chunks_per_tap;
+              if (b_issued >= NS && !TR_WAIT(tr_w0, mbar_wait_backoff(bar_bempty + 8 * b_slot, b_phase, 32))) { ok = false; break; }
               const uint32_t dst = smem_u32(b_smem) + (uint32_t)b_slot * p.b_slot_bytes;
               mbar_expect_tx(bar_bfull + 8 * b_slot, stage_bytes);
               if (Nt == NtL) {
@@ -239,6 +297,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         *abort_flag = 1;
         raise_status(p.status, 2);
       }
+      TR_REPORT(0, clock64() - tr_t0, tr_w0, 0, 0);
       // never leave with copies in flight: wait (bounded) for the last load of every slot
       for (int s = 0; s < NS; ++s) {
         long long last = -1;
@@ -257,42 +316,37 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       int a_slot = 0, b_slot = 0, acc_slot = 0;
       uint32_t a_phase = 0, b_phase = 0, acc_phase = 1;
       long long tiles_done = 0;
+      long long tr_w0 = 0, tr_w1 = 0, tr_w2 = 0, tr_t0 = clock64();
+      (void)tr_w0; (void)tr_w1; (void)tr_w2; (void)tr_t0;
       const uint32_t a_slot_units = p.a_slot_bytes >> 4, b_slot_units = p.b_slot_bytes >> 4;
       for (int l = 0; l < p.n_layers && ok; ++l) {
         const GLayer& L = lay[l];
         const int Nt = L.Nt, Rr = L.Rr, n_cb = L.n_cb, MT = L.MT, kpt = L.kpt, total = L.total_tiles;
-        const int st_ksteps = L.st_ksteps;
+        const int st_taps = L.st_taps;
         // instruction descriptor: D format, A/B formats, K-major both, N>>3, M>>4
-        const uint32_t idesc = F16 ? ((1u << 4) | ((uint32_t)(Nt >> 3) << 17) | ((128u >> 4) << 24))
-                                   : ((2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(Nt >> 3) << 17) |
-                                      ((128u >> 4) << 24));
+        // (4-bit mode: A/B format e2m1, scale format ue8m0, scale ids 0)
+        const uint32_t idesc =
+            F16 ? ((1u << 4) | ((uint32_t)(Nt >> 3) << 17) | ((128u >> 4) << 24))
+                : FP4 ? ((1u << 7) | (1u << 10) | ((uint32_t)(Nt >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24))
+                      : ((2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(Nt >> 3) << 17) | ((128u >> 4) << 24));
         const uint64_t a_desc0 = make_desc(smem_u32(a_smem), (uint32_t)Rr * 16, 128);
         const uint64_t b_desc0 = make_desc(smem_u32(b_smem), (uint32_t)Nt * 16, 128);
         const uint32_t a_step = 2u * (uint32_t)Rr, b_step = 2u * (uint32_t)Nt;  // two chunks per MMA
-        // rows (16-byte units) from a unit's origin to tap t: plane offset + shift inside the plane
-        __syncwarp();
-        if (lane < 9) {
-          const int t = lane;
-          const int ky = t / 3, kx = t % 3;
-          tapu[t] = L.stride == 1 ? (uint32_t)(ky * L.Wq + kx)
-                                  : (uint32_t)((ky & 1) * 2 + (kx & 1)) * (uint32_t)(L.cb_chunks * Rr) +
-                                        (uint32_t)((ky >> 1) * L.Wq + (kx >> 1));
-        }
-        __syncwarp();
         for (int tile = g_first_tile(L); tile < total && ok; tile += G, ++tiles_done) {
           if (tiles_done >= 2) {
-            if (!mbar_wait(bar_accempty + 8 * acc_slot, acc_phase)) { ok = false; break; }
+            if (!TR_WAIT(tr_w0, mbar_wait(bar_accempty + 8 * acc_slot, acc_phase))) { ok = false; break; }
             tc_fence_after();
           }
-          const uint32_t d0 = tmem_base + (uint32_t)acc_slot * G_ACC_COLS;
+          const uint32_t d0 = tmem_base + (uint32_t)acc_slot * p.acc_cols;
           uint32_t acc = 0;  // 0 only for the first MMA of every sub-tile
           for (int cb = 0; cb < n_cb && ok; ++cb) {
-            if (!mbar_wait(bar_afull + 8 * a_slot, a_phase)) { ok = false; break; }
+            if (!TR_WAIT(tr_w1, mbar_wait(bar_afull + 8 * a_slot, a_phase))) { ok = false; break; }
             tc_fence_after();
             const uint64_t a_unit = a_desc0 + (uint64_t)((uint32_t)a_slot * a_slot_units);
 #define G_ISSUE(M, KP)                                                                                       \
-  ok = g_issue_block<F16, M, KP>(a_unit, tapu, a_step, b_desc0, b_slot_units, b_step, d0, (uint32_t)Nt, idesc, acc, \
-                                 st_ksteps, NS, bar_bfull, bar_bempty, b_slot, b_phase, leader)
+  ok = g_issue_block<MODE, M, KP>(a_unit, (uint32_t)L.Wq, (uint32_t)(L.cb_chunks * Rr), L.stride != 1, a_step, b_desc0, b_slot_units, b_step, d0, (uint32_t)Nt, idesc, acc, \
+                                  st_taps, NS, bar_bfull, bar_bempty, b_slot, b_phase, leader,                   \
+                                  tmem_base + G_SCALE_COL, tr_w2)
 #define G_ISSUE_K(M)                   \
   do {                                 \
     if (kpt == 4) G_ISSUE(M, 4);       \
@@ -301,6 +355,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     else G_ISSUE(M, 1);                \
   } while (0)
             if (MT == 4) G_ISSUE_K(4);
+            else if (MT == 3) G_ISSUE_K(3);
             else if (MT == 2) G_ISSUE_K(2);
             else G_ISSUE_K(1);
 #undef G_ISSUE_K
@@ -318,6 +373,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         *abort_flag = 1;
         raise_status(p.status, 3);
       }
+      if (leader) TR_REPORT(1, clock64() - tr_t0, tr_w0, tr_w1, tr_w2);
     }
     __syncwarp();
   } else if (warp < 2 + G_EW) {
@@ -333,6 +389,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     int acc_slot = 0;
     uint32_t acc_phase = 0;
     bool live = true;
+    long long tr_w0 = 0, tr_w1 = 0, tr_w2 = 0, tr_t0 = clock64();
+    (void)tr_w0; (void)tr_w1; (void)tr_w2; (void)tr_t0;
     for (int l = 0; l < p.n_layers && live; ++l) {
       const GLayer& L = lay[l];
       const int Nt = L.Nt, MT = L.MT, K = L.K;
@@ -344,7 +402,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
         const int n0 = nti * Nt;
         int okw = 1;
-        if (lane == 0) okw = (!*abort_flag && mbar_wait_backoff(bar_accfull + 8 * acc_slot, acc_phase, 100)) ? 1 : 0;
+        if (lane == 0) okw = (!*abort_flag && TR_WAIT(tr_w0, mbar_wait_backoff(bar_accfull + 8 * acc_slot, acc_phase, 100))) ? 1 : 0;
         okw = __shfl_sync(0xffffffffu, okw, 0);
         if (!okw) {
           if (lane == 0 && !*abort_flag) {
@@ -355,7 +413,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           break;
         }
         tc_fence_after();
-        const uint32_t d0 = tmem_base + (uint32_t)acc_slot * G_ACC_COLS;
+        const uint32_t d0 = tmem_base + (uint32_t)acc_slot * p.acc_cols;
         // output pixel (n*Ho + y)*Wo + x of the row of sub-tile mt this lane owns in TMEM, or -1
         auto row_pixel = [&](int mt) -> int {
           const uint32_t q = Q0 + (uint32_t)(mt * 128 + rq * 32 + lane);
@@ -388,7 +446,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 #pragma unroll
                   for (int e = 0; e < 32; ++e) {
                     const float a = co0 + e < K ? __ldg(alpha + co0 + e) : -1.f;  // a missing channel gives bit 0 ...
-                    const float s = co0 + e < K ? small_int_to_float(v[e]) : 1.f;  // ... through 1 * -1 < 0
+                    const float s = co0 + e >= K ? 1.f  // ... through 1 * -1 < 0
+                                                 : FACC ? __uint_as_float(v[e]) : small_int_to_float(v[e]);
                     word |= (__fmul_rn(s, a) >= 0.f ? 1u : 0u) << e;
                   }
                   out32[wide_mul((uint32_t)pix, (uint32_t)Kw) + (uint32_t)(co0 >> 5)] = word;
@@ -413,7 +472,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 #pragma unroll
                   for (int e = 0; e < 16; ++e) {
                     const float a = co0 + e < K ? __ldg(alpha + co0 + e) : -1.f;
-                    const float s = co0 + e < K ? small_int_to_float(v[e]) : 1.f;
+                    const float s = co0 + e >= K ? 1.f : FACC ? __uint_as_float(v[e]) : small_int_to_float(v[e]);
                     hw |= (__fmul_rn(s, a) >= 0.f ? 1u : 0u) << e;
                   }
                   const size_t at = wide_mul((uint32_t)pix, (uint32_t)(2 * Kw)) + (uint32_t)(co0 >> 4);
@@ -462,8 +521,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
               if (!p.out_i32) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                  scale_pair<F16>(u[i].x, u[i].y, al.x, al.y);
-                  scale_pair<F16>(u[i].z, u[i].w, al.z, al.w);
+                  scale_pair<FACC>(u[i].x, u[i].y, al.x, al.y);
+                  scale_pair<FACC>(u[i].z, u[i].w, al.z, al.w);
+                }
+              } else if (FACC) {
+                // int32 sums asked of fp32 accumulators: the sums are integers, the conversion is exact
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  u[i].x = (uint32_t)__float2int_rn(__uint_as_float(u[i].x));
+                  u[i].y = (uint32_t)__float2int_rn(__uint_as_float(u[i].y));
+                  u[i].z = (uint32_t)__float2int_rn(__uint_as_float(u[i].z));
+                  u[i].w = (uint32_t)__float2int_rn(__uint_as_float(u[i].w));
                 }
               }
               uint32_t* obase32 = out32 + co;
@@ -490,9 +558,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 #pragma unroll
               for (int e = 0; e < 16; ++e) {
                 if (co0 + e < K) {
-                  if (p.out_i32) o[e] = v[e];
+                  if (p.out_i32) o[e] = FACC ? (uint32_t)__float2int_rn(__uint_as_float(v[e])) : v[e];
                   else
-                    o[e] = __float_as_uint(__fmul_rn(F16 ? __uint_as_float(v[e]) : small_int_to_float(v[e]),
+                    o[e] = __float_as_uint(__fmul_rn(FACC ? __uint_as_float(v[e]) : small_int_to_float(v[e]),
                                                      __ldg(alpha + co0 + e)));
                 }
               }
@@ -506,6 +574,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         if (++acc_slot == 2) { acc_slot = 0; acc_phase ^= 1u; }
       }
     }
+    if (warp == 2 && lane == 0) TR_REPORT(2, clock64() - tr_t0, tr_w0, tr_w1, tr_w2);
   } else if (warp != 13 && warp != 17) {
     // ------------------------------------------------ expanders (warps 10-12, 14-16, 18, 19)
     // Fill activation unit (problem, tile, channel block) of the ring: for every plane, row and
@@ -517,6 +586,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     uint32_t a_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
     volatile int* exp_flag = abort_flag + 1;
     bool stop = false;
+    long long tr_w0 = 0, tr_t0 = clock64();
+    (void)tr_w0; (void)tr_t0;
     for (int l = 0; l < p.n_layers && !stop; ++l) {
       const GLayer& L = lay[l];
       const int Rr = L.Rr, n_planes = L.n_planes, n_cb = L.n_cb, cb_chunks = L.cb_chunks, MT = L.MT;
@@ -528,10 +599,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       {
         const uintptr_t addr = (uintptr_t)act;
         if (F16) vec = (addr & 15) == 0 && (C & 7) == 0;
+        else if (FP4) vec = (addr & 7) == 0 && (Cw & 1) == 0;  // pairs of words (a block's first word is even)
         else if (cb_chunks == 8) vec = (addr & 15) == 0 && (Cw & 3) == 0;
         else if (cb_chunks == 4) vec = (addr & 7) == 0 && (Cw & 1) == 0;
         else vec = false;
       }
+      const bool vec4 = FP4 && vec && ((uintptr_t)act & 15) == 0 && (Cw & 3) == 0 && (cb_chunks & 3) == 0;
       const int nstep = cb_chunks / 2;  // pairs of chunks per unit
       for (int tile = g_first_tile(L); tile < total && !stop; tile += G) {
         const int mg = (int)fdiv((uint32_t)tile, dNt);
@@ -549,7 +622,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         for (int cb = 0; cb < n_cb; ++cb) {
           if (a_done >= NA) {
             // one elected thread polls; the rest wait on a hardware barrier instead of spinning
-            if (et == 0) *exp_flag = (!*abort_flag && mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 64)) ? 1 : 0;
+            if (et == 0) *exp_flag = (!*abort_flag && TR_WAIT(tr_w0, mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 64))) ? 1 : 0;
             asm volatile("bar.sync 3, %0;" ::"n"(G_EXP_THREADS) : "memory");
             const int okf = *exp_flag;
             asm volatile("bar.sync 3, %0;" ::"n"(G_EXP_THREADS) : "memory");
@@ -607,6 +680,46 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
                     }
                   }
                 }
+              } else if (FP4) {
+                // a 32-channel word is one chunk of nibbles; four (or two) words per row as one vector load
+                const int wb = cb * cb_chunks;
+                for (int k0 = 0; k0 < cb_chunks; k0 += 4) {
+                  const int nw = cb_chunks - k0 < 4 ? cb_chunks - k0 : 4;  // 4 or 2
+                  uint32_t bits[G_EXP_ROWS][4];
+#pragma unroll
+                  for (int j = 0; j < G_EXP_ROWS; ++j) {
+                    bits[j][0] = bits[j][1] = bits[j][2] = bits[j][3] = 0;
+                    const int w0 = wb + k0;
+                    if (pix[j] >= 0 && w0 < Cw) {
+                      const uint32_t* src = (const uint32_t*)act + wide_mul((uint32_t)pix[j], (uint32_t)Cw) + w0;
+                      if (vec4) {
+                        const uint4 t = __ldg(reinterpret_cast<const uint4*>(src));
+                        bits[j][0] = t.x; bits[j][1] = t.y; bits[j][2] = t.z; bits[j][3] = t.w;
+                      } else if (vec) {
+                        const uint2 t = __ldg(reinterpret_cast<const uint2*>(src));
+                        bits[j][0] = t.x; bits[j][1] = t.y;
+                        if (nw == 4) {
+                          const uint2 t2 = __ldg(reinterpret_cast<const uint2*>(src + 2));
+                          bits[j][2] = t2.x; bits[j][3] = t2.y;
+                        }
+                      } else {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                          if (k < nw && w0 + k < Cw) bits[j][k] = __ldg(src + k);
+                      }
+                    }
+                  }
+#pragma unroll
+                  for (int j = 0; j < G_EXP_ROWS; ++j) {
+                    if (pix[j] != -2) {
+#pragma unroll
+                      for (int k = 0; k < 4; ++k)
+                        if (k < nw)
+                          *reinterpret_cast<uint4*>(dst[j] + (size_t)(k0 + k) * Rr * 16) =
+                              expand_word_fp4(bits[j][k], pix[j] >= 0 && wb + k0 + k < Cw);
+                    }
+                  }
+                }
               } else {
                 // up to four 32-channel words per row and block, as one vector load when aligned
                 const int w0 = cb * nstep;
@@ -653,6 +766,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         }
       }
     }
+    if (et == 0) TR_REPORT(3, clock64() - tr_t0, tr_w0, 0, 0);
   }
 
   // ---------------------------------------------------------------- teardown
@@ -665,7 +779,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 
 // ------------------------------------------------------------------ host side
 struct GroupDev {
-  int count = 0, act_type = 0;
+  int count = 0, act_type = 0, mode = M_I8;
   GLayer* layers_dev = nullptr;   // [count]
   uint8_t* weights = nullptr;     // the group's own weight operands, one after the other
   uint16_t* ranks = nullptr;      // [count][grid] tile assignment, see tcg_create
@@ -677,8 +791,68 @@ struct GroupDev {
 namespace {
 
 // Tile shape, channel blocks and weight stages of one problem under the group's fixed slot sizes.
-bool g_plan_layer(const Geom& g, bool f16, GLayer* L, int* n_chunks_out, int* Kpad_out) {
-  const int cpc = f16 ? 8 : 16;
+// Operand of the weights: wt[layout tile][channel block][tap][chunk][NtL][16 B]; a chunk is 16 bytes along the
+// input channels (16 int8, 8 fp16 or 32 e2m1 values), cb_chunks chunks per block, NtL output channels per
+// layout tile.  Channels that do not exist are zeros, so whatever the activation operand holds there adds 0.
+template <int MODE>
+__global__ void g_expand_weights_kernel(const uint32_t* __restrict__ wplanes, uint8_t* __restrict__ wt, int C, int K,
+                                        int Cw, long long total, int cb_chunks, int n_cb, int NtL) {
+  long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  int row = (int)(i % NtL);
+  long long r = i / NtL;
+  int c = (int)(r % cb_chunks);
+  r /= cb_chunks;
+  int t = (int)(r % 9);
+  r /= 9;
+  int cb = (int)(r % n_cb), tile = (int)(r / n_cb);
+  int co = tile * NtL + row;
+  constexpr int cpc = MODE == M_F16 ? 8 : MODE == M_FP4 ? 32 : 16;
+  uint4 v = make_uint4(0, 0, 0, 0);
+  if (co < K) {
+    int ch0 = (cb * cb_chunks + c) * cpc;
+    int wd = ch0 >> 5, sh = ch0 & 31;
+    uint32_t bits = wd < Cw ? wplanes[((size_t)t * Cw + wd) * K + co] >> sh : 0u;
+    uint32_t w[4] = {0, 0, 0, 0};
+    if (MODE == M_F16) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (ch0 + e < C) w[e >> 1] |= (((bits >> e) & 1u) ? 0x3c00u : 0xbc00u) << (16 * (e & 1));  // +1.0 / -1.0
+    } else if (MODE == M_FP4) {
+#pragma unroll
+      for (int e = 0; e < 32; ++e)
+        if (ch0 + e < C) w[e >> 3] |= (((bits >> e) & 1u) ? 0x2u : 0xau) << (4 * (e & 7));         // e2m1 +1.0 / -1.0
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; ++e)
+        if (ch0 + e < C) w[e >> 2] |= (((bits >> e) & 1u) ? 0x01u : 0xffu) << (8 * (e & 3));       // +1 / -1
+    }
+    v = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  reinterpret_cast<uint4*>(wt)[i] = v;
+}
+
+cudaError_t g_expand_weights(int mode, const uint32_t* wplanes, void* dst, int C, int K, int Cw, int Kpad, int n_chunks,
+                             int cb_chunks, int NtL, cudaStream_t s) {
+  const long long total = (long long)9 * n_chunks * Kpad;
+  const unsigned blocks = (unsigned)((total + 255) / 256);
+  const int n_cb = n_chunks / cb_chunks;
+  if (mode == M_F16)
+    g_expand_weights_kernel<M_F16><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL);
+  else if (mode == M_FP4)
+    g_expand_weights_kernel<M_FP4><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL);
+  else
+    g_expand_weights_kernel<M_I8><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL);
+  return cudaGetLastError();
+}
+
+// Cycles of one MMA of 128 positions x nt channels as measured on B200 (any operand type): half a cycle per
+// channel plus a constant that does not overlap the previous MMA.
+inline double g_mma_cycles(int nt) { return 0.5 * nt + 33.0; }
+
+bool g_plan_layer(const Geom& g, int mode, GLayer* L, int* n_chunks_out, int* Kpad_out) {
+  const int cpc = mode == M_F16 ? 8 : mode == M_FP4 ? 32 : 16;
+  const int acc_cols = mode == M_FP4 ? (int)G_ACC_COLS_FP4 : (int)G_ACC_COLS;
   const int raw = round_up(g.C, 2 * cpc) / cpc;  // 16-byte chunks along the channels, even
   GLayer& o = *L;
   o.N = g.N; o.H = g.H; o.W = g.W; o.C = g.C; o.K = g.K; o.Cw = g.Cw;
@@ -697,7 +871,8 @@ bool g_plan_layer(const Geom& g, bool f16, GLayer* L, int* n_chunks_out, int* Kp
   if ((long long)g.N * g.H * g.W >= (1ll << 31) || (long long)g.N * g.Ho * g.Wo >= (1ll << 31)) return false;
   // layout tile of the weight operand = channels per tile: all of them up to 256; beyond that 256
   // when that pads little (fewer channel tiles re-expand the same activations), else 128
-  o.NtL = g.K <= 256 ? round_up(g.K, 16) : (round_up(g.K, 256) - g.K < 64 ? 256 : 128);
+  if (mode == M_FP4) o.NtL = g.K <= acc_cols ? round_up(g.K, 16) : 128;
+  else o.NtL = g.K <= 256 ? round_up(g.K, 16) : (round_up(g.K, 256) - g.K < 64 ? 256 : 128);
   o.Nt = o.NtL;
   const int Kpad = round_up(g.K, o.NtL);
   o.n_ntiles = Kpad / o.Nt;
@@ -713,24 +888,21 @@ bool g_plan_layer(const Geom& g, bool f16, GLayer* L, int* n_chunks_out, int* Kp
   o.n_cb = raw / d;
   o.kpt = d / 2;
   int MT = 1;
-  for (int m = 4; m >= 2; m /= 2)
-    if ((size_t)o.n_planes * d * (128 * m + o.halo) * 16 <= kGASlotMax && m * o.Nt <= (int)G_ACC_COLS) { MT = m; break; }
+  for (int m = 4; m >= 2; --m)
+    if ((size_t)o.n_planes * d * (128 * m + o.halo) * 16 <= kGASlotMax && m * o.Nt <= acc_cols) { MT = m; break; }
   const long long mtiles = (o.Qtot + 127) / 128;
-  while (MT > 1 && mtiles < MT) MT /= 2;  // a tiny problem does not need the larger tile
+  while (MT > 1 && mtiles < MT) --MT;  // a tiny problem does not need the larger tile
   o.MT = MT;
   o.Rr = 128 * MT + o.halo;
   if ((uint32_t)o.Rr * 16 >= (1u << 18)) return false;  // leading-offset field of the descriptor
   const long long mgroups = (mtiles + MT - 1) / MT;
   if (mgroups * o.n_ntiles > 0x7fffffffLL || mgroups * o.Rr >= (1ll << 31)) return false;
   o.total_tiles = (int)(mgroups * o.n_ntiles);
-  // weight stage: the longest run of K steps that divides a channel block's 9*kpt and fits a slot
-  const int ks_bytes = 2 * o.Nt * 16;
-  int st = 0;
-  for (int s = 9 * o.kpt; s >= 1; --s)
-    if ((9 * o.kpt) % s == 0 && (size_t)s * ks_bytes <= kGBSlot) { st = s; break; }
-  if (!st) return false;
-  o.st_ksteps = st;
-  o.stage_bytes = (uint32_t)(st * ks_bytes);
+  // weight stage: as many whole taps of a channel block as fit a slot
+  o.tap_bytes = (uint32_t)(o.kpt * 2 * o.Nt * 16);
+  int st = (int)(kGBSlot / o.tap_bytes);
+  if (st < 1) return false;
+  o.st_taps = st > 9 ? 9 : st;
   *n_chunks_out = raw;
   *Kpad_out = Kpad;
   return true;
@@ -742,14 +914,14 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
                        GroupDev** out, int* launched) {
   *out = nullptr;
   if (count < 1 || count > SNN_GROUP_MAX) return cudaErrorInvalidConfiguration;
-  const bool f16 = act_type == SNN_ACT_F16;
+  const int mode = act_type == SNN_ACT_F16 ? M_F16 : (env_int("SNN_TCG_I8", 0) ? M_I8 : M_FP4);
   GLayer host[SNN_GROUP_MAX];
   int n_chunks[SNN_GROUP_MAX], Kpad[SNN_GROUP_MAX];
   size_t w_off[SNN_GROUP_MAX], w_total = 0;
   size_t a_slot = 0, pix_bytes = 0;
   long long tiles = 0;
   for (int i = 0; i < count; ++i) {
-    if (!g_plan_layer(gs[i], f16, &host[i], &n_chunks[i], &Kpad[i])) return cudaErrorInvalidConfiguration;
+    if (!g_plan_layer(gs[i], mode, &host[i], &n_chunks[i], &Kpad[i])) return cudaErrorInvalidConfiguration;
     const size_t unit = (size_t)host[i].n_planes * host[i].cb_chunks * host[i].Rr * 16;
     if (unit > a_slot) a_slot = unit;
     const size_t pb = (size_t)host[i].n_planes * host[i].Rr * 4;
@@ -784,7 +956,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
     std::vector<int> order(grid);
     for (int i = 0; i < count; ++i) {
       const GLayer& o = host[i];
-      const double mma = (double)o.MT * o.n_cb * 9 * o.kpt * (o.Nt > 146 ? o.Nt / 2 : 73);
+      const double mma = (double)o.MT * o.n_cb * 9 * o.kpt * g_mma_cycles(o.Nt);
       const double wr = 128.0 * o.MT * (o.Nt < o.K ? o.Nt : o.K) * 4 / 13.0;
       const double cost = (mma > wr ? mma : wr) + 300.0;
       for (int b = 0; b < grid; ++b) order[b] = b;
@@ -799,6 +971,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   GroupDev* G = new GroupDev();
   G->count = count;
   G->act_type = act_type;
+  G->mode = mode;
   G->grid = grid;
   cudaError_t e = cudaMalloc(&G->weights, w_total);
   if (e == cudaSuccess) e = cudaMalloc(&G->layers_dev, sizeof(GLayer) * count);
@@ -809,8 +982,8 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
     host[i].rank = G->ranks + (size_t)i * grid;
     host[i].wt = G->weights + w_off[i];
     host[i].alpha = Ls[i]->alpha;
-    e = tc_expand_weights_custom(Ls[i]->wplanes, G->weights + w_off[i], gs[i].C, gs[i].K, gs[i].Cw, Kpad[i],
-                                 n_chunks[i], host[i].cb_chunks, host[i].NtL, f16, s);
+    e = g_expand_weights(mode, Ls[i]->wplanes, G->weights + w_off[i], gs[i].C, gs[i].K, gs[i].Cw, Kpad[i],
+                         n_chunks[i], host[i].cb_chunks, host[i].NtL, s);
     if (e == cudaSuccess) *launched += 1;
   }
   if (e == cudaSuccess) e = cudaMemcpyAsync(G->layers_dev, host, sizeof(GLayer) * count, cudaMemcpyHostToDevice, s);
@@ -824,6 +997,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   p.n_layers = count;
   p.NA = na;
   p.NS = ns;
+  p.acc_cols = mode == M_FP4 ? G_ACC_COLS_FP4 : G_ACC_COLS;
   p.a_slot_bytes = (uint32_t)a_slot;
   p.b_slot_bytes = kGBSlot;
   p.off_b = (uint32_t)((size_t)na * a_slot);
@@ -872,17 +1046,38 @@ cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, i
   cfg.blockDim = dim3(G_THREADS);
   cfg.dynamicSmemBytes = G->smem;
   cudaError_t e;
-  if (G->act_type == SNN_ACT_F16) {
+  if (G->mode == M_F16) {
     static unsigned long long done = 0;
-    e = allow_max_smem(tcg_conv_kernel<true>, &done);
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<true>, p);
+    e = allow_max_smem(tcg_conv_kernel<M_F16>, &done);
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<M_F16>, p);
+  } else if (G->mode == M_FP4) {
+    static unsigned long long done = 0;
+    e = allow_max_smem(tcg_conv_kernel<M_FP4>, &done);
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<M_FP4>, p);
   } else {
     static unsigned long long done = 0;
-    e = allow_max_smem(tcg_conv_kernel<false>, &done);
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<false>, p);
+    e = allow_max_smem(tcg_conv_kernel<M_I8>, &done);
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<M_I8>, p);
   }
   if (e != cudaSuccess) return e;
   *launched += 1;
+#ifdef SNN_TRACE
+  {
+    static long long h[256 * 16];
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(h, g_trace, sizeof(h));
+    static const char* role[4] = {"producer", "mma", "epilogue", "expander"};
+    for (int r = 0; r < 4; ++r) {
+      double a[4] = {0, 0, 0, 0}, mx = 0;
+      for (int b = 0; b < G->grid; ++b) {
+        for (int k = 0; k < 4; ++k) a[k] += (double)h[b * 16 + r * 4 + k] / G->grid;
+        if ((double)h[b * 16 + r * 4] > mx) mx = (double)h[b * 16 + r * 4];
+      }
+      fprintf(stderr, "[trace] %-9s total %8.0f (max %8.0f)  waits %8.0f %8.0f %8.0f cycles\n", role[r], a[0], mx, a[1], a[2],
+              a[3]);
+    }
+  }
+#endif
   return cudaGetLastError();
 }
 
