@@ -56,10 +56,13 @@ enum { SNN_ACT_BIN = 0, SNN_ACT_F16 = 1 };
 enum {
   SNN_OUT_F32 = 0,
   SNN_OUT_I32 = 1,  /* only with SNN_ACT_BIN */
-  SNN_OUT_BITS = 2  /* only with SNN_ACT_BIN and the tensor-core path: the signs of Y, packed as the next
-                       layer's binary input (Algorithm 1: layer i consumes sign(a^{i-1})):
-                       uint32 [N][Ho][Wo][ceil(c_out/32)], bit co%32 of word co/32 = 1 iff Y >= 0
-                       (so S = 0 gives +1), unused high bits 0 */
+  SNN_OUT_BITS = 2  /* only with SNN_ACT_BIN and the tensor-core path: the thresholded signs of Y, packed as the
+                       next layer's binary input (Algorithm 1: layer i consumes sign(a^{i-1}); between two
+                       binary layers sit a batch normalisation and a Hardtanh, Sec. 5, i.e. a per-channel
+                       affine map whose sign is the sign of Y plus a per-channel constant):
+                       uint32 [N][Ho][Wo][ceil(c_out/32)], bit co%32 of word co/32 = 1 iff
+                       fl(fl(alpha[co] * S) + shift[co]) >= 0 in fp32, round to nearest even
+                       (so 0 gives +1; shift is 0 where the descriptor has none), unused high bits 0 */
 };
 enum {
   SNN_PATH_AUTO = 0,       /* tuned choice if snn_conv_tune ran for the shape, else a heuristic */
@@ -77,6 +80,8 @@ typedef struct {
   const uint16_t* codebook;   /* HOST, 2^tau codes, each < 512; duplicates allowed */
   const uint8_t* idx_packed;  /* HOST, ceil(c_out*c_in*tau/8) bytes, see above */
   const float* alpha;         /* HOST, c_out finite fp32 scales */
+  const float* shift;         /* HOST, c_out finite fp32 thresholds added to Y before its sign is taken
+                                 (SNN_OUT_BITS only; fp32 and int32 outputs ignore it), or NULL for none */
 } snn_conv_desc_t;
 
 /*
@@ -84,7 +89,7 @@ typedef struct {
  * them on return), unpacks the index stream and decodes the weights on the
  * device.  *out receives a handle that owns its device buffers.
  * Errors: INVALID_ARG (null pointer, tau/stride/pad out of range, code >= 512,
- * non-finite alpha, c_in/c_out < 1), CUDA, OOM.
+ * non-finite alpha or shift, c_in/c_out < 1), CUDA, OOM.
  */
 SNN_API snn_status_t snn_conv_create(const snn_conv_desc_t* desc, snn_conv_t** out);
 

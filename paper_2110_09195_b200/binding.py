@@ -43,6 +43,7 @@ class _Desc(ctypes.Structure):
         ("stride", ctypes.c_int32), ("pad", ctypes.c_int32), ("act_type", ctypes.c_int32),
         ("device", ctypes.c_int32),
         ("codebook", ctypes.c_void_p), ("idx_packed", ctypes.c_void_p), ("alpha", ctypes.c_void_p),
+        ("shift", ctypes.c_void_p),
     ]
 
 
@@ -135,9 +136,24 @@ def forward_static(c_in, c_out, tau, codebook, idx_packed, alpha, act, out, stri
         raise SnnError(1, "index stream or alpha of the wrong size")
     if not (act.is_cuda and out.is_cuda and act.is_contiguous() and out.is_contiguous()):
         raise SnnError(1, "act and out must be contiguous CUDA tensors")
+    # the C entry point cannot see the sizes of the buffers behind its pointers: check them here
+    if act.device.index != int(device) or out.device.index != int(device):
+        raise SnnError(1, f"act and out must live on cuda:{device}")
+    if act.dtype not in (torch.int32, torch.uint32) or act.dim() != 4 or act.shape[3] != (int(c_in) + 31) // 32:
+        raise SnnError(1, "binary activations must be int32/uint32 (N, H, W, ceil(c_in/32))")
+    if int(stride) not in (1, 2) or int(pad) not in (0, 1):
+        raise SnnError(1, "stride must be 1 or 2 and pad 0 or 1")
     n, h, w = int(act.shape[0]), int(act.shape[1]), int(act.shape[2])
+    if h + 2 * int(pad) < 3 or w + 2 * int(pad) < 3:
+        raise SnnError(1, "the map is smaller than the kernel")
+    ho, wo = (h + 2 * int(pad) - 3) // int(stride) + 1, (w + 2 * int(pad) - 3) // int(stride) + 1
+    if out_type not in (OUT_F32, OUT_I32):
+        raise SnnError(1, "forward_static writes fp32 or int32 outputs")
+    want = torch.float32 if out_type == OUT_F32 else torch.int32
+    if out.dtype != want or tuple(out.shape) != (n, ho, wo, int(c_out)):
+        raise SnnError(1, f"out must be {want} of shape {(n, ho, wo, int(c_out))}")
     d = _Desc(int(c_in), int(c_out), int(tau), int(stride), int(pad), ACT_BIN, int(device),
-              cb.ctypes.data, ip.ctypes.data, al.ctypes.data)
+              cb.ctypes.data, ip.ctypes.data, al.ctypes.data, None)
     if stream is None:
         stream = torch.cuda.current_stream(device)
     _check(load_library().snn_conv_forward_static(ctypes.byref(d), act.data_ptr(), n, h, w, out.data_ptr(),
@@ -148,7 +164,8 @@ def forward_static(c_in, c_out, tau, codebook, idx_packed, alpha, act, out, stri
 class SnnConv:
     """One sub-bit 3x3 layer on one GPU (wraps a snn_conv_t handle)."""
 
-    def __init__(self, c_in, c_out, tau, codebook, idx_packed, alpha, stride=1, pad=1, act_type=ACT_BIN, device=0):
+    def __init__(self, c_in, c_out, tau, codebook, idx_packed, alpha, stride=1, pad=1, act_type=ACT_BIN, device=0,
+                 shift=None):
         lib = load_library()
         cb = np.ascontiguousarray(codebook, dtype=np.uint16)
         ip = np.ascontiguousarray(idx_packed, dtype=np.uint8)
@@ -161,8 +178,11 @@ class SnnConv:
             raise SnnError(1, "index stream shorter than c_out*c_in*tau bits")
         if al.size != int(c_out):
             raise SnnError(1, f"alpha has {al.size} entries, expected {c_out}")
+        sh = None if shift is None else np.ascontiguousarray(shift, dtype=np.float32)
+        if sh is not None and sh.size != int(c_out):
+            raise SnnError(1, f"shift has {sh.size} entries, expected {c_out}")
         d = _Desc(int(c_in), int(c_out), int(tau), int(stride), int(pad), int(act_type), int(device),
-                  cb.ctypes.data, ip.ctypes.data, al.ctypes.data)
+                  cb.ctypes.data, ip.ctypes.data, al.ctypes.data, None if sh is None else sh.ctypes.data)
         h = ctypes.c_void_p()
         self._h = None
         _check(lib.snn_conv_create(ctypes.byref(d), ctypes.byref(h)))

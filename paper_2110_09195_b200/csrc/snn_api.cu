@@ -55,7 +55,8 @@ struct snn_conv {
   int C, K, tau, stride, pad, act_type, device;
   LayerDev L;
   std::mutex mu;
-  std::map<std::tuple<int, int, int>, std::pair<int, int>> tuned;  // (N,H,W) -> (path, tensor-core variant)
+  std::map<std::tuple<int, int, int>, int> tuned;        // (N,H,W) -> path measured fastest by snn_conv_tune
+  std::map<std::tuple<int, int, int>, GroupDev*> solo;   // (N,H,W) -> tensor-core plan and weight operand (a group of one)
   // staging for snn_conv_forward_host
   void* stage_in = nullptr;
   void* stage_out = nullptr;
@@ -86,14 +87,14 @@ bool path_ok(const snn_conv* h, int path, const Geom& g) {
   switch (path) {
     case SNN_PATH_REUSE: return reuse_supported(g, h->act_type);
     case SNN_PATH_DECODED: return popc_supported(g, h->act_type);
-    case SNN_PATH_DECODED_TC: return tc_supported(g, h->act_type);
+    case SNN_PATH_DECODED_TC: return tcg_supported(g, h->act_type);
     default: return false;
   }
 }
 
 // Untuned default: tensor cores when they apply, else the popcount path for
 // small c_out relative to the codebook and the reuse path for large (Sec. 4.5:
-// sharing pays in proportion to c_out / 2^tau).
+// sharing pays in proportion to c_out / 2^tau).  0 when no path can run the layer.
 int heuristic_path(const snn_conv* h, const Geom& g) {
   if (path_ok(h, SNN_PATH_DECODED_TC, g)) return SNN_PATH_DECODED_TC;
   if (h->act_type == SNN_ACT_BIN) {
@@ -101,7 +102,7 @@ int heuristic_path(const snn_conv* h, const Geom& g) {
     if (path_ok(h, SNN_PATH_DECODED, g)) return SNN_PATH_DECODED;
   }
   if (path_ok(h, SNN_PATH_REUSE, g)) return SNN_PATH_REUSE;
-  return SNN_PATH_DECODED;
+  return 0;
 }
 
 int auto_path(snn_conv* h, const Geom& g) {
@@ -112,27 +113,39 @@ int auto_path(snn_conv* h, const Geom& g) {
   {
     std::lock_guard<std::mutex> lk(h->mu);
     auto it = h->tuned.find(std::make_tuple(g.N, g.H, g.W));
-    if (it != h->tuned.end()) return it->second.first;
+    if (it != h->tuned.end()) return it->second;
   }
   return heuristic_path(h, g);
 }
 
-// Tensor-core tile variant remembered by snn_conv_tune for this shape (0 = heuristic).
-int tuned_variant(snn_conv* h, const Geom& g) {
+// The tensor-core kernel's plan and weight operand for this input shape: built (and allocated) at the first
+// call for the shape, reused afterwards.
+cudaError_t solo_group(snn_conv* h, const Geom& g, GroupDev** out, int* launched) {
   std::lock_guard<std::mutex> lk(h->mu);
-  auto it = h->tuned.find(std::make_tuple(g.N, g.H, g.W));
-  return (it != h->tuned.end() && it->second.first == SNN_PATH_DECODED_TC) ? it->second.second : 0;
+  const auto key = std::make_tuple(g.N, g.H, g.W);
+  auto it = h->solo.find(key);
+  if (it != h->solo.end()) { *out = it->second; return cudaSuccess; }
+  const LayerDev* Lp = &h->L;
+  GroupDev* G = nullptr;
+  cudaError_t e = tcg_create(&Lp, &g, 1, h->act_type, h->host_stream, &G, launched);
+  if (e != cudaSuccess) return e;
+  h->solo[key] = G;
+  *out = G;
+  return cudaSuccess;
 }
 
-snn_status_t run_path(snn_conv* h, int path, const Geom& g, const Launch& l, int variant = -1) {
+snn_status_t run_path(snn_conv* h, int path, const Geom& g, const Launch& l) {
   int launched = 0;
   cudaError_t e = cudaSuccess;
   switch (path) {
     case SNN_PATH_REUSE: e = reuse_forward(h->L, g, h->act_type, l, &launched); break;
     case SNN_PATH_DECODED: e = popc_forward(h->L, g, l, &launched); break;
-    case SNN_PATH_DECODED_TC:
-      e = tc_forward(h->L, g, h->act_type, l, &launched, h->tc_status_dev, variant >= 0 ? variant : tuned_variant(h, g));
+    case SNN_PATH_DECODED_TC: {
+      GroupDev* G = nullptr;
+      e = solo_group(h, g, &G, &launched);
+      if (e == cudaSuccess) e = tcg_forward(G, &l.act, &l.out, l.out_i32, l.stream, h->tc_status_dev, &launched);
       break;
+    }
     default: return fail(SNN_ERR_INVALID_ARG, "unknown path %d", path);
   }
   g_launches += launched;
@@ -161,8 +174,12 @@ snn_status_t check_forward_args(snn_conv* h, const void* act, int N, int H, int 
     pth = SNN_PATH_DECODED_TC;
     if (!path_ok(h, pth, *g))
       return fail(SNN_ERR_UNSUPPORTED, "packed-sign output needs the tensor-core path, which cannot run this layer");
-  } else if (pth == SNN_PATH_AUTO) pth = auto_path(h, *g);
-  else if (!path_ok(h, pth, *g))
+  } else if (pth == SNN_PATH_AUTO) {
+    pth = auto_path(h, *g);
+    if (pth < SNN_PATH_REUSE || !path_ok(h, pth, *g))
+      return fail(SNN_ERR_UNSUPPORTED, "no path can run this layer at this shape (act_type %d, C=%d K=%d, N=%d %dx%d)",
+                  h->act_type, h->C, h->K, N, H, W);
+  } else if (!path_ok(h, pth, *g))
     return fail(SNN_ERR_UNSUPPORTED, "path %d does not support this layer (act_type %d, C=%d K=%d)", pth, h->act_type,
                 h->C, h->K);
   *chosen = pth;
@@ -213,6 +230,8 @@ snn_status_t snn_conv_create(const snn_conv_desc_t* d, snn_conv_t** out) {
     if (d->codebook[j] >= 512) return fail(SNN_ERR_INVALID_ARG, "codebook[%d]=%u is not a 9-bit code", j, d->codebook[j]);
   for (int k = 0; k < d->c_out; ++k)
     if (!std::isfinite(d->alpha[k])) return fail(SNN_ERR_INVALID_ARG, "alpha[%d] is not finite", k);
+  for (int k = 0; d->shift && k < d->c_out; ++k)
+    if (!std::isfinite(d->shift[k])) return fail(SNN_ERR_INVALID_ARG, "shift[%d] is not finite", k);
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
     cudaGetLastError();
@@ -240,15 +259,10 @@ snn_status_t snn_conv_create(const snn_conv_desc_t* d, snn_conv_t** out) {
   alloc((void**)&h->L.idx, n_elem * 2);
   alloc((void**)&h->L.codebook, (size_t)T * 2);
   alloc((void**)&h->L.alpha, (size_t)h->K * 4);
+  alloc((void**)&h->L.shift, (size_t)h->K * 4);
   alloc((void**)&h->L.wplanes, (size_t)9 * g.Cw * h->K * 4);
   alloc((void**)&h->L.corr, (size_t)16 * h->K * 4);
   alloc((void**)&h->L.match9, (size_t)Tp * 512);
-  size_t tcw = tc_weight_bytes(g, h->act_type, &h->L.Kpad, &h->L.Cpad);
-  if (tcw) {
-    if (h->act_type == SNN_ACT_BIN) alloc((void**)&h->L.w8, tcw);
-    else alloc((void**)&h->L.w16, tcw);
-    alloc(&h->L.wcm, cm_weight_bytes(g, h->act_type));
-  }
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->host_stream, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&h->tc_status_host, sizeof(int), cudaHostAllocMapped);
   if (e == cudaSuccess) *h->tc_status_host = 0;
@@ -257,10 +271,11 @@ snn_status_t snn_conv_create(const snn_conv_desc_t* d, snn_conv_t** out) {
   if (e == cudaSuccess) e = cudaMemcpyAsync(d_stream, d->idx_packed, idx_bytes, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(h->L.codebook, d->codebook, (size_t)T * 2, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(h->L.alpha, d->alpha, (size_t)h->K * 4, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess)
+    e = d->shift ? cudaMemcpyAsync(h->L.shift, d->shift, (size_t)h->K * 4, cudaMemcpyHostToDevice, s)
+                 : cudaMemsetAsync(h->L.shift, 0, (size_t)h->K * 4, s);
   int launched = 0;
   if (e == cudaSuccess) e = decode_layer(h->L, d_stream, g, h->act_type, s, &launched);
-  if (e == cudaSuccess && tcw) e = tc_expand_weights(h->L, g, h->act_type, s, &launched);
-  if (e == cudaSuccess && tcw) e = cm_expand_weights(h->L, g, h->act_type, s, &launched);
   g_launches += launched;
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (d_stream) cudaFree(d_stream);
@@ -280,12 +295,11 @@ snn_status_t snn_conv_destroy(snn_conv_t* h) {
   cudaFree(h->L.idx);
   cudaFree(h->L.codebook);
   cudaFree(h->L.alpha);
+  cudaFree(h->L.shift);
   cudaFree(h->L.wplanes);
   cudaFree(h->L.corr);
   cudaFree(h->L.match9);
-  cudaFree(h->L.w8);
-  cudaFree(h->L.w16);
-  cudaFree(h->L.wcm);
+  for (auto& kv : h->solo) tcg_destroy(kv.second);
   cudaFree(h->stage_in);
   cudaFree(h->stage_out);
   if (h->tc_status_host) cudaFreeHost(h->tc_status_host);
@@ -396,16 +410,16 @@ snn_status_t snn_conv_tune(snn_conv_t* h, int32_t N, int32_t H, int32_t W, int32
   if (h->act_type == SNN_ACT_F16) cudaMemset(a, 0x3c, act_bytes(h, g));  // 0x3c3c = 1.0586 in fp16
   cudaStream_t s = h->host_stream;
   float best = -1.f;
-  int best_p = 0, best_v = 0;
+  int best_p = 0;
   snn_status_t st = SNN_OK;
-  auto time_one = [&](int pth, int variant, float* t_out) -> snn_status_t {
+  auto time_one = [&](int pth, float* t_out) -> snn_status_t {
     Launch l{a, o, 0, s};
     const int reps = 5;
     snn_status_t r = SNN_OK;
-    for (int w = 0; w < 2 && r == SNN_OK; ++w) r = run_path(h, pth, g, l, variant);
+    for (int w = 0; w < 2 && r == SNN_OK; ++w) r = run_path(h, pth, g, l);
     if (r != SNN_OK) return r;
     cudaEventRecord(e0, s);
-    for (int k = 0; k < reps && r == SNN_OK; ++k) r = run_path(h, pth, g, l, variant);
+    for (int k = 0; k < reps && r == SNN_OK; ++k) r = run_path(h, pth, g, l);
     cudaEventRecord(e1, s);
     cudaError_t ce = cudaEventSynchronize(e1);
     if (r != SNN_OK) return r;
@@ -418,15 +432,11 @@ snn_status_t snn_conv_tune(snn_conv_t* h, int32_t N, int32_t H, int32_t W, int32
   for (int pth = 1; pth <= 3 && st == SNN_OK; ++pth) {
     if (ms) ms[pth] = -1.f;
     if (!path_ok(h, pth, g)) continue;
-    const int nvar = pth == SNN_PATH_DECODED_TC ? tc_variant_count() : 1;
-    for (int v = 0; v < nvar && st == SNN_OK; ++v) {
-      if (pth == SNN_PATH_DECODED_TC && !tc_variant_ok(g, h->act_type, v)) continue;
-      float t = 0.f;
-      st = time_one(pth, pth == SNN_PATH_DECODED_TC ? v : -1, &t);
-      if (st != SNN_OK) break;
-      if (ms && (ms[pth] < 0.f || t < ms[pth])) ms[pth] = t;
-      if (best < 0.f || t < best) { best = t; best_p = pth; best_v = v; }
-    }
+    float t = 0.f;
+    st = time_one(pth, &t);
+    if (st != SNN_OK) break;
+    if (ms) ms[pth] = t;
+    if (best < 0.f || t < best) { best = t; best_p = pth; }
   }
   if (ms) ms[0] = best;
   cudaEventDestroy(e0);
@@ -437,12 +447,12 @@ snn_status_t snn_conv_tune(snn_conv_t* h, int32_t N, int32_t H, int32_t W, int32
   if (!best_p) return fail(SNN_ERR_UNSUPPORTED, "no path supports this layer");
   {
     std::lock_guard<std::mutex> lk(h->mu);
-    h->tuned[std::make_tuple(N, H, W)] = std::make_pair(best_p, best_p == SNN_PATH_DECODED_TC ? best_v : 0);
+    h->tuned[std::make_tuple(N, H, W)] = best_p;
   }
   if (best_path) *best_path = best_p;
   if (getenv("SNN_LOG"))
-    fprintf(stderr, "[snnconv] tuned C=%d K=%d tau=%d N=%d %dx%d -> path %d variant %d (%.4f ms)\n", h->C, h->K,
-            h->tau, N, H, W, best_p, best_v, best);
+    fprintf(stderr, "[snnconv] tuned C=%d K=%d tau=%d N=%d %dx%d -> path %d (%.4f ms)\n", h->C, h->K, h->tau, N, H, W,
+            best_p, best);
   return SNN_OK;
 }
 

@@ -23,14 +23,10 @@ struct LayerDev {
   uint16_t* idx = nullptr;       // [K][C] unpacked 0-based indices
   uint16_t* codebook = nullptr;  // [T] 9-bit codes
   float* alpha = nullptr;        // [K]
+  float* shift = nullptr;        // [K] added to alpha*S before the sign is taken (packed-sign output), zeros if none
   uint32_t* wplanes = nullptr;   // [9][Cw][K] bit-planes of the decoded +/-1 weights (bit = +1)
   int32_t* corr = nullptr;       // [16][K] border corrections, see snn_decode.cu
   uint8_t* match9 = nullptr;     // [T/16 or 1][512][16] matching-tap counts per (window, codebook kernel)
-  int8_t* w8 = nullptr;          // tensor-core operand: +/-1 int8 weights, tiled (snn_tc.cu)
-  uint16_t* w16 = nullptr;       // tensor-core operand: +/-1 fp16 weights, tiled (fp16 activations)
-  void* wcm = nullptr;           // channel-major tensor-core operand, [channel tile][K step][half][128][16 B] (snn_tcm.cu)
-  int Kpad = 0;                  // K rounded up for the tensor-core tiling
-  int Cpad = 0;                  // C rounded up for the tensor-core tiling
 };
 
 struct Launch {
@@ -51,31 +47,8 @@ cudaError_t popc_forward(const LayerDev& L, const Geom& g, const Launch& l, int*
 bool reuse_supported(const Geom& g, int act_type);
 cudaError_t reuse_forward(const LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched);
 
-bool tc_supported(const Geom& g, int act_type);
-// Tile variants of the tensor-core kernel (sub-tiles per CTA, weight-stage size, CTAs per SM);
-// variant 0 is the heuristic choice, the others are what snn_conv_tune sweeps.
-int tc_variant_count();
-bool tc_variant_ok(const Geom& g, int act_type, int variant);
-cudaError_t tc_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched, int* status_dev,
-                       int variant);
-size_t tc_weight_bytes(const Geom& g, int act_type, int* Kpad, int* Cpad);
-cudaError_t tc_expand_weights(const LayerDev& L, const Geom& g, int act_type, cudaStream_t s, int* launched);
-
-// Channel-major tensor-core kernel (weights in tensor memory); its variants are the positions
-// per tile.  tc_variant_count()/tc_variant_ok()/tc_forward() present them after the
-// position-major kernel's variants.
-int cm_variant_count();
-bool cm_variant_ok(const Geom& g, int act_type, int variant);
-cudaError_t cm_forward(LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched, int* status_dev,
-                       int variant);
-size_t cm_weight_bytes(const Geom& g, int act_type);
-cudaError_t cm_expand_weights(const LayerDev& L, const Geom& g, int act_type, cudaStream_t s, int* launched);
-
-// Tensor-core weight operand of the position-major layout with a caller-chosen channel block and
-// layout tile, written to `dst` (9 * n_chunks * Kpad * 16 bytes); used by the grouped kernel.
-cudaError_t tc_expand_weights_custom(const uint32_t* wplanes, void* dst, int C, int K, int Cw, int Kpad, int n_chunks,
-                                     int cb_chunks, int NtL, bool f16, cudaStream_t s);
-
+// The tensor-core kernel (snn_tcg.cu) runs one layer, several independent layers, or a chain of dependent
+// layers as ONE persistent launch; a single layer is a group of one.
 // Several independent problems in one persistent tensor-core launch (snn_tcg.cu).
 struct GroupDev;
 cudaError_t tcg_create(const LayerDev* const* layers, const Geom* geoms, int count, int act_type, cudaStream_t s,
@@ -84,6 +57,7 @@ cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, i
                         int* status_dev, int* launched);
 void tcg_destroy(GroupDev* G);
 int tcg_count(const GroupDev* G);
+bool tcg_supported(const Geom& g, int act_type);   // can the tensor-core kernel run this layer at this shape?
 
 cudaError_t microbench(int kind, double* rate);
 

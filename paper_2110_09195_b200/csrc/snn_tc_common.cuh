@@ -1,6 +1,5 @@
-// Device and host helpers shared by the two tensor-core kernels (position-major
-// and channel-major accumulators): PTX wrappers for mbarriers, bulk copies and
-// tcgen05, bit -> +/-1 expansion, exact division by run-time constants.
+// Device and host helpers of the tensor-core kernel: PTX wrappers for mbarriers,
+// bulk copies and tcgen05, bit -> e2m1 expansion, exact division by run-time constants.
 #pragma once
 #include <cuda_fp16.h>
 
@@ -103,15 +102,6 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
-// Shared -> global bulk copy in this thread's bulk group (16-byte aligned addresses, size a multiple of 16).
-__device__ __forceinline__ void bulk_s2g(const void* dst, uint32_t src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// all of this thread's bulk groups have read their shared-memory source
-__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-// all of this thread's bulk groups are complete (their writes done)
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void raise_status(int* status, int code) {
   *reinterpret_cast<volatile int*>(status) = code;
   __threadfence_system();
@@ -148,22 +138,14 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo, uint3
   return d;
 }
 
-template <bool F16>
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                       uint32_t accumulate) {
-  if (F16) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  } else {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  }
+// fp16 operands, fp32 accumulators: D[128 x N] (+)= A[128 x 16] * B[N x 16]^T
+__device__ __forceinline__ void mma_ss_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
 }
 
 // Block-scaled 4-bit MMA (e2m1 operands, one ue8m0 scale per 32 elements along K, fp32 accumulators):
@@ -207,56 +189,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
       : "r"(taddr)
       : "memory");
 }
-// 16 lanes x 32 columns in the 256-bit shape: with r = lane / 4 and q = lane % 4, register 4j + 2s + e holds
-// row (r + 8s) of the 16, column 8j + 2q + e  (j = 0..3, s = 0..1, e = 0..1).
-__device__ __forceinline__ void tmem_ld16x256(uint32_t taddr, uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr)
-      : "memory");
-}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// 4 activation bits -> 4 bytes of +1 (0x01) / -1 (0xff).  The multiply copies the nibble to
-// bit offsets 0/7/14/21 (no overlap for 4 bits), the mask keeps bit i at byte i, and
-// 0xffffffff - 0xfe*t turns each byte into 0x01 or 0xff without borrows between bytes.
-__device__ __forceinline__ uint32_t nibble_to_pm1(uint32_t nib) {
-  const uint32_t t = (nib * 0x00204081u) & 0x01010101u;
-  return t * 0xffffff02u + 0xffffffffu;
-}
-__device__ __forceinline__ uint32_t nibble_to_mask(uint32_t nib) {
-  const uint32_t t = (nib * 0x00204081u) & 0x01010101u;
-  return t * 0xffu;
-}
-
-// 32 activation bits -> 32 bytes of +1 / -1 (zero where the channel does not exist)
-__device__ __forceinline__ void expand_word(uint32_t bits, int channels_left, bool present, uint4& lo, uint4& hi) {
-  lo = make_uint4(0, 0, 0, 0);
-  hi = make_uint4(0, 0, 0, 0);
-  if (present && channels_left > 0) {
-    lo.x = nibble_to_pm1(bits & 15u);
-    lo.y = nibble_to_pm1((bits >> 4) & 15u);
-    lo.z = nibble_to_pm1((bits >> 8) & 15u);
-    lo.w = nibble_to_pm1((bits >> 12) & 15u);
-    hi.x = nibble_to_pm1((bits >> 16) & 15u);
-    hi.y = nibble_to_pm1((bits >> 20) & 15u);
-    hi.z = nibble_to_pm1((bits >> 24) & 15u);
-    hi.w = nibble_to_pm1(bits >> 28);
-    if (channels_left < 32) {
-      const uint32_t vm = (1u << channels_left) - 1u;
-      lo.x &= nibble_to_mask(vm & 15u);
-      lo.y &= nibble_to_mask((vm >> 4) & 15u);
-      lo.z &= nibble_to_mask((vm >> 8) & 15u);
-      lo.w &= nibble_to_mask((vm >> 12) & 15u);
-      hi.x &= nibble_to_mask((vm >> 16) & 15u);
-      hi.y &= nibble_to_mask((vm >> 20) & 15u);
-      hi.z &= nibble_to_mask((vm >> 24) & 15u);
-      hi.w &= nibble_to_mask(vm >> 28);
-    }
-  }
-}
 
 // 32 activation bits -> 32 e2m1 nibbles (16 bytes): +1.0 is 0x2, -1.0 is 0xA; channel c of the word sits in
 // nibble c (byte c/2, low nibble first).  A byte is looked up from its two bits with a byte permute whose
@@ -280,43 +213,19 @@ __device__ __forceinline__ uint4 expand_word_fp4(uint32_t bits, bool present) {
   return r;
 }
 
-// int32 -> float for |s| < 2^22 without the conversion unit (which handles only 16 lanes per SM
-// and clock and was the slowest step of the accumulator drain): adding s to the bit pattern of
-// 1.5 * 2^23 gives the float 1.5 * 2^23 + s exactly, and the subtraction is exact too.  The sums of
-// a 3x3 layer are bounded by 9 * c_in, so the launch plans require 9 * c_in < 2^22.
-__device__ __forceinline__ float small_int_to_float(uint32_t s) {
-  return __fadd_rn(__uint_as_float(0x4B400000u + s), -12582912.0f);
-}
-// Two accumulators -> two scaled outputs with the packed fp32 instructions (one add and one
-// multiply for the pair; each lane rounds exactly as the scalar instruction does):
-// F16 = false: a, b hold int32 sums (|s| < 2^22) and become (float)s * alpha; F16 = true: they
-// hold fp32 sums and become sum * alpha.
-template <bool F16>
+// Two fp32 accumulators times two channel scales with the packed fp32 multiply (each lane rounds exactly
+// as the scalar instruction does).
 __device__ __forceinline__ void scale_pair(uint32_t& a, uint32_t& b, float ax, float ay) {
   unsigned long long v, m;
   asm("mov.b64 %0, {%1, %2};" : "=l"(m) : "f"(ax), "f"(ay));
-  if (F16) {
-    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "r"(a), "r"(b));
-  } else {
-    unsigned long long c;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "r"(0x4B400000u + a), "r"(0x4B400000u + b));
-    asm("mov.b64 %0, {%1, %1};" : "=l"(c) : "f"(-12582912.0f));
-    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(v) : "l"(c));
-  }
+  asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "r"(a), "r"(b));
   asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(v) : "l"(m));
   asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
 }
 // 32 x 32 -> 64-bit product in one instruction (element offsets of pixels: both factors are non-negative 32-bit)
 __device__ __forceinline__ size_t wide_mul(uint32_t a, uint32_t b) { return (size_t)a * (size_t)b; }
 
-constexpr int kMaxChannelsSmallInt = ((1 << 22) - 1) / 9;
-
 static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
-
-static inline int env_int(const char* name, int dflt) {
-  const char* v = getenv(name);
-  return v ? atoi(v) : dflt;
-}
 
 static inline int sm_count() {
   static int sms = 0;
@@ -326,19 +235,6 @@ static inline int sm_count() {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148;
   }
   return sms;
-}
-
-// Channel blocks of the K loop: at most 8 chunks (128 int8 / 64 fp16 channels) each.  The
-// chunk count is even (an MMA consumes two); when no block size in 4..8 divides it, the
-// channels are padded with zeros to a multiple of 8 chunks.
-static inline void channel_blocks(int C, bool f16, int* n_chunks, int* cb_chunks) {
-  const int cpc = f16 ? 8 : 16;
-  const int raw = round_up(C, 2 * cpc) / cpc;
-  if (raw <= 8) { *n_chunks = raw; *cb_chunks = raw; return; }
-  for (int d = 8; d >= 4; d -= 2)
-    if (raw % d == 0) { *n_chunks = raw; *cb_chunks = d; return; }
-  *n_chunks = round_up(raw, 8);
-  *cb_chunks = 8;
 }
 
 }  // namespace

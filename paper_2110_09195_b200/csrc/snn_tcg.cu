@@ -39,9 +39,10 @@ namespace snn {
 namespace {
 
 // Operand modes of the kernel.  Binary activations run on 4-bit e2m1 operands (+1 / -1 / 0 are exact, the
-// block scales are all 1, fp32 accumulators hold the exact integer sums): an MMA then covers 64 input
-// channels in the time an int8 MMA covers 32.  The int8 mode is the same contraction with int32 accumulators.
-enum { M_I8 = 0, M_F16 = 1, M_FP4 = 2 };
+// block scales are all 1, and the fp32 accumulators hold the exact integer sums: |S| <= 9 * c_in < 2^24);
+// an MMA then covers 64 input channels in the time an 8-bit MMA covers 32.  fp16 activations run on fp16
+// operands.  Both accumulate in fp32.
+enum { M_F16 = 1, M_FP4 = 2 };
 constexpr int G_EW = 8;                       // epilogue warps = expander warps
 // Warps 13 and 17 stay idle: a warp's scheduler is warp % 4, and the MMA-issuing warp (1) then
 // shares its scheduler with two epilogue warps only instead of two epilogue and two expander warps.
@@ -50,7 +51,7 @@ constexpr int G_EXP_THREADS = 32 * G_EW;
 constexpr int G_EXP_ROWS = 3;                 // rows of a unit one expander thread loads together
 constexpr int G_EPI_PITCH = 128;
 constexpr int G_EPI_BYTES = G_EW * 32 * G_EPI_PITCH;
-constexpr int G_NA_MAX = 4, G_NS_MAX = 8;
+constexpr int G_NS_MAX = 8;
 constexpr uint32_t G_ACC_COLS = 256;          // tensor-memory columns of one accumulator buffer
 constexpr uint32_t G_ACC_COLS_FP4 = 240;      // 4-bit mode: columns 480..511 hold the (unit) block scales
 constexpr uint32_t G_SCALE_COL = 480;
@@ -63,6 +64,7 @@ constexpr uint32_t kGBSlot = 32 * 1024;            // bytes of a weight-stage sl
 struct GLayer {
   const uint8_t* wt;      // [layout tile][channel block][tap][chunk][NtL][16 B], owned by the group
   const float* alpha;
+  const float* shift;     // per-channel constant added to alpha*S before the sign is taken (packed-sign output)
   int N, H, W, C, K, Cw, stride, pad, Ho, Wo;
   int NtL, Nt;            // channels per layout tile of the weight operand / per tile
   int Hq, Wq;             // rows per image / row pitch of the flattened position space
@@ -121,14 +123,6 @@ __device__ __forceinline__ int g_position_to_pixel(const GLayer& L, uint32_t q, 
   return ((int)n * L.H + r) * L.W + c;
 }
 
-// one accumulator value (fp32, or int32 below 2^22 in magnitude) times the channel's scale: one rounding
-template <bool FACC>
-__device__ __forceinline__ uint32_t g_scale(uint32_t v, float a) {
-  return __float_as_uint(__fmul_rn(FACC ? __uint_as_float(v) : small_int_to_float(v), a));
-}
-// an fp32 accumulator that holds an integer, as that integer
-__device__ __forceinline__ uint32_t g_to_int(uint32_t v) { return (uint32_t)__float2int_rn(__uint_as_float(v)); }
-
 // first tile of problem L for this CTA (tiles then follow at a stride of the grid)
 __device__ __forceinline__ int g_first_tile(const GLayer& L) {
   return (int)__ldg(L.rank + blockIdx.x);
@@ -169,7 +163,7 @@ __device__ __forceinline__ bool g_issue_block(uint64_t a_unit, uint32_t wq, uint
             const uint64_t bdk = bd + (uint64_t)((uint32_t)k * b_step);
             const uint32_t accum = k == 0 ? acc : 1u;
             if (MODE == M_FP4) mma_ss_fp4(d0 + (uint32_t)mt * nt, ad, bdk, idesc, accum, sf, sf + 16);
-            else mma_ss<MODE == M_F16>(d0 + (uint32_t)mt * nt, ad, bdk, idesc, accum);
+            else mma_ss_f16(d0 + (uint32_t)mt * nt, ad, bdk, idesc, accum);
           }
         }
       }
@@ -188,7 +182,6 @@ template <int MODE>
 __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p) {
   constexpr bool F16 = MODE == M_F16;   // fp16 activations (copied, not expanded)
   constexpr bool FP4 = MODE == M_FP4;   // binary activations as e2m1 nibbles
-  constexpr bool FACC = MODE != M_I8;   // fp32 accumulators
   extern __shared__ __align__(128) uint8_t smem[];
   // carve-up: [NA activation slots][NS weight slots][epilogue tiles][pixel table][problem table][barriers, flags]
   uint8_t* a_smem = smem;
@@ -327,8 +320,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         // (4-bit mode: A/B format e2m1, scale format ue8m0, scale ids 0)
         const uint32_t idesc =
             F16 ? ((1u << 4) | ((uint32_t)(Nt >> 3) << 17) | ((128u >> 4) << 24))
-                : FP4 ? ((1u << 7) | (1u << 10) | ((uint32_t)(Nt >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24))
-                      : ((2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(Nt >> 3) << 17) | ((128u >> 4) << 24));
+                : ((1u << 7) | (1u << 10) | ((uint32_t)(Nt >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24));
         const uint64_t a_desc0 = make_desc(smem_u32(a_smem), (uint32_t)Rr * 16, 128);
         const uint64_t b_desc0 = make_desc(smem_u32(b_smem), (uint32_t)Nt * 16, 128);
         const uint32_t a_step = 2u * (uint32_t)Rr, b_step = 2u * (uint32_t)Nt;  // two chunks per MMA
@@ -395,6 +387,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       const GLayer& L = lay[l];
       const int Nt = L.Nt, MT = L.MT, K = L.K;
       const float* alpha = L.alpha;
+      const float* shift = L.shift;
       uint32_t* out32 = reinterpret_cast<uint32_t*>(p.out[l]);  // int32 and fp32 outputs share the layout
       const bool fast = ((K & 3) == 0) && ((Nt & 31) == 0);
       for (int tile = g_first_tile(L); tile < L.total_tiles; tile += G) {
@@ -446,9 +439,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 #pragma unroll
                   for (int e = 0; e < 32; ++e) {
                     const float a = co0 + e < K ? __ldg(alpha + co0 + e) : -1.f;  // a missing channel gives bit 0 ...
-                    const float s = co0 + e >= K ? 1.f  // ... through 1 * -1 < 0
-                                                 : FACC ? __uint_as_float(v[e]) : small_int_to_float(v[e]);
-                    word |= (__fmul_rn(s, a) >= 0.f ? 1u : 0u) << e;
+                    const float s = co0 + e < K ? __uint_as_float(v[e]) : 1.f;     // ... through 1 * -1 + 0 < 0
+                    const float t = co0 + e < K ? __ldg(shift + co0 + e) : 0.f;
+                    word |= (__fadd_rn(__fmul_rn(s, a), t) >= 0.f ? 1u : 0u) << e;
                   }
                   out32[wide_mul((uint32_t)pix, (uint32_t)Kw) + (uint32_t)(co0 >> 5)] = word;
                 }
@@ -472,8 +465,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 #pragma unroll
                   for (int e = 0; e < 16; ++e) {
                     const float a = co0 + e < K ? __ldg(alpha + co0 + e) : -1.f;
-                    const float s = co0 + e >= K ? 1.f : FACC ? __uint_as_float(v[e]) : small_int_to_float(v[e]);
-                    hw |= (__fmul_rn(s, a) >= 0.f ? 1u : 0u) << e;
+                    const float s = co0 + e < K ? __uint_as_float(v[e]) : 1.f;
+                    const float t = co0 + e < K ? __ldg(shift + co0 + e) : 0.f;
+                    hw |= (__fadd_rn(__fmul_rn(s, a), t) >= 0.f ? 1u : 0u) << e;
                   }
                   const size_t at = wide_mul((uint32_t)pix, (uint32_t)(2 * Kw)) + (uint32_t)(co0 >> 4);
                   if ((co0 >> 4) < 2 * Kw) out16[at] = (uint16_t)hw;
@@ -521,10 +515,10 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
               if (!p.out_i32) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                  scale_pair<FACC>(u[i].x, u[i].y, al.x, al.y);
-                  scale_pair<FACC>(u[i].z, u[i].w, al.z, al.w);
+                  scale_pair(u[i].x, u[i].y, al.x, al.y);
+                  scale_pair(u[i].z, u[i].w, al.z, al.w);
                 }
-              } else if (FACC) {
+              } else {
                 // int32 sums asked of fp32 accumulators: the sums are integers, the conversion is exact
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
@@ -558,10 +552,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 #pragma unroll
               for (int e = 0; e < 16; ++e) {
                 if (co0 + e < K) {
-                  if (p.out_i32) o[e] = FACC ? (uint32_t)__float2int_rn(__uint_as_float(v[e])) : v[e];
-                  else
-                    o[e] = __float_as_uint(__fmul_rn(FACC ? __uint_as_float(v[e]) : small_int_to_float(v[e]),
-                                                     __ldg(alpha + co0 + e)));
+                  if (p.out_i32) o[e] = (uint32_t)__float2int_rn(__uint_as_float(v[e]));
+                  else o[e] = __float_as_uint(__fmul_rn(__uint_as_float(v[e]), __ldg(alpha + co0 + e)));
                 }
               }
             }
@@ -600,12 +592,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         const uintptr_t addr = (uintptr_t)act;
         if (F16) vec = (addr & 15) == 0 && (C & 7) == 0;
         else if (FP4) vec = (addr & 7) == 0 && (Cw & 1) == 0;  // pairs of words (a block's first word is even)
-        else if (cb_chunks == 8) vec = (addr & 15) == 0 && (Cw & 3) == 0;
-        else if (cb_chunks == 4) vec = (addr & 7) == 0 && (Cw & 1) == 0;
         else vec = false;
       }
       const bool vec4 = FP4 && vec && ((uintptr_t)act & 15) == 0 && (Cw & 3) == 0 && (cb_chunks & 3) == 0;
-      const int nstep = cb_chunks / 2;  // pairs of chunks per unit
       for (int tile = g_first_tile(L); tile < total && !stop; tile += G) {
         const int mg = (int)fdiv((uint32_t)tile, dNt);
         const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
@@ -720,42 +709,6 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
                     }
                   }
                 }
-              } else {
-                // up to four 32-channel words per row and block, as one vector load when aligned
-                const int w0 = cb * nstep;
-                uint32_t bits[G_EXP_ROWS][4];
-#pragma unroll
-                for (int j = 0; j < G_EXP_ROWS; ++j) {
-                  bits[j][0] = bits[j][1] = bits[j][2] = bits[j][3] = 0;
-                  if (pix[j] >= 0 && w0 < Cw) {
-                    const uint32_t* src = (const uint32_t*)act + wide_mul((uint32_t)pix[j], (uint32_t)Cw) + w0;
-                    if (vec && nstep == 4) {
-                      const uint4 t = __ldg(reinterpret_cast<const uint4*>(src));
-                      bits[j][0] = t.x; bits[j][1] = t.y; bits[j][2] = t.z; bits[j][3] = t.w;
-                    } else if (vec && nstep == 2) {
-                      const uint2 t = __ldg(reinterpret_cast<const uint2*>(src));
-                      bits[j][0] = t.x; bits[j][1] = t.y;
-                    } else {
-#pragma unroll
-                      for (int k = 0; k < 4; ++k)
-                        if (k < nstep && w0 + k < Cw) bits[j][k] = __ldg(src + k);
-                    }
-                  }
-                }
-#pragma unroll
-                for (int j = 0; j < G_EXP_ROWS; ++j) {
-                  if (pix[j] != -2) {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                      if (k < nstep) {
-                        uint4 lo, hi;
-                        expand_word(bits[j][k], C - (w0 + k) * 32, pix[j] >= 0 && w0 + k < Cw, lo, hi);
-                        *reinterpret_cast<uint4*>(dst[j] + (size_t)(2 * k) * Rr * 16) = lo;
-                        *reinterpret_cast<uint4*>(dst[j] + (size_t)(2 * k + 1) * Rr * 16) = hi;
-                      }
-                    }
-                  }
-                }
               }
             }
           }
@@ -779,7 +732,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 
 // ------------------------------------------------------------------ host side
 struct GroupDev {
-  int count = 0, act_type = 0, mode = M_I8;
+  int count = 0, act_type = 0, mode = M_FP4;
   GLayer* layers_dev = nullptr;   // [count]
   uint8_t* weights = nullptr;     // the group's own weight operands, one after the other
   uint16_t* ranks = nullptr;      // [count][grid] tile assignment, see tcg_create
@@ -807,7 +760,7 @@ __global__ void g_expand_weights_kernel(const uint32_t* __restrict__ wplanes, ui
   r /= 9;
   int cb = (int)(r % n_cb), tile = (int)(r / n_cb);
   int co = tile * NtL + row;
-  constexpr int cpc = MODE == M_F16 ? 8 : MODE == M_FP4 ? 32 : 16;
+  constexpr int cpc = MODE == M_F16 ? 8 : 32;
   uint4 v = make_uint4(0, 0, 0, 0);
   if (co < K) {
     int ch0 = (cb * cb_chunks + c) * cpc;
@@ -818,14 +771,10 @@ __global__ void g_expand_weights_kernel(const uint32_t* __restrict__ wplanes, ui
 #pragma unroll
       for (int e = 0; e < 8; ++e)
         if (ch0 + e < C) w[e >> 1] |= (((bits >> e) & 1u) ? 0x3c00u : 0xbc00u) << (16 * (e & 1));  // +1.0 / -1.0
-    } else if (MODE == M_FP4) {
+    } else {
 #pragma unroll
       for (int e = 0; e < 32; ++e)
         if (ch0 + e < C) w[e >> 3] |= (((bits >> e) & 1u) ? 0x2u : 0xau) << (4 * (e & 7));         // e2m1 +1.0 / -1.0
-    } else {
-#pragma unroll
-      for (int e = 0; e < 16; ++e)
-        if (ch0 + e < C) w[e >> 2] |= (((bits >> e) & 1u) ? 0x01u : 0xffu) << (8 * (e & 3));       // +1 / -1
     }
     v = make_uint4(w[0], w[1], w[2], w[3]);
   }
@@ -839,19 +788,19 @@ cudaError_t g_expand_weights(int mode, const uint32_t* wplanes, void* dst, int C
   const int n_cb = n_chunks / cb_chunks;
   if (mode == M_F16)
     g_expand_weights_kernel<M_F16><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL);
-  else if (mode == M_FP4)
-    g_expand_weights_kernel<M_FP4><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL);
   else
-    g_expand_weights_kernel<M_I8><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL);
+    g_expand_weights_kernel<M_FP4><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL);
   return cudaGetLastError();
 }
+
+inline int g_mode_for(int act_type) { return act_type == SNN_ACT_F16 ? M_F16 : M_FP4; }
 
 // Cycles of one MMA of 128 positions x nt channels as measured on B200 (any operand type): half a cycle per
 // channel plus a constant that does not overlap the previous MMA.
 inline double g_mma_cycles(int nt) { return 0.5 * nt + 33.0; }
 
 bool g_plan_layer(const Geom& g, int mode, GLayer* L, int* n_chunks_out, int* Kpad_out) {
-  const int cpc = mode == M_F16 ? 8 : mode == M_FP4 ? 32 : 16;
+  const int cpc = mode == M_F16 ? 8 : 32;
   const int acc_cols = mode == M_FP4 ? (int)G_ACC_COLS_FP4 : (int)G_ACC_COLS;
   const int raw = round_up(g.C, 2 * cpc) / cpc;  // 16-byte chunks along the channels, even
   GLayer& o = *L;
@@ -867,11 +816,11 @@ bool g_plan_layer(const Geom& g, int mode, GLayer* L, int* n_chunks_out, int* Kp
   o.Qtot = (long long)g.N * o.Hq * o.Wq;
   if (g.N < 1) return false;
   if (o.Qtot + 1024 + o.halo >= (1ll << 31)) return false;  // positions are 32-bit in the kernel
-  if (g.C > kMaxChannelsSmallInt) return false;             // the drain's int -> float shortcut
+  if (g.C > (1 << 20)) return false;                        // 9 * c_in stays far below 2^24: exact fp32 sums
   if ((long long)g.N * g.H * g.W >= (1ll << 31) || (long long)g.N * g.Ho * g.Wo >= (1ll << 31)) return false;
   // layout tile of the weight operand = channels per tile: all of them up to 256; beyond that 256
   // when that pads little (fewer channel tiles re-expand the same activations), else 128
-  if (mode == M_FP4) o.NtL = g.K <= acc_cols ? round_up(g.K, 16) : 128;
+  if (mode == M_FP4) o.NtL = g.K <= acc_cols ? round_up(g.K, 16) : 128;   // (columns 480..511 hold the scales)
   else o.NtL = g.K <= 256 ? round_up(g.K, 16) : (round_up(g.K, 256) - g.K < 64 ? 256 : 128);
   o.Nt = o.NtL;
   const int Kpad = round_up(g.K, o.NtL);
@@ -914,7 +863,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
                        GroupDev** out, int* launched) {
   *out = nullptr;
   if (count < 1 || count > SNN_GROUP_MAX) return cudaErrorInvalidConfiguration;
-  const int mode = act_type == SNN_ACT_F16 ? M_F16 : (env_int("SNN_TCG_I8", 0) ? M_I8 : M_FP4);
+  const int mode = g_mode_for(act_type);
   GLayer host[SNN_GROUP_MAX];
   int n_chunks[SNN_GROUP_MAX], Kpad[SNN_GROUP_MAX];
   size_t w_off[SNN_GROUP_MAX], w_total = 0;
@@ -982,6 +931,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
     host[i].rank = G->ranks + (size_t)i * grid;
     host[i].wt = G->weights + w_off[i];
     host[i].alpha = Ls[i]->alpha;
+    host[i].shift = Ls[i]->shift;
     e = g_expand_weights(mode, Ls[i]->wplanes, G->weights + w_off[i], gs[i].C, gs[i].K, gs[i].Cw, Kpad[i],
                          n_chunks[i], host[i].cb_chunks, host[i].NtL, s);
     if (e == cudaSuccess) *launched += 1;
@@ -1024,6 +974,17 @@ void tcg_destroy(GroupDev* G) {
 
 int tcg_count(const GroupDev* G) { return G->count; }
 
+bool tcg_supported(const Geom& g, int act_type) {
+  GLayer L;
+  int n_chunks = 0, Kpad = 0;
+  if (!g_plan_layer(g, g_mode_for(act_type), &L, &n_chunks, &Kpad)) return false;
+  // one problem alone: three activation slots, the fixed parts and three weight slots must fit
+  const size_t unit = (((size_t)L.n_planes * L.cb_chunks * L.Rr * 16) + 127) & ~(size_t)127;
+  const size_t pix = (((size_t)L.n_planes * L.Rr * 4) + 127) & ~(size_t)127;
+  const size_t fixed = (size_t)G_EPI_BYTES + pix + 256 + kGTail;
+  return 2 * unit + fixed + 3 * (size_t)kGBSlot <= kGSmemBudget;
+}
+
 cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, int out_i32, cudaStream_t s,
                         int* status_dev, int* launched) {
   GParams p = G->p;
@@ -1050,14 +1011,10 @@ cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, i
     static unsigned long long done = 0;
     e = allow_max_smem(tcg_conv_kernel<M_F16>, &done);
     if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<M_F16>, p);
-  } else if (G->mode == M_FP4) {
+  } else {
     static unsigned long long done = 0;
     e = allow_max_smem(tcg_conv_kernel<M_FP4>, &done);
     if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<M_FP4>, p);
-  } else {
-    static unsigned long long done = 0;
-    e = allow_max_smem(tcg_conv_kernel<M_I8>, &done);
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<M_I8>, p);
   }
   if (e != cudaSuccess) return e;
   *launched += 1;

@@ -94,6 +94,37 @@ def test_group_stack_small_batch(snn, oracle_mod, net, cfg):
     check_bin_group(snn, oracle_mod, [(s, 2) for s in wk.layers], wk.tau, 31 + cfg, repeats=2)
 
 
+def test_group_of_32_members(snn, oracle_mod):
+    """The largest group the library takes (SNN_GROUP_MAX): the 32 layers of the ResNet-34-shaped stack, batch 2."""
+    wk = wl.get_workload("resnet34")
+    assert len(wk.layers) == 32
+    check_bin_group(snn, oracle_mod, [(s, 2) for s in wk.layers], wk.tau, 35)
+
+
+def test_group_benchmark_step_at_full_size(snn, oracle_mod):
+    """Exactly what bench.py times: the 16 ResNet-18-shaped layers at batch 64 with the benchmark's seeds, as one
+    grouped launch.  fp32 outputs of every member against the oracle, element by element."""
+    wk = wl.get_workload("resnet18")
+    layers, acts, refs = [], [], []
+    for i, shape in enumerate(wk.layers):
+        seed = wl.layer_seed(wk.config, i)
+        p = wl.draw_layer_params(shape, wk.tau, seed)
+        packed = wl.pack_activation_bits(wl.draw_activation_bits(shape, wk.batch, seed))
+        refs.append(oracle_mod.conv_bin(p.codebook, wk.tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out, shape.stride,
+                                        shape.pad, packed)[1])
+        layers.append(snn.SnnConv(shape.c_in, shape.c_out, wk.tau, p.codebook, p.idx_packed, p.alpha, shape.stride,
+                                  shape.pad, snn.ACT_BIN))
+        acts.append(torch.from_numpy(packed.view(np.int32)).cuda())
+    group = snn.SnnConvGroup(layers, [(wk.batch, s.h, s.w) for s in wk.layers])
+    outs = group.forward(acts, out_type=snn.OUT_F32)
+    torch.cuda.synchronize()
+    for i, y_ref in enumerate(refs):
+        assert (outs[i].cpu().numpy() == y_ref).all(), f"layer {i}"
+    group.destroy()
+    for l in layers:
+        l.destroy()
+
+
 def test_group_many_tiles_per_cta(snn, oracle_mod):
     """More tiles than twice the CTAs in several members: every ring (activation units, weight
     stages, accumulator buffers) wraps around many times and carries over between members."""
@@ -160,8 +191,11 @@ def test_group_argument_errors(snn):
     b.destroy()
 
 
-def _pack_signs(y):
-    """Oracle-side packing of sign(Y) (Y >= 0 -> bit 1) along c_out into little-endian uint32 words."""
+def _pack_signs(y, shift=None):
+    """Oracle-side packing of the thresholded sign (fl(Y + shift) >= 0 -> bit 1, in fp32) along c_out into
+    little-endian uint32 words.  Y is the oracle's fp32 output fl(alpha * S)."""
+    if shift is not None:
+        y = (y.astype(np.float32) + shift.astype(np.float32)[None, None, None, :]).astype(np.float32)
     bits = (y >= 0)
     n, h, w, k = bits.shape
     kw = (k + 31) // 32
@@ -208,6 +242,60 @@ def test_group_packed_sign_outputs(snn, oracle_mod):
         bad = np.argwhere(got != ref)
         assert bad.size == 0, f"member {i} {members[i][0]}: {len(bad)} words differ, first at {bad[0]}: " \
                               f"{got[tuple(bad[0])]:#x} vs {ref[tuple(bad[0])]:#x}"
+    group.destroy()
+    for l in layers:
+        l.destroy()
+
+
+def test_group_packed_signs_with_channel_thresholds(snn, oracle_mod):
+    """SNN_OUT_BITS with a per-channel shift (the folded batch-normalisation threshold): bit = fl(fl(alpha*S) + shift) >= 0.
+    Random shifts, negative scales, and channels whose scale is a power of two with a shift of minus a small
+    multiple of it, so that many sums land exactly on zero (which must give bit 1) or one step beside it."""
+    members = [
+        (wl.LayerShape(33, 7, 9, 11, 1, 1), 3),
+        (wl.LayerShape(70, 37, 13, 6, 2, 1), 2),
+        (wl.LayerShape(64, 48, 5, 8, 1, 0), 2),
+        (wl.LayerShape(96, 130, 3, 17, 1, 1), 1),
+        (wl.LayerShape(64, 64, 20, 20, 1, 1), 4),
+        (wl.LayerShape(128, 256, 12, 12, 2, 1), 3),
+        (wl.LayerShape(2, 40, 6, 6, 1, 1), 2),
+        (wl.LayerShape(8, 72, 9, 9, 1, 1), 2),
+    ]
+    layers, acts, refs, yrefs, zeros = [], [], [], [], 0
+    for i, (shape, n) in enumerate(members):
+        p = wl.draw_layer_params(shape, 5, 161 + i)
+        rng = np.random.default_rng(900 + i)
+        alpha = p.alpha.copy()
+        alpha[::3] *= -1.0
+        shift = rng.normal(0.0, 3.0, size=shape.c_out).astype(np.float32)
+        ks = np.array([0, 2, -2, 4, 1, 3, -1, 6], dtype=np.float32)
+        sel = np.arange(1, shape.c_out, 5)
+        alpha[sel] = np.where(np.arange(sel.size) % 2 == 0, 0.5, -0.25).astype(np.float32)
+        shift[sel] = -alpha[sel] * ks[np.arange(sel.size) % ks.size]
+        packed = wl.pack_activation_bits(wl.draw_activation_bits(shape, n, 161 + i))
+        _, y_ref = oracle_mod.conv_bin(p.codebook, 5, p.idx_packed, alpha, shape.c_in, shape.c_out, shape.stride,
+                                       shape.pad, packed)
+        zeros += int(((y_ref + shift[None, None, None, :]).astype(np.float32) == 0).sum())
+        refs.append(_pack_signs(y_ref, shift))
+        yrefs.append(y_ref)
+        layers.append(snn.SnnConv(shape.c_in, shape.c_out, 5, p.codebook, p.idx_packed, alpha, shape.stride,
+                                  shape.pad, snn.ACT_BIN, shift=shift))
+        acts.append(torch.from_numpy(packed.view(np.int32)).cuda())
+    assert zeros > 100, "the inputs were meant to land many sums exactly on the threshold"
+    group = snn.SnnConvGroup(layers, [(n, s.h, s.w) for s, n in members])
+    guarded = [_guarded(r.shape, torch.int32) for r in refs]
+    group.forward(acts, [g[1] for g in guarded], snn.OUT_BITS)
+    torch.cuda.synchronize()
+    for i, ref in enumerate(refs):
+        got = guarded[i][1].cpu().numpy().view(np.uint32)
+        assert _intact(guarded[i][0], ref.size), f"member {i}: canary overwritten"
+        bad = np.argwhere(got != ref)
+        assert bad.size == 0, f"member {i} {members[i][0]}: {len(bad)} words differ, first at {bad[0]}"
+        # the single-layer entry point gives the same words
+        one = layers[i].forward(acts[i], out_type=snn.OUT_BITS)
+        assert (one.cpu().numpy().view(np.uint32) == ref).all(), f"member {i} through snn_conv_forward"
+    # fp32 outputs ignore the shift
+    assert (layers[0].forward(acts[0], out_type=snn.OUT_F32).cpu().numpy() == yrefs[0]).all()
     group.destroy()
     for l in layers:
         l.destroy()
@@ -274,10 +362,10 @@ def test_chained_layers_through_packed_signs(snn, oracle_mod):
     (33, 7, 9, 11, 1, 1, 3), (70, 37, 13, 6, 2, 1, 2), (64, 48, 5, 8, 1, 0, 2), (96, 130, 3, 17, 1, 1, 1),
     (40, 300, 6, 5, 1, 1, 2), (64, 64, 56, 56, 1, 1, 6), (128, 256, 12, 12, 2, 1, 3), (512, 512, 7, 7, 1, 1, 8),
 ])
-def test_single_layer_packed_sign_outputs(snn, oracle_mod, monkeypatch, c_in, c_out, h, w, stride, pad, n):
-    """SNN_OUT_BITS through snn_conv_forward (tensor-core path: tuned or heuristic full-size tiles, and
-    the half-size CTAs), through snn_conv_forward_host, and after tuning (a tuned channel-major tile
-    must not be used for it): bit-exact against the oracle's outputs."""
+def test_single_layer_packed_sign_outputs(snn, oracle_mod, c_in, c_out, h, w, stride, pad, n):
+    """SNN_OUT_BITS through snn_conv_forward, through snn_conv_forward_host, and after tuning (whatever
+    path the tuner picked for fp32 outputs, packed signs come from the tensor-core path): bit-exact
+    against the oracle's outputs."""
     shape = wl.LayerShape(c_in, c_out, h, w, stride, pad)
     p = wl.draw_layer_params(shape, 5, 91)
     alpha = p.alpha.copy()
@@ -287,17 +375,11 @@ def test_single_layer_packed_sign_outputs(snn, oracle_mod, monkeypatch, c_in, c_
     ref = _pack_signs(y_ref)
     layer = snn.SnnConv(c_in, c_out, 5, p.codebook, p.idx_packed, alpha, stride, pad, snn.ACT_BIN)
     act = torch.from_numpy(packed.view(np.int32)).cuda()
-    for variant in (None, 22, 25, 17):
-        if variant is None:
-            monkeypatch.delenv("SNN_TC_VARIANT", raising=False)
-        else:
-            monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
-        flat, out = _guarded(ref.shape, torch.int32)
-        layer.forward(act, out, snn.OUT_BITS)
-        torch.cuda.synchronize()
-        assert _intact(flat, ref.size), f"variant {variant}: canary overwritten"
-        assert (out.cpu().numpy().view(np.uint32) == ref).all(), f"variant {variant}"
-    monkeypatch.delenv("SNN_TC_VARIANT", raising=False)
+    flat, out = _guarded(ref.shape, torch.int32)
+    layer.forward(act, out, snn.OUT_BITS)
+    torch.cuda.synchronize()
+    assert _intact(flat, ref.size), "canary overwritten"
+    assert (out.cpu().numpy().view(np.uint32) == ref).all()
     host = layer.forward_host(torch.from_numpy(packed.view(np.int32)).pin_memory(), out_type=snn.OUT_BITS)
     assert (host.numpy().view(np.uint32) == ref).all()
     layer.tune(n, h, w)

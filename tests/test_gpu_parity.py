@@ -209,89 +209,57 @@ def test_tensor_core_path_runs_the_stack_shapes(snn):
         layer.destroy()
 
 
-@pytest.mark.parametrize("c_in,c_out,h,w,stride", [(64, 64, 20, 20, 1), (256, 128, 9, 9, 1), (128, 256, 12, 12, 2)])
-def test_tensor_core_tile_variants(snn, oracle_mod, monkeypatch, c_in, c_out, h, w, stride):
-    """Every tile shape of the position-major kernel the tuner may pick (sub-tiles per CTA,
-    weight-stage size) gives the same sums."""
-    shape = wl.LayerShape(c_in, c_out, h, w, stride, 1)
-    for mt in (1, 2, 4):
-        for kb in (16, 32, 64):
-            monkeypatch.setenv("SNN_TC_MT", str(mt))
-            monkeypatch.setenv("SNN_TC_STAGE_KB", str(kb))
-            p = wl.draw_layer_params(shape, 5, 77)
-            layer = snn.SnnConv(c_in, c_out, 5, p.codebook, p.idx_packed, p.alpha, stride, 1)
-            ok = layer.path_supported(snn.PATH_DECODED_TC, 3, h, w)
-            layer.destroy()
-            if ok:
-                check_bin_layer(snn, oracle_mod, shape, 5, 3, 77, paths=[snn.PATH_DECODED_TC])
-
-
-CM_SHAPES = [
-    (64, 64, 20, 20, 1, 3),      # resident weights, several tiles per CTA
-    (16, 16, 8, 8, 1, 2),        # one K step per tap, channels far below one tile
-    (256, 128, 9, 9, 1, 3),      # streamed weights, two channel blocks
+TC_SHAPES = [
+    (64, 64, 20, 20, 1, 3),      # one K step per tap, several tiles per CTA
+    (16, 16, 8, 8, 1, 2),        # channels far below one K step and one tile
+    (256, 128, 9, 9, 1, 3),      # eight 32-channel chunks in one block
     (128, 256, 12, 12, 2, 3),    # stride 2 (four parity planes), two channel tiles
     (200, 130, 7, 5, 1, 2),      # ragged channels in and out
-    (1056, 48, 9, 8, 2, 1),      # padded channel blocks
-    (512, 512, 7, 7, 1, 4),      # deep layer: 144 K steps, four channel tiles
+    (1056, 48, 9, 8, 2, 1),      # several channel blocks, padded
+    (512, 512, 7, 7, 1, 4),      # deep layer: two channel blocks, four channel tiles
+    (96, 240, 6, 6, 1, 2),       # the widest single channel tile of the 4-bit mode
+    (64, 248, 6, 6, 1, 2),       # just beyond it: two tiles, the second mostly padding
 ]
 
 
-@pytest.mark.parametrize("c_in,c_out,h,w,stride,n", CM_SHAPES)
-def test_channel_major_variants(snn, oracle_mod, monkeypatch, c_in, c_out, h, w, stride, n):
-    """The channel-major tensor-core kernel (weights in tensor memory) at every tile width."""
+@pytest.mark.parametrize("c_in,c_out,h,w,stride,n", TC_SHAPES)
+def test_tensor_core_shapes(snn, oracle_mod, c_in, c_out, h, w, stride, n):
+    """The tensor-core path alone (4-bit e2m1 operands, fp32 accumulators) on shapes that exercise its
+    channel blocks, channel tiles and parity planes; sums must be exact."""
     shape = wl.LayerShape(c_in, c_out, h, w, stride, 1)
-    ran = 0
-    for variant in range(16, 22):
-        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
-        check_bin_layer(snn, oracle_mod, shape, 5, n, 91, paths=[snn.PATH_DECODED_TC])
-        ran += 1
-    assert ran == 6
+    ran = check_bin_layer(snn, oracle_mod, shape, 5, n, 91, paths=[snn.PATH_DECODED_TC])
+    assert ran == [snn.PATH_DECODED_TC]
 
 
-def test_channel_major_many_tiles(snn, oracle_mod, monkeypatch):
-    """More tiles than CTAs: both accumulator buffers, ring wrap-around, streamed weights over
-    several tiles of one CTA."""
-    for variant, shape, n in [(16, wl.LayerShape(128, 128, 28, 28, 1, 1), 40), (20, wl.LayerShape(64, 64, 56, 56, 1, 1), 8),
-                              (17, wl.LayerShape(256, 256, 14, 14, 1, 1), 48)]:
-        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
-        check_bin_layer(snn, oracle_mod, shape, 5, n, 93, paths=[snn.PATH_DECODED_TC])
-
-
-HALF_VARIANTS = range(22, 30)  # position-major kernel, two half-size CTAs per SM
-
-
-@pytest.mark.parametrize("c_in,c_out,h,w,stride,n", CM_SHAPES)
-def test_half_size_cta_variants(snn, oracle_mod, monkeypatch, c_in, c_out, h, w, stride, n):
-    """The position-major kernel as CTAs of half an SM's shared and tensor memory (four epilogue and
-    four expander warps), at every tile and weight-stage size the tuner may pick."""
-    shape = wl.LayerShape(c_in, c_out, h, w, stride, 1)
-    for variant in HALF_VARIANTS:
-        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
-        check_bin_layer(snn, oracle_mod, shape, 5, n, 97, paths=[snn.PATH_DECODED_TC])
-
-
-def test_half_size_cta_many_tiles(snn, oracle_mod, monkeypatch):
-    """More tiles than CTAs with two CTAs per SM: both accumulator buffers, ring wrap-around, resident and
-    streamed weights, a channel tile narrower than the weight operand's layout tile."""
-    for variant, shape, n in [(22, wl.LayerShape(128, 128, 28, 28, 1, 1), 40), (25, wl.LayerShape(64, 64, 56, 56, 1, 1), 8),
-                              (24, wl.LayerShape(256, 256, 14, 14, 1, 1), 48), (23, wl.LayerShape(512, 512, 7, 7, 1, 1), 64),
-                              (26, wl.LayerShape(64, 128, 56, 56, 2, 1), 6)]:
-        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
+def test_tensor_core_many_tiles(snn, oracle_mod):
+    """More tiles than CTAs: both accumulator buffers, ring wrap-around, weight stages streamed over
+    several tiles of one CTA, and a tile assignment with a ragged last round."""
+    for shape, n in [(wl.LayerShape(128, 128, 28, 28, 1, 1), 40), (wl.LayerShape(64, 64, 56, 56, 1, 1), 8),
+                     (wl.LayerShape(256, 256, 14, 14, 1, 1), 48), (wl.LayerShape(512, 512, 7, 7, 1, 1), 64),
+                     (wl.LayerShape(64, 128, 56, 56, 2, 1), 6)]:
         check_bin_layer(snn, oracle_mod, shape, 5, n, 99, paths=[snn.PATH_DECODED_TC])
 
 
-def test_half_size_cta_fp16(snn, oracle_mod, monkeypatch):
-    for variant in (22, 23, 26):
-        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
-        for shape, n in [(wl.LayerShape(64, 64, 14, 14, 1, 1), 3), (wl.LayerShape(136, 72, 9, 7, 2, 1), 2)]:
-            ran = check_f16_layer(snn, oracle_mod, shape, 5, n, 95)
-            assert snn.PATH_DECODED_TC in ran
+def test_tensor_core_fp16(snn, oracle_mod):
+    for shape, n in [(wl.LayerShape(64, 64, 14, 14, 1, 1), 3), (wl.LayerShape(136, 72, 9, 7, 2, 1), 2),
+                     (wl.LayerShape(128, 128, 28, 28, 1, 1), 24)]:
+        ran = check_f16_layer(snn, oracle_mod, shape, 5, n, 95)
+        assert snn.PATH_DECODED_TC in ran
 
 
-def test_channel_major_fp16(snn, oracle_mod, monkeypatch):
-    for variant in (16, 17, 18):
-        monkeypatch.setenv("SNN_TC_VARIANT", str(variant))
-        for shape, n in [(wl.LayerShape(64, 64, 14, 14, 1, 1), 3), (wl.LayerShape(136, 72, 9, 7, 2, 1), 2)]:
-            ran = check_f16_layer(snn, oracle_mod, shape, 5, n, 95)
-            assert snn.PATH_DECODED_TC in ran
+def test_auto_refuses_a_layer_no_path_can_run(snn):
+    """fp16 activations run on the tensor-core path only; a map so wide that one activation unit no longer
+    fits shared memory must be refused (status UNSUPPORTED), by name and by AUTO, with nothing launched."""
+    shape = wl.LayerShape(16, 16, 3, 700, 1, 1)
+    p = wl.draw_layer_params(shape, 5, 7)
+    layer = snn.SnnConv(16, 16, 5, p.codebook, p.idx_packed, p.alpha, act_type=snn.ACT_F16)
+    assert not layer.path_supported(snn.PATH_DECODED_TC, 1, 3, 700)
+    act = torch.zeros((1, 3, 700, 16), dtype=torch.float16, device="cuda")
+    before = snn.kernel_launches()
+    for path in (snn.PATH_AUTO, snn.PATH_DECODED_TC, snn.PATH_DECODED, snn.PATH_REUSE):
+        with pytest.raises(snn.SnnError) as ei:
+            layer.forward(act, path=path)
+        assert ei.value.status == 2
+    assert snn.kernel_launches() == before
+    assert layer.chosen_path(1, 3, 700) == snn.PATH_AUTO   # "none"
+    layer.destroy()
