@@ -186,6 +186,41 @@ SNN_API snn_status_t snn_conv_group_forward(snn_conv_group_t* g, const void* con
 SNN_API snn_status_t snn_conv_group_destroy(snn_conv_group_t* g);
 
 /*
+ * A stack of layers that feed one another, run as ONE persistent tensor-core launch.
+ * The paper times whole networks (Sec. 5.3, Table 4); in a binary network layer i + 1
+ * consumes sign(a^i) (Algorithm 1, forward step), so the members of a stack are chained
+ * through their packed thresholded signs (SNN_OUT_BITS: bit = fl(fl(alpha*S) + shift) >= 0,
+ * shift standing for the batch normalisation / Hardtanh between two binary layers, Sec. 5):
+ * member i writes them into a buffer the stack owns and member i + 1 reads them as its
+ * binary input.  Shortcut additions are not part of the path.  Inside the launch a tile of
+ * member i + 1 starts as soon as the tiles of member i that hold its input pixels are
+ * complete (per-tile completion counters in device memory, every wait bounded); there is
+ * no grid-wide step between layers.
+ *
+ * snn_conv_stack_create: `layers` are `count` (1..SNN_GROUP_MAX) handles with binary
+ * activations on one device whose shapes follow from one another (c_in of member i + 1 =
+ * c_out of member i, its input map = member i's output map); N, H, W fix the input of
+ * member 0.  The handles must outlive the stack.  The stack owns the buffers between its
+ * members, the counters and its tiled weight operands.  Errors: INVALID_ARG (null, count,
+ * fp16 activations, shapes that do not chain, mixed devices), UNSUPPORTED (a member the
+ * tensor-core path cannot run), CUDA, OOM.
+ *
+ * snn_conv_stack_forward: act_dev is member 0's input (DEVICE, binary layout), out_dev the
+ * last member's output (DEVICE) of type out_type (SNN_OUT_F32, SNN_OUT_I32 or SNN_OUT_BITS);
+ * both 16-byte aligned, neither kept.  Asynchronous on cuda_stream; allocates nothing.  Calls
+ * on one stack must not overlap on the GPU (they share the buffers and counters).  All CTAs
+ * of the launch must be resident together, which the launch checks (CUDA error otherwise).
+ * Errors: INVALID_ARG, TIMEOUT (an earlier launch gave up a bounded wait), CUDA.
+ */
+typedef struct snn_conv_stack snn_conv_stack_t; /* opaque; owned by the library */
+SNN_API snn_status_t snn_conv_stack_create(snn_conv_t* const* layers, int32_t count, int32_t N, int32_t H, int32_t W,
+                                           snn_conv_stack_t** out);
+SNN_API snn_status_t snn_conv_stack_forward(snn_conv_stack_t* s, const void* act_dev, void* out_dev, int32_t out_type,
+                                            void* cuda_stream);
+/* Frees the stack and its device buffers (not the member handles).  NULL is a no-op. */
+SNN_API snn_status_t snn_conv_stack_destroy(snn_conv_stack_t* s);
+
+/*
  * Forward pass for callers that must not allocate device memory.  (The paper has
  * no counterpart to this entry point; it exists for how the library is embedded.)
  *

@@ -48,6 +48,12 @@ def _load():
         lib.snn_oracle_conv_bin.argtypes = [vp, ci, vp, vp, ci, ci, ci, ci, vp, ci, ci, ci, vp, vp]
         lib.snn_oracle_conv_f16.restype = ci
         lib.snn_oracle_conv_f16.argtypes = [vp, ci, vp, vp, ci, ci, ci, ci, vp, ci, ci, ci, vp]
+        lib.snn_oracle_decode1x1.restype = ci
+        lib.snn_oracle_decode1x1.argtypes = [vp, ci, vp, ci, ci, vp]
+        lib.snn_oracle_conv1x1_bin.restype = ci
+        lib.snn_oracle_conv1x1_bin.argtypes = [vp, ci, vp, vp, ci, ci, ci, vp, ci, ci, ci, vp, vp]
+        lib.snn_oracle_conv1x1_f16.restype = ci
+        lib.snn_oracle_conv1x1_f16.argtypes = [vp, ci, vp, vp, ci, ci, ci, vp, ci, ci, ci, vp]
         _lib = lib
     return _lib
 
@@ -153,4 +159,79 @@ def conv_bin_shared_order(codebook, tau, idx, c_in, c_out, stride, pad, act_bits
     for co in range(c_out):
         for ci in range(c_in):
             s[..., co] += p[..., ci, idx[co, ci]]
+    return s
+
+
+# ---------------------------------------------------------------------------------------------
+# 1x1 extension (appendix "Extending to Bottleneck with 1x1 Kernels"): 8-input-channel +/-1 vectors
+# ---------------------------------------------------------------------------------------------
+
+def out_hw1x1(h: int, w: int, stride: int):
+    if stride < 1 or h < 1 or w < 1:
+        raise ValueError("bad stride / map size")
+    return (h - 1) // stride + 1, (w - 1) // stride + 1
+
+
+def decode_weights1x1(codebook, tau: int, idx_packed, c_in: int, c_out: int) -> np.ndarray:
+    """+/-1 weights (c_out, c_in) int8 of a 1x1 layer from its stored form: tau-bit indices of 8-channel vectors."""
+    cb = np.ascontiguousarray(codebook, dtype=np.uint16)
+    ip = np.ascontiguousarray(idx_packed, dtype=np.uint8)
+    assert cb.size == (1 << tau) and c_in % 8 == 0
+    assert ip.size >= (c_out * (c_in // 8) * tau + 7) // 8
+    w = np.empty((c_out, c_in), dtype=np.int8)
+    rc = _load().snn_oracle_decode1x1(_ptr(cb), tau, _ptr(ip), c_in, c_out, _ptr(w))
+    if rc:
+        raise ValueError(f"oracle decode1x1 failed rc={rc}")
+    return w
+
+
+def conv1x1_bin(codebook, tau, idx_packed, alpha, c_in, c_out, stride, act_packed):
+    """Binary-activation sub-bit 1x1 conv.  Returns (S int32, Y float32), both (N, Ho, Wo, c_out)."""
+    cb, ip, al = _prep(codebook, idx_packed, alpha)
+    act = np.ascontiguousarray(act_packed, dtype=np.uint32)
+    n, h, w, cw = act.shape
+    assert cw == (c_in + 31) // 32 and cb.size == (1 << tau) and al.size == c_out
+    ho, wo = out_hw1x1(h, w, stride)
+    s = np.empty((n, ho, wo, c_out), dtype=np.int32)
+    y = np.empty((n, ho, wo, c_out), dtype=np.float32)
+    rc = _load().snn_oracle_conv1x1_bin(_ptr(cb), tau, _ptr(ip), _ptr(al), c_in, c_out, stride, _ptr(act), n, h, w,
+                                        _ptr(s), _ptr(y))
+    if rc:
+        raise ValueError(f"oracle conv1x1_bin failed rc={rc}")
+    return s, y
+
+
+def conv1x1_f16(codebook, tau, idx_packed, alpha, c_in, c_out, stride, act_f16):
+    """Weights-only 1x1 variant: fp16 activations, double accumulation.  Returns Y float32."""
+    cb, ip, al = _prep(codebook, idx_packed, alpha)
+    act = np.ascontiguousarray(act_f16, dtype=np.float16)
+    n, h, w, c = act.shape
+    assert c == c_in and cb.size == (1 << tau) and al.size == c_out
+    ho, wo = out_hw1x1(h, w, stride)
+    y = np.empty((n, ho, wo, c_out), dtype=np.float32)
+    rc = _load().snn_oracle_conv1x1_f16(_ptr(cb), tau, _ptr(ip), _ptr(al), c_in, c_out, stride,
+                                        _ptr(act.view(np.uint16)), n, h, w, _ptr(y))
+    if rc:
+        raise ValueError(f"oracle conv1x1_f16 failed rc={rc}")
+    return y
+
+
+def conv1x1_shared_order(codebook, tau, idx, c_in, c_out, stride, act_bits):
+    """The shared computation carried over to 1x1 layers (appendix): first the dot product of every group of
+    8 input channels with each of the 2^tau codebook vectors (P), then for each output channel the sum, over
+    the groups, of the entry its index selects.  idx is the (c_out, c_in/8) integer array, act_bits the
+    (N, H, W, C) 0/1 array.  Returns S int64 (N, Ho, Wo, c_out)."""
+    codebook = np.asarray(codebook, dtype=np.int64)
+    idx = np.asarray(idx, dtype=np.int64)
+    a = (np.asarray(act_bits, dtype=np.int64) * 2 - 1)[:, ::stride, ::stride, :]
+    n, ho, wo, c = a.shape
+    g = c // 8
+    assert c == c_in and idx.shape == (c_out, g)
+    t = 1 << tau
+    vec = np.array([[1 if (int(codebook[k]) >> (7 - e)) & 1 else -1 for e in range(8)] for k in range(t)], dtype=np.int64)
+    p = np.einsum("nhwge,ke->nhwgk", a.reshape(n, ho, wo, g, 8), vec)     # step 1
+    s = np.zeros((n, ho, wo, c_out), dtype=np.int64)
+    for co in range(c_out):                                              # step 2: lookup + addition over groups
+        for gi in range(g):
+            s[..., co] += p[..., gi, idx[co, gi]]
     return s

@@ -206,3 +206,106 @@ int snn_oracle_conv_f16(const uint16_t* codebook, int tau, const uint8_t* idx_pa
   free(w);
   return ORACLE_OK;
 }
+
+/*
+ * ---------------------------------------------------------------------------
+ * 1x1 extension (appendix "Extending to Bottleneck with 1x1 Kernels" and its
+ * comparison table): the weights of a 1x1 layer are cut into c_out * c_in / 8
+ * vectors of 8 consecutive input channels; every vector is a tau'-bit index
+ * (1 <= tau' <= 8; tau' = 8 is the full set, i.e. a plain 1-bit layer) into a
+ * layer-specific set of 2^tau' vectors from {-1,+1}^8 (256 in all).
+ *
+ *   S[n,co,y,x] = sum_{ci} w(co,ci) * a(n, y*s, x*s, ci)        (no padding)
+ *   w(co, 8g + j) = +1 if bit (7 - j) of codebook[idx[co][g]] is set, else -1
+ *   Y = (float)S * alpha[co]
+ *
+ * The numbering follows the 3x3 kernels' (Sec. 4.1): the flattened vector read
+ * as a binary sequence, first element most significant, all -1 first (code 0)
+ * and all +1 last (code 255).  The index stream is the same LSB-first tau'-bit
+ * stream, element e = co * (c_in/8) + g.  Bit order and packing are conventions
+ * of this repository (parity unpinned by the paper for those two).
+ * ---------------------------------------------------------------------------
+ */
+static int8_t* decode_weights1x1(const uint16_t* codebook, int tau, const uint8_t* idx_packed, int C, int K) {
+  int8_t* w = (int8_t*)malloc((size_t)K * C);
+  if (!w) return NULL;
+  const int G = C / 8;
+  for (int co = 0; co < K; ++co)
+    for (int g = 0; g < G; ++g) {
+      uint32_t j = stream_get(idx_packed, tau, (size_t)co * G + g);
+      uint32_t code = codebook[j];
+      for (int e = 0; e < 8; ++e) w[(size_t)co * C + 8 * g + e] = ((code >> (7 - e)) & 1) ? 1 : -1;
+    }
+  return w;
+}
+
+static int check_1x1(const uint16_t* codebook, int tau, const uint8_t* idx_packed, int C, int K) {
+  if (!codebook || !idx_packed || tau < 1 || tau > 8 || C < 8 || (C % 8) || K < 1) return ORACLE_BAD_ARG;
+  for (int j = 0; j < (1 << tau); ++j)
+    if (codebook[j] >= 256) return ORACLE_BAD_ARG;
+  return ORACLE_OK;
+}
+
+int snn_oracle_decode1x1(const uint16_t* codebook, int tau, const uint8_t* idx_packed, int C, int K, int8_t* w_out) {
+  int rc = check_1x1(codebook, tau, idx_packed, C, K);
+  if (rc || !w_out) return ORACLE_BAD_ARG;
+  int8_t* w = decode_weights1x1(codebook, tau, idx_packed, C, K);
+  if (!w) return ORACLE_NO_MEM;
+  memcpy(w_out, w, (size_t)K * C);
+  free(w);
+  return ORACLE_OK;
+}
+
+int snn_oracle_conv1x1_bin(const uint16_t* codebook, int tau, const uint8_t* idx_packed, const float* alpha, int C,
+                           int K, int stride, const uint32_t* act, int N, int H, int W, int32_t* S_out,
+                           float* Y_out) {
+  int rc = check_1x1(codebook, tau, idx_packed, C, K);
+  if (rc) return rc;
+  if (!alpha || !act || N < 0 || H < 1 || W < 1 || stride < 1) return ORACLE_BAD_ARG;
+  const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+  const int Cw = (C + 31) / 32;
+  int8_t* w = decode_weights1x1(codebook, tau, idx_packed, C, K);
+  if (!w) return ORACLE_NO_MEM;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int co = 0; co < K; ++co)
+      for (int y = 0; y < Ho; ++y)
+        for (int x = 0; x < Wo; ++x) {
+          const size_t px = ((size_t)n * H + (size_t)y * stride) * W + (size_t)x * stride;
+          int32_t s = 0;
+          for (int ci = 0; ci < C; ++ci) {
+            uint32_t word = act[px * Cw + (ci >> 5)];
+            int av = ((word >> (ci & 31)) & 1u) ? 1 : -1;
+            s += (int)w[(size_t)co * C + ci] * av;
+          }
+          size_t o = (((size_t)n * Ho + y) * Wo + x) * K + co;
+          if (S_out) S_out[o] = s;
+          if (Y_out) Y_out[o] = (float)s * alpha[co];
+        }
+  free(w);
+  return ORACLE_OK;
+}
+
+int snn_oracle_conv1x1_f16(const uint16_t* codebook, int tau, const uint8_t* idx_packed, const float* alpha, int C,
+                           int K, int stride, const uint16_t* act_half_bits, int N, int H, int W, float* Y_out) {
+  int rc = check_1x1(codebook, tau, idx_packed, C, K);
+  if (rc) return rc;
+  if (!alpha || !act_half_bits || !Y_out || N < 0 || H < 1 || W < 1 || stride < 1) return ORACLE_BAD_ARG;
+  const int Ho = (H - 1) / stride + 1, Wo = (W - 1) / stride + 1;
+  int8_t* w = decode_weights1x1(codebook, tau, idx_packed, C, K);
+  if (!w) return ORACLE_NO_MEM;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < N; ++n)
+    for (int co = 0; co < K; ++co)
+      for (int y = 0; y < Ho; ++y)
+        for (int x = 0; x < Wo; ++x) {
+          const size_t px = ((size_t)n * H + (size_t)y * stride) * W + (size_t)x * stride;
+          double s = 0.0;
+          for (int ci = 0; ci < C; ++ci)
+            s += (double)w[(size_t)co * C + ci] * half_bits_to_double(act_half_bits[px * C + ci]);
+          size_t o = (((size_t)n * Ho + y) * Wo + x) * K + co;
+          Y_out[o] = (float)((double)alpha[co] * s);
+        }
+  free(w);
+  return ORACLE_OK;
+}

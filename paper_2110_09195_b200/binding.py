@@ -27,6 +27,7 @@ EXPORTED_SYMBOLS = (
     "snn_conv_path_supported", "snn_conv_destroy", "snn_last_error", "snn_version", "snn_kernel_launches",
     "snn_microbench", "snn_conv_forward_static",
     "snn_conv_group_create", "snn_conv_group_forward", "snn_conv_group_destroy",
+    "snn_conv_stack_create", "snn_conv_stack_forward", "snn_conv_stack_destroy",
 )
 
 
@@ -91,6 +92,12 @@ def load_library():
     lib.snn_conv_group_forward.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), i32, vp]
     lib.snn_conv_group_destroy.restype = i32
     lib.snn_conv_group_destroy.argtypes = [vp]
+    lib.snn_conv_stack_create.restype = i32
+    lib.snn_conv_stack_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, i32, ctypes.POINTER(vp)]
+    lib.snn_conv_stack_forward.restype = i32
+    lib.snn_conv_stack_forward.argtypes = [vp, vp, vp, i32, vp]
+    lib.snn_conv_stack_destroy.restype = i32
+    lib.snn_conv_stack_destroy.argtypes = [vp]
     lib.snn_microbench.restype = i32
     lib.snn_microbench.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double)]
     _lib = lib
@@ -347,6 +354,71 @@ class SnnConvGroup:
         if getattr(self, "_g", None) is not None:
             load_library().snn_conv_group_destroy(self._g)
             self._g = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+class SnnConvStack:
+    """Layers that feed one another through their packed thresholded signs, run as one persistent
+    launch (wraps snn_conv_stack_t).  `layers` are SnnConv objects with binary activations whose
+    shapes chain; (n, h, w) is the input shape of the first.  The SnnConv objects must outlive the stack."""
+
+    def __init__(self, layers, n, h, w):
+        lib = load_library()
+        cnt = len(layers)
+        if cnt < 1:
+            raise SnnError(1, "a stack needs at least one layer")
+        self.layers = list(layers)
+        self.n, self.h, self.w = int(n), int(h), int(w)
+        hs = (ctypes.c_void_p * cnt)(*[l._h for l in self.layers])
+        st = ctypes.c_void_p()
+        self._s = None
+        _check(lib.snn_conv_stack_create(hs, cnt, self.n, self.h, self.w, ctypes.byref(st)))
+        self._s = st
+        self.device = self.layers[0].device
+        ho, wo = self.h, self.w
+        for l in self.layers:
+            ho, wo = l.out_hw(ho, wo)
+        self.out_hw = (ho, wo)
+
+    def alloc_out(self, out_type=OUT_F32):
+        import torch
+        last = self.layers[-1]
+        k = (last.c_out + 31) // 32 if out_type == OUT_BITS else last.c_out
+        dt = torch.float32 if out_type == OUT_F32 else torch.int32
+        return torch.empty((self.n, *self.out_hw, k), dtype=dt, device=f"cuda:{self.device}")
+
+    def forward(self, act, out=None, out_type=OUT_F32, stream=None):
+        """snn_conv_stack_forward: act is the first layer's input, out the last layer's output."""
+        import torch
+        first = self.layers[0]
+        if not act.is_cuda or act.device.index != self.device:
+            raise SnnError(1, f"activations must live on cuda:{self.device}")
+        first._check_act(act)
+        if tuple(act.shape[:3]) != (self.n, self.h, self.w):
+            raise SnnError(1, "activation tensor does not have the shape the stack was created for")
+        if out is None:
+            out = self.alloc_out(out_type)
+        last = self.layers[-1]
+        k = (last.c_out + 31) // 32 if out_type == OUT_BITS else last.c_out
+        dt = torch.float32 if out_type == OUT_F32 else torch.int32
+        if (not out.is_cuda or out.device.index != self.device or out.dtype != dt or not out.is_contiguous()
+                or tuple(out.shape) != (self.n, *self.out_hw, k)):
+            raise SnnError(1, "output tensor has the wrong device, dtype, shape or layout")
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        _check(load_library().snn_conv_stack_forward(self._s, act.data_ptr(), out.data_ptr(), int(out_type),
+                                                     ctypes.c_void_p(stream.cuda_stream)))
+        return out
+
+    def destroy(self):
+        if getattr(self, "_s", None) is not None:
+            load_library().snn_conv_stack_destroy(self._s)
+            self._s = None
 
     def __del__(self):
         try:

@@ -127,7 +127,7 @@ cudaError_t solo_group(snn_conv* h, const Geom& g, GroupDev** out, int* launched
   if (it != h->solo.end()) { *out = it->second; return cudaSuccess; }
   const LayerDev* Lp = &h->L;
   GroupDev* G = nullptr;
-  cudaError_t e = tcg_create(&Lp, &g, 1, h->act_type, h->host_stream, &G, launched);
+  cudaError_t e = tcg_create(&Lp, &g, 1, h->act_type, 0, h->host_stream, &G, launched);
   if (e != cudaSuccess) return e;
   h->solo[key] = G;
   *out = G;
@@ -493,7 +493,7 @@ snn_status_t snn_conv_group_create(snn_conv_t* const* layers, int32_t count, con
     e = cudaHostGetDevicePointer((void**)&g->status_dev, g->status_host, 0);
   }
   int launched = 0;
-  if (e == cudaSuccess) e = tcg_create(Ls, gs, count, g->act_type, layers[0]->host_stream, &g->G, &launched);
+  if (e == cudaSuccess) e = tcg_create(Ls, gs, count, g->act_type, 0, layers[0]->host_stream, &g->G, &launched);
   g_launches += launched;
   if (e != cudaSuccess) {
     if (g->status_host) cudaFreeHost(g->status_host);
@@ -542,6 +542,96 @@ snn_status_t snn_conv_group_destroy(snn_conv_group_t* g) {
   tcg_destroy(g->G);
   if (g->status_host) cudaFreeHost(g->status_host);
   delete g;
+  return SNN_OK;
+}
+
+struct snn_conv_stack {
+  int device = 0, count = 0;
+  GroupDev* G = nullptr;
+  int* status_host = nullptr;  // pinned, written by the kernel on a bounded-wait timeout
+  int* status_dev = nullptr;
+};
+
+snn_status_t snn_conv_stack_create(snn_conv_t* const* layers, int32_t count, int32_t N, int32_t H, int32_t W,
+                                   snn_conv_stack_t** out) {
+  if (!out) return fail(SNN_ERR_INVALID_ARG, "null output pointer");
+  *out = nullptr;
+  if (!layers) return fail(SNN_ERR_INVALID_ARG, "null argument");
+  if (count < 1 || count > SNN_GROUP_MAX)
+    return fail(SNN_ERR_INVALID_ARG, "a stack has 1..%d members, not %d", SNN_GROUP_MAX, count);
+  const LayerDev* Ls[SNN_GROUP_MAX];
+  Geom gs[SNN_GROUP_MAX];
+  int h_in = H, w_in = W;
+  for (int i = 0; i < count; ++i) {
+    if (!layers[i]) return fail(SNN_ERR_INVALID_ARG, "member %d is a null handle", i);
+    if (layers[i]->act_type != SNN_ACT_BIN)
+      return fail(SNN_ERR_INVALID_ARG, "member %d: a stack chains binary activations", i);
+    if (layers[i]->device != layers[0]->device) return fail(SNN_ERR_INVALID_ARG, "member %d is on another device", i);
+    if (i > 0 && layers[i]->C != layers[i - 1]->K)
+      return fail(SNN_ERR_INVALID_ARG, "member %d takes %d channels, member %d gives %d", i, layers[i]->C, i - 1,
+                  layers[i - 1]->K);
+    if (N < 1 || !make_geom(layers[i], N, h_in, w_in, &gs[i]))
+      return fail(SNN_ERR_INVALID_ARG, "member %d: shape N=%d H=%d W=%d gives no output", i, N, h_in, w_in);
+    if (!tcg_supported(gs[i], SNN_ACT_BIN))
+      return fail(SNN_ERR_UNSUPPORTED, "member %d: the tensor-core path cannot run this layer at this shape", i);
+    h_in = gs[i].Ho;
+    w_in = gs[i].Wo;
+    Ls[i] = &layers[i]->L;
+  }
+  DeviceGuard guard(layers[0]->device);
+  if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", layers[0]->device);
+  snn_conv_stack* st = new (std::nothrow) snn_conv_stack();
+  if (!st) return fail(SNN_ERR_OOM, "host allocation failed");
+  st->device = layers[0]->device;
+  st->count = count;
+  cudaError_t e = cudaHostAlloc((void**)&st->status_host, sizeof(int), cudaHostAllocMapped);
+  if (e == cudaSuccess) {
+    *st->status_host = 0;
+    e = cudaHostGetDevicePointer((void**)&st->status_dev, st->status_host, 0);
+  }
+  int launched = 0;
+  if (e == cudaSuccess) e = tcg_create(Ls, gs, count, SNN_ACT_BIN, 1, layers[0]->host_stream, &st->G, &launched);
+  g_launches += launched;
+  if (e != cudaSuccess) {
+    if (st->status_host) cudaFreeHost(st->status_host);
+    delete st;
+    if (e == cudaErrorInvalidConfiguration) {
+      cudaGetLastError();
+      return fail(SNN_ERR_UNSUPPORTED, "the tensor-core kernel cannot run these layers as one stack");
+    }
+    return cuda_fail(e, "snn_conv_stack_create");
+  }
+  *out = st;
+  return SNN_OK;
+}
+
+snn_status_t snn_conv_stack_forward(snn_conv_stack_t* st, const void* act_dev, void* out_dev, int32_t out_type,
+                                    void* cuda_stream) {
+  if (!st || !st->G) return fail(SNN_ERR_INVALID_ARG, "null stack");
+  if (!act_dev || !out_dev) return fail(SNN_ERR_INVALID_ARG, "null device pointer");
+  if (out_type != SNN_OUT_F32 && out_type != SNN_OUT_I32 && out_type != SNN_OUT_BITS)
+    return fail(SNN_ERR_INVALID_ARG, "unknown output type %d", out_type);
+  if (((uintptr_t)act_dev & 15) || ((uintptr_t)out_dev & 15)) return fail(SNN_ERR_INVALID_ARG, "misaligned device pointer");
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", st->device);
+  if (*st->status_host) {
+    const int code = *st->status_host;
+    *st->status_host = 0;
+    return fail(SNN_ERR_TIMEOUT, "an earlier launch of the stack gave up a bounded wait (code %d)", code);
+  }
+  int launched = 0;
+  cudaError_t e = tcg_forward(st->G, &act_dev, &out_dev, out_type, (cudaStream_t)cuda_stream, st->status_dev, &launched);
+  g_launches += launched;
+  if (e != cudaSuccess) return cuda_fail(e, "snn_conv_stack_forward");
+  return SNN_OK;
+}
+
+snn_status_t snn_conv_stack_destroy(snn_conv_stack_t* st) {
+  if (!st) return SNN_OK;
+  DeviceGuard guard(st->device);
+  tcg_destroy(st->G);
+  if (st->status_host) cudaFreeHost(st->status_host);
+  delete st;
   return SNN_OK;
 }
 

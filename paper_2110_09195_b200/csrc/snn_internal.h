@@ -51,9 +51,12 @@ cudaError_t reuse_forward(const LayerDev& L, const Geom& g, int act_type, const 
 // layers as ONE persistent launch; a single layer is a group of one.
 // Several independent problems in one persistent tensor-core launch (snn_tcg.cu).
 struct GroupDev;
-cudaError_t tcg_create(const LayerDev* const* layers, const Geom* geoms, int count, int act_type, cudaStream_t s,
-                       GroupDev** out, int* launched);
-cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, int out_i32, cudaStream_t s,
+// chain = 1: member i + 1 reads the packed signs member i writes (binary activations; the members' shapes must
+// follow from one another); tcg_forward then takes the first member's input in act[0] and the last member's
+// output in out[0], and out_type is the last member's.
+cudaError_t tcg_create(const LayerDev* const* layers, const Geom* geoms, int count, int act_type, int chain,
+                       cudaStream_t s, GroupDev** out, int* launched);
+cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, int out_type, cudaStream_t s,
                         int* status_dev, int* launched);
 void tcg_destroy(GroupDev* G);
 int tcg_count(const GroupDev* G);

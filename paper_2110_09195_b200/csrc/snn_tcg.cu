@@ -77,6 +77,12 @@ struct GLayer {
   int n_ntiles, total_tiles;
   const uint16_t* rank;   // [grid] CTA b takes this problem's tiles rank[b], rank[b] + grid, ...
   long long Qtot;
+  // A chain (every member reads the packed signs its predecessor writes, all in one launch): a tile may be
+  // staged once the predecessor's tiles that hold its input pixels are complete, and says so itself when done.
+  const uint2* deps;          // [M groups] first and last M group of the predecessor this M group reads (x > y: none)
+  const uint32_t* prev_done;  // the predecessor's completion counters, and the count that means "complete"
+  uint32_t prev_target;
+  uint32_t* done;             // [M groups] epilogue warps that have finished the group, over all its channel tiles
 };
 
 struct GParams {
@@ -85,7 +91,7 @@ struct GParams {
   const void* act[SNN_GROUP_MAX];
   void* out[SNN_GROUP_MAX];
   int* status;
-  int out_i32;            // 0: fp32 alpha*S, 1: int32 S, 2: packed signs of alpha*S
+  uint8_t out_type[SNN_GROUP_MAX];   // per member: 0 fp32 alpha*S, 1 int32 S, 2 packed signs of alpha*S + shift
   uint32_t acc_cols;      // tensor-memory columns of one accumulator buffer
   int NA, NS;
   uint32_t a_slot_bytes, b_slot_bytes;
@@ -121,6 +127,27 @@ __device__ __forceinline__ int g_position_to_pixel(const GLayer& L, uint32_t q, 
   const int r = L.stride * i + pa - L.pad, c = L.stride * j + pb - L.pad;
   if (r < 0 || r >= L.H || c < 0 || c >= L.W) return -1;
   return ((int)n * L.H + r) * L.W + c;
+}
+
+// Bounded wait until a completion counter another CTA advances has reached `target` (acquire: what that CTA
+// wrote before is visible afterwards).  False when the limit ran out or the CTA is giving up.
+__device__ __forceinline__ bool g_wait_counter(const uint32_t* ctr, uint32_t target, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < (1u << 21); ++it) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+    if (v >= target) return true;
+    if (*abort_flag) return false;
+    __nanosleep(100);
+  }
+  return false;
+}
+// Activation words: through the read-only path, or - when another CTA of this launch wrote them - from L2.
+__device__ __forceinline__ uint32_t g_ld1(const uint32_t* p, bool fresh) { return fresh ? __ldcg(p) : __ldg(p); }
+__device__ __forceinline__ uint2 g_ld2(const uint32_t* p, bool fresh) {
+  return fresh ? __ldcg(reinterpret_cast<const uint2*>(p)) : __ldg(reinterpret_cast<const uint2*>(p));
+}
+__device__ __forceinline__ uint4 g_ld4(const uint32_t* p, bool fresh) {
+  return fresh ? __ldcg(reinterpret_cast<const uint4*>(p)) : __ldg(reinterpret_cast<const uint4*>(p));
 }
 
 // first tile of problem L for this CTA (tiles then follow at a stride of the grid)
@@ -388,6 +415,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       const int Nt = L.Nt, MT = L.MT, K = L.K;
       const float* alpha = L.alpha;
       const float* shift = L.shift;
+      const int out_i32 = p.out_type[l];
       uint32_t* out32 = reinterpret_cast<uint32_t*>(p.out[l]);  // int32 and fp32 outputs share the layout
       const bool fast = ((K & 3) == 0) && ((Nt & 31) == 0);
       for (int tile = g_first_tile(L); tile < L.total_tiles; tile += G) {
@@ -417,7 +445,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           const bool valid = ((long long)q < L.Qtot) && ((int)n < L.N) && (y < L.Ho) && (x < L.Wo);
           return valid ? ((int)n * L.Ho + y) * L.Wo + x : -1;
         };
-        if (p.out_i32 == 2) {
+        if (out_i32 == 2) {
           // Packed signs of the scaled output (Algorithm 1: the next layer consumes sign(a)): a thread
           // owns one position and the 32 (or 16) consecutive channels of a slice, i.e. one word (or
           // half-word) of the next layer's binary input.  No transposition, one small store per slice.
@@ -495,7 +523,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
             }
             const int co = n0 + c0 + scol * 4;
             float4 al = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (!p.out_i32 && co < K) al = __ldg(reinterpret_cast<const float4*>(alpha + co));
+            if (!out_i32 && co < K) al = __ldg(reinterpret_cast<const float4*>(alpha + co));
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 8; ++e)
@@ -512,7 +540,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
                 const int row = srow + 4 * i;
                 u[i] = *reinterpret_cast<const uint4*>(stage + row * G_EPI_PITCH + ((scol ^ (row & 7)) << 4));
               }
-              if (!p.out_i32) {
+              if (!out_i32) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                   scale_pair(u[i].x, u[i].y, al.x, al.y);
@@ -552,7 +580,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 #pragma unroll
               for (int e = 0; e < 16; ++e) {
                 if (co0 + e < K) {
-                  if (p.out_i32) o[e] = (uint32_t)__float2int_rn(__uint_as_float(v[e]));
+                  if (out_i32) o[e] = (uint32_t)__float2int_rn(__uint_as_float(v[e]));
                   else o[e] = __float_as_uint(__fmul_rn(__uint_as_float(v[e]), __ldg(alpha + co0 + e)));
                 }
               }
@@ -563,6 +591,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_accempty + 8 * acc_slot);
+        if (L.done) {
+          // chain: this warp's part of the tile is written; the successor may read it
+          __threadfence();
+          __syncwarp();
+          if (lane == 0) atomicAdd(L.done + mg, 1u);
+        }
         if (++acc_slot == 2) { acc_slot = 0; acc_phase ^= 1u; }
       }
     }
@@ -577,6 +611,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     long long a_done = 0;
     uint32_t a_phase = 1;  // parity of the previous use of a slot (valid from the second lap)
     volatile int* exp_flag = abort_flag + 1;
+    volatile int* dep_flag = abort_flag + 2;
     bool stop = false;
     long long tr_w0 = 0, tr_t0 = clock64();
     (void)tr_w0; (void)tr_t0;
@@ -586,6 +621,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       const int C = L.C, Cw = L.Cw, total = L.total_tiles;
       const FastDiv dNt = L.dNt;
       const void* act = p.act[l];
+      const bool fresh = L.deps != nullptr;   // written by other CTAs of this launch: read from L2
       // vector loads of a row's words need the base pointer and the row pitch aligned to the load
       bool vec;
       {
@@ -598,8 +634,28 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       for (int tile = g_first_tile(L); tile < total && !stop; tile += G) {
         const int mg = (int)fdiv((uint32_t)tile, dNt);
         const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
+        if (L.deps) {
+          // chain: wait until the predecessor has written every input pixel of this tile (one thread polls)
+          if (et == 0) {
+            const uint2 d = __ldg(L.deps + mg);
+            int okd = 1;
+            for (uint32_t m = d.x; m <= d.y && okd; ++m) okd = g_wait_counter(L.prev_done + m, L.prev_target, abort_flag) ? 1 : 0;
+            *dep_flag = okd;
+          }
+          asm volatile("bar.sync 3, %0;" ::"n"(G_EXP_THREADS) : "memory");
+          const int okd = *dep_flag;
+          if (!okd) {
+            if (et == 0 && !*abort_flag) {
+              *abort_flag = 1;
+              raise_status(p.status, 5);
+            }
+            stop = true;
+            break;
+          }
+        }
         // Input pixel of every staged row, once per tile.  The table is private to the expanders:
-        // the barrier keeps a fast thread from overwriting entries another still reads.
+        // the barrier keeps a fast thread from overwriting entries another still reads (and, in a chain,
+        // the polling thread from setting the next tile's flag before everyone has read this one).
         asm volatile("bar.sync 3, %0;" ::"n"(G_EXP_THREADS) : "memory");
         // (plane, row) pairs form one index space f = plane*Rr + row, dealt to the threads at a stride of
         // the expander count, here and below: a thread reads back only entries it wrote itself
@@ -682,19 +738,19 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
                     if (pix[j] >= 0 && w0 < Cw) {
                       const uint32_t* src = (const uint32_t*)act + wide_mul((uint32_t)pix[j], (uint32_t)Cw) + w0;
                       if (vec4) {
-                        const uint4 t = __ldg(reinterpret_cast<const uint4*>(src));
+                        const uint4 t = g_ld4(src, fresh);
                         bits[j][0] = t.x; bits[j][1] = t.y; bits[j][2] = t.z; bits[j][3] = t.w;
                       } else if (vec) {
-                        const uint2 t = __ldg(reinterpret_cast<const uint2*>(src));
+                        const uint2 t = g_ld2(src, fresh);
                         bits[j][0] = t.x; bits[j][1] = t.y;
                         if (nw == 4) {
-                          const uint2 t2 = __ldg(reinterpret_cast<const uint2*>(src + 2));
+                          const uint2 t2 = g_ld2(src + 2, fresh);
                           bits[j][2] = t2.x; bits[j][3] = t2.y;
                         }
                       } else {
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                          if (k < nw && w0 + k < Cw) bits[j][k] = __ldg(src + k);
+                          if (k < nw && w0 + k < Cw) bits[j][k] = g_ld1(src + k, fresh);
                       }
                     }
                   }
@@ -733,6 +789,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 // ------------------------------------------------------------------ host side
 struct GroupDev {
   int count = 0, act_type = 0, mode = M_FP4;
+  int chain = 0;                  // 1: member i + 1 reads the packed signs member i writes (one launch, dependency counters)
+  uint8_t* chain_buf = nullptr;   // the packed signs between the members, one buffer per boundary
+  size_t chain_off[SNN_GROUP_MAX] = {};
+  uint32_t* done = nullptr;       // completion counters of all members' M groups
+  size_t done_words = 0;
+  uint2* deps = nullptr;
   GLayer* layers_dev = nullptr;   // [count]
   uint8_t* weights = nullptr;     // the group's own weight operands, one after the other
   uint16_t* ranks = nullptr;      // [count][grid] tile assignment, see tcg_create
@@ -859,10 +921,26 @@ bool g_plan_layer(const Geom& g, int mode, GLayer* L, int* n_chunks_out, int* Kp
 
 }  // namespace
 
-cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int act_type, cudaStream_t s,
+namespace {
+// host copy of the kernel's position -> input pixel map
+int h_position_to_pixel(const GLayer& L, long long q, int pa, int pb) {
+  if (q >= L.Qtot) return -1;
+  const long long rg = q / L.Wq;
+  const int j = (int)(q - rg * L.Wq);
+  const long long n = rg / L.Hq;
+  const int i = (int)(rg - n * L.Hq);
+  if (n >= L.N) return -1;
+  const int r = L.stride * i + pa - L.pad, c = L.stride * j + pb - L.pad;
+  if (r < 0 || r >= L.H || c < 0 || c >= L.W) return -1;
+  return (int)((n * L.H + r) * L.W + c);
+}
+}  // namespace
+
+cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int act_type, int chain, cudaStream_t s,
                        GroupDev** out, int* launched) {
   *out = nullptr;
   if (count < 1 || count > SNN_GROUP_MAX) return cudaErrorInvalidConfiguration;
+  if (chain && act_type != SNN_ACT_BIN) return cudaErrorInvalidConfiguration;
   const int mode = g_mode_for(act_type);
   GLayer host[SNN_GROUP_MAX];
   int n_chunks[SNN_GROUP_MAX], Kpad[SNN_GROUP_MAX];
@@ -892,7 +970,55 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   if (na < 2 || ns < 3) return cudaErrorInvalidConfiguration;
   if (ns > G_NS_MAX) ns = G_NS_MAX;
   const int sms = sm_count();
-  const int grid = tiles < sms ? (int)tiles : sms;
+  int grid = tiles < sms ? (int)tiles : sms;
+  // A chain's CTAs wait for one another, so all of them must be resident together (a cooperative launch
+  // checks that); members with fewer tiles than CTAs simply leave some CTAs without work in that member.
+  std::vector<uint2> deps;
+  std::vector<size_t> deps_off(count, 0), done_off(count, 0);
+  size_t done_words = 0, chain_bytes = 0;
+  size_t chain_off[SNN_GROUP_MAX] = {};
+  if (chain) {
+    for (int i = 0; i < count; ++i) {
+      if (i > 0 && (gs[i].C != gs[i - 1].K || gs[i].H != gs[i - 1].Ho || gs[i].W != gs[i - 1].Wo || gs[i].N != gs[0].N))
+        return cudaErrorInvalidConfiguration;
+      const int mgroups = host[i].total_tiles / host[i].n_ntiles;
+      done_off[i] = done_words;
+      done_words += (size_t)mgroups;
+      if (i + 1 < count) {
+        chain_off[i] = chain_bytes;
+        chain_bytes += (((size_t)gs[i].N * gs[i].Ho * gs[i].Wo * ((gs[i].K + 31) / 32) * 4) + 255) & ~(size_t)255;
+      }
+      if (i == 0) continue;
+      // which M groups of the predecessor hold the input pixels of each of this member's M groups
+      const GLayer& L = host[i];
+      const GLayer& P = host[i - 1];
+      deps_off[i] = deps.size();
+      for (int mg = 0; mg < mgroups; ++mg) {
+        const long long Q0 = (long long)mg * 128 * L.MT;
+        long long lo = -1, hi = -1;
+        for (int pl = 0; pl < L.n_planes; ++pl)
+          for (int r = 0; r < L.Rr; ++r) {
+            const int px = h_position_to_pixel(L, Q0 + r, pl >> 1, pl & 1);
+            if (px < 0) continue;
+            if (lo < 0 || px < lo) lo = px;
+            if (px > hi) hi = px;
+          }
+        uint2 d = make_uint2(1u, 0u);
+        if (lo >= 0) {
+          // output pixel of the predecessor -> its position -> its M group
+          auto group_of = [&](long long px) {
+            const long long n = px / ((long long)P.Ho * P.Wo);
+            const long long rem = px - n * (long long)P.Ho * P.Wo;
+            const long long y = rem / P.Wo, x = rem - y * P.Wo;
+            const long long q = (n * P.Hq + y) * P.Wq + x;
+            return (uint32_t)(q / (128 * P.MT));
+          };
+          d = make_uint2(group_of(lo), group_of(hi));
+        }
+        deps.push_back(d);
+      }
+    }
+  }
   // Which CTAs take a problem's odd tiles.  Every CTA gets floor(tiles / grid) tiles of a problem
   // and the first (tiles % grid) CTAs in the problem's rank order get one more; the rank order is
   // by the time the CTAs have been given so far, least first, so that the CTAs end close
@@ -922,7 +1048,17 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   G->act_type = act_type;
   G->mode = mode;
   G->grid = grid;
+  G->chain = chain;
   cudaError_t e = cudaMalloc(&G->weights, w_total);
+  if (chain) {
+    G->done_words = done_words;
+    for (int i = 0; i < count; ++i) G->chain_off[i] = chain_off[i];
+    if (e == cudaSuccess) e = cudaMalloc(&G->done, done_words * sizeof(uint32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&G->chain_buf, chain_bytes ? chain_bytes : 256);
+    if (e == cudaSuccess) e = cudaMalloc(&G->deps, (deps.size() ? deps.size() : 1) * sizeof(uint2));
+    if (e == cudaSuccess && !deps.empty())
+      e = cudaMemcpyAsync(G->deps, deps.data(), deps.size() * sizeof(uint2), cudaMemcpyHostToDevice, s);
+  }
   if (e == cudaSuccess) e = cudaMalloc(&G->layers_dev, sizeof(GLayer) * count);
   if (e == cudaSuccess) e = cudaMalloc(&G->ranks, ranks.size() * sizeof(uint16_t));
   if (e == cudaSuccess)
@@ -932,6 +1068,15 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
     host[i].wt = G->weights + w_off[i];
     host[i].alpha = Ls[i]->alpha;
     host[i].shift = Ls[i]->shift;
+    host[i].deps = nullptr; host[i].prev_done = nullptr; host[i].prev_target = 0; host[i].done = nullptr;
+    if (chain) {
+      host[i].done = G->done + done_off[i];
+      if (i > 0) {
+        host[i].deps = G->deps + deps_off[i];
+        host[i].prev_done = G->done + done_off[i - 1];
+        host[i].prev_target = (uint32_t)(G_EW * host[i - 1].n_ntiles);
+      }
+    }
     e = g_expand_weights(mode, Ls[i]->wplanes, G->weights + w_off[i], gs[i].C, gs[i].K, gs[i].Cw, Kpad[i],
                          n_chunks[i], host[i].cb_chunks, host[i].NtL, s);
     if (e == cudaSuccess) *launched += 1;
@@ -969,6 +1114,9 @@ void tcg_destroy(GroupDev* G) {
   cudaFree(G->weights);
   cudaFree(G->layers_dev);
   cudaFree(G->ranks);
+  cudaFree(G->done);
+  cudaFree(G->chain_buf);
+  cudaFree(G->deps);
   delete G;
 }
 
@@ -985,20 +1133,34 @@ bool tcg_supported(const Geom& g, int act_type) {
   return 2 * unit + fixed + 3 * (size_t)kGBSlot <= kGSmemBudget;
 }
 
-cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, int out_i32, cudaStream_t s,
+cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, int out_type, cudaStream_t s,
                         int* status_dev, int* launched) {
   GParams p = G->p;
-  for (int i = 0; i < G->count; ++i) {
-    p.act[i] = act[i];
-    p.out[i] = out[i];
-  }
-  p.out_i32 = out_i32;
-  p.status = status_dev;
-  // Launched as a programmatic dependent of its predecessor in the stream: set-up overlaps that
-  // kernel's tail; the warps that read activations or write outputs wait on the device for it.
   cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  if (G->chain) {
+    // act[0] is the first member's input and out[0] the last member's output; the packed signs in between
+    // stay in the group's own buffers
+    for (int i = 0; i < G->count; ++i) {
+      p.act[i] = i == 0 ? act[0] : (const void*)(G->chain_buf + G->chain_off[i - 1]);
+      p.out[i] = i + 1 == G->count ? out[0] : (void*)(G->chain_buf + G->chain_off[i]);
+      p.out_type[i] = (uint8_t)(i + 1 == G->count ? out_type : 2);
+    }
+    cudaError_t e0 = cudaMemsetAsync(G->done, 0, G->done_words * sizeof(uint32_t), s);
+    if (e0 != cudaSuccess) return e0;
+    attr[0].id = cudaLaunchAttributeCooperative;   // the CTAs wait for one another: all must be resident
+    attr[0].val.cooperative = 1;
+  } else {
+    for (int i = 0; i < G->count; ++i) {
+      p.act[i] = act[i];
+      p.out[i] = out[i];
+      p.out_type[i] = (uint8_t)out_type;
+    }
+    // Launched as a programmatic dependent of its predecessor in the stream: set-up overlaps that
+    // kernel's tail; the warps that read activations or write outputs wait on the device for it.
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+  }
+  p.status = status_dev;
   cudaLaunchConfig_t cfg{};
   cfg.stream = s;
   cfg.attrs = attr;

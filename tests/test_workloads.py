@@ -115,3 +115,46 @@ def test_shard_batch_covers_everything():
                 assert 0 <= a <= b <= n
                 got += list(range(a, b))
             assert got == list(range(n))
+
+
+# ------------------------------------------------------- clustered (skewed) indices, Sec. 4.2
+def test_skewed_probabilities_follow_the_stated_shares():
+    """Sec. 4.2 observation: the 64 most frequent kernels hold more than 70 % of a layer's kernels, and in deep
+    layers 8 kernels hold about 60 %.  The generator's probabilities carry exactly these shares."""
+    p = wl.skewed_probabilities(512, wl.SKEW_TOP64)
+    assert abs(p.sum() - 1) < 1e-12 and abs(np.sort(p)[::-1][:64].sum() - 0.70) < 1e-12
+    p = wl.skewed_probabilities(32, wl.SKEW_DEEP)
+    assert abs(p.sum() - 1) < 1e-12 and abs(np.sort(p)[::-1][:8].sum() - 0.60) < 1e-12
+    assert (np.diff(p[:8]) < 0).all()                        # falling within the frequent entries
+    assert np.allclose(p[8:], 0.40 / 24)                     # the rest share the remainder evenly
+    q = wl.skewed_probabilities(4, wl.SKEW_DEEP)             # codebook smaller than the frequent set
+    assert abs(q.sum() - 1) < 1e-12 and (np.diff(q) < 0).all()
+
+
+def test_skewed_indices_empirical_frequencies():
+    shape = wl.LayerShape(512, 512, 7, 7)
+    p = wl.draw_layer_params(shape, 5, 42, index_skew=wl.SKEW_DEEP)
+    counts = np.sort(np.bincount(p.idx.reshape(-1), minlength=32))[::-1]
+    share = counts[:8].sum() / counts.sum()
+    assert abs(share - 0.60) < 0.01
+    assert p.idx.min() >= 0 and p.idx.max() < 32
+    again = wl.draw_layer_params(shape, 5, 42, index_skew=wl.SKEW_DEEP)
+    assert (again.idx == p.idx).all() and (again.codebook == p.codebook).all()      # seeded
+    uniform = wl.draw_layer_params(shape, 5, 42)
+    assert (uniform.codebook == p.codebook).all()            # same codebook draw, only the indices differ
+    # full kernel space (tau = 9): top-64 share
+    q = wl.draw_layer_params(wl.LayerShape(256, 256, 14, 14), 9, 43, index_skew=wl.SKEW_TOP64)
+    c = np.sort(np.bincount(q.idx.reshape(-1), minlength=512))[::-1]
+    assert abs(c[:64].sum() / c.sum() - 0.70) < 0.01
+
+
+def test_resnet50_1x1_layer_list():
+    """32 bottleneck 1x1 layers (3/4/6/3 blocks, two per block), channel counts chaining through the blocks'
+    3x3 layers: narrow to the block's width, widen four-fold."""
+    ls = wl.resnet50_1x1_layers()
+    assert len(ls) == 32 and all(l.ksize == 1 and l.pad == 0 and l.c_in % 8 == 0 for l in ls)
+    assert (ls[0].c_in, ls[0].c_out, ls[1].c_in, ls[1].c_out) == (64, 64, 64, 256)
+    assert (ls[-2].c_in, ls[-2].c_out, ls[-1].c_in, ls[-1].c_out) == (2048, 512, 512, 2048)
+    assert ls[-1].h == 7 and ls[0].h == 56
+    p = wl.draw_layer_params(ls[2], 5, 1)
+    assert p.idx.shape == (64, 256 // 8) and p.codebook.max() < 256 and len(set(p.codebook.tolist())) == 32

@@ -37,17 +37,18 @@ class LayerShape:
     w: int
     stride: int = 1
     pad: int = 1
+    ksize: int = 3       # 3: the 3x3 layers of the main text; 1: the 1x1 extension of the appendix (pad 0)
 
     @property
     def h_out(self) -> int:
-        return (self.h + 2 * self.pad - 3) // self.stride + 1
+        return (self.h + 2 * self.pad - self.ksize) // self.stride + 1
 
     @property
     def w_out(self) -> int:
-        return (self.w + 2 * self.pad - 3) // self.stride + 1
+        return (self.w + 2 * self.pad - self.ksize) // self.stride + 1
 
     def dense_macs(self, n: int) -> int:
-        return n * self.h_out * self.w_out * self.c_out * self.c_in * 9
+        return n * self.h_out * self.w_out * self.c_out * self.c_in * self.ksize * self.ksize
 
     def in_bytes_bin(self, n: int) -> int:
         return n * self.h * self.w * ((self.c_in + 31) // 32) * 4
@@ -84,6 +85,24 @@ def _imagenet_resnet(blocks) -> List[LayerShape]:
     ls += _stage(64, 128, 56, 2 * blocks[1], False)
     ls += _stage(128, 256, 28, 2 * blocks[2], False)
     ls += _stage(256, 512, 14, 2 * blocks[3], False)
+    return ls
+
+
+def resnet50_1x1_layers() -> List[LayerShape]:
+    """The 32 1x1 layers inside the bottleneck blocks of the ImageNet ResNet-50 (3/4/6/3 blocks; the first 1x1 of a
+    block narrows to the block's width, the last widens four-fold; shortcut projections excluded).  The appendix
+    applies the 1x1 extension to this architecture."""
+    ls: List[LayerShape] = []
+    c_prev, hw = 64, 56
+    for stage, (width, blocks) in enumerate(((64, 3), (128, 4), (256, 6), (512, 3))):
+        for b in range(blocks):
+            if stage > 0 and b == 0:
+                ls.append(LayerShape(c_prev, width, hw, hw, 1, 0, 1))   # narrows on the previous stage's map
+                hw //= 2                                                # the block's 3x3 has stride 2
+            else:
+                ls.append(LayerShape(c_prev, width, hw, hw, 1, 0, 1))
+            ls.append(LayerShape(width, 4 * width, hw, hw, 1, 0, 1))
+            c_prev = 4 * width
     return ls
 
 
@@ -134,6 +153,8 @@ def get_workload(name: str, tau: int | None = None, batch: int | None = None) ->
         wl = Workload("resnet34", 3, 64, 5, "bin", tuple(resnet34_layers()))
     elif name == "tausweep":
         wl = Workload("tausweep", 4, 64, 5, "bin", (LayerShape(256, 256, 14, 14, 1),))
+    elif name == "resnet50_1x1":
+        wl = Workload("resnet50_1x1", 5, 64, 5, "bin", tuple(resnet50_1x1_layers()))
     else:
         raise KeyError(name)
     if tau is not None:
@@ -143,7 +164,7 @@ def get_workload(name: str, tau: int | None = None, batch: int | None = None) ->
     return wl
 
 
-WORKLOAD_NAMES = ("single16", "resnet20", "resnet18", "resnet18_f16", "resnet34", "tausweep")
+WORKLOAD_NAMES = ("single16", "resnet20", "resnet18", "resnet18_f16", "resnet34", "tausweep", "resnet50_1x1")
 
 
 def layer_seed(config: int, layer_index: int, tau: int | None = None) -> int:
@@ -191,18 +212,64 @@ class LayerParams:
     alpha: np.ndarray        # (c_out,) float32 in [0.5, 1.5)
 
 
-def draw_layer_params(shape: LayerShape, tau: int, seed: int) -> LayerParams:
-    """Random layer-specific subset of the 512-kernel space (Sec. 4.2 sampling
-    distribution), uniform indices, uniform scales."""
+def draw_layer_params(shape: LayerShape, tau: int, seed: int, index_skew: "IndexSkew | None" = None) -> LayerParams:
+    """Random layer-specific subset of the kernel space (Sec. 4.2 sampling distribution; 512 binary 3x3 kernels,
+    or the 256 8-channel vectors of a 1x1 layer), indices uniform or, with `index_skew`, concentrated on a few
+    codebook entries, and uniform scales."""
     rng = np.random.default_rng(seed)
     t = 1 << tau
-    if tau == 9:
-        codebook = rng.permutation(512).astype(np.uint16)
+    space = 512 if shape.ksize == 3 else 256
+    if t > space:
+        raise ValueError("codebook larger than the kernel space")
+    if t == space:
+        codebook = rng.permutation(space).astype(np.uint16)
     else:
-        codebook = rng.choice(512, size=t, replace=False).astype(np.uint16)
-    idx = rng.integers(0, t, size=(shape.c_out, shape.c_in), dtype=np.int64).astype(np.int32)
+        codebook = rng.choice(space, size=t, replace=False).astype(np.uint16)
+    cols = shape.c_in if shape.ksize == 3 else shape.c_in // 8
+    if shape.ksize == 1 and shape.c_in % 8:
+        raise ValueError("a 1x1 layer needs c_in divisible by 8")
+    if index_skew is None:
+        idx = rng.integers(0, t, size=(shape.c_out, cols), dtype=np.int64).astype(np.int32)
+    else:
+        idx = draw_skewed_indices(rng, t, (shape.c_out, cols), index_skew)
     alpha = rng.uniform(0.5, 1.5, size=shape.c_out).astype(np.float32)
     return LayerParams(tau, codebook, idx, pack_indices(idx, tau), alpha)
+
+
+@dataclass(frozen=True)
+class IndexSkew:
+    """Kernel-frequency profile of a trained layer, as far as Sec. 4.2 states it: the `top` most frequent
+    kernels together hold the share `mass` of a layer's kernels (the 64 most frequent of the 512 hold more than
+    70 %; in deep layers 8 kernels hold about 60 %); the remaining entries share the rest evenly."""
+    top: int
+    mass: float
+
+
+SKEW_TOP64 = IndexSkew(64, 0.70)     # Sec. 4.2: top 64 kernels, > 70 % (meaningful for codebooks larger than 64)
+SKEW_DEEP = IndexSkew(8, 0.60)       # Sec. 4.2: 8 kernels, about 60 %, in deep layers
+
+
+def skewed_probabilities(t: int, skew: IndexSkew) -> np.ndarray:
+    """Probability of each of the t codebook entries: the first min(top, t) entries carry `mass` with weights
+    falling off harmonically (rank r gets 1/(r+1)), the others share 1 - mass evenly.  With top >= t the whole
+    codebook follows the harmonic profile."""
+    top = min(skew.top, t)
+    head = 1.0 / np.arange(1, top + 1, dtype=np.float64)
+    head /= head.sum()
+    if top == t:
+        return head
+    p = np.empty(t, dtype=np.float64)
+    p[:top] = head * skew.mass
+    p[top:] = (1.0 - skew.mass) / (t - top)
+    return p
+
+
+def draw_skewed_indices(rng, t: int, size, skew: IndexSkew) -> np.ndarray:
+    """Indices in [0, t) drawn from skewed_probabilities; the frequent entries sit at a seeded random
+    permutation of the codebook slots (a trained layer's frequent kernels are not sorted either)."""
+    p = skewed_probabilities(t, skew)
+    slots = rng.permutation(t)
+    return slots[rng.choice(t, size=size, p=p)].astype(np.int32)
 
 
 def draw_activation_bits(shape: LayerShape, n: int, seed: int) -> np.ndarray:
