@@ -82,6 +82,13 @@ typedef struct {
   const float* alpha;         /* HOST, c_out finite fp32 scales */
   const float* shift;         /* HOST, c_out finite fp32 thresholds added to Y before its sign is taken
                                  (SNN_OUT_BITS only; fp32 and int32 outputs ignore it), or NULL for none */
+  int32_t ksize;              /* 0 or 3: a 3x3 layer as above.  1: the 1x1 extension (appendix "Extending to
+                                 Bottleneck with 1x1 Kernels"): the weights are c_out * c_in/8 vectors of 8
+                                 consecutive input channels, each a tau-bit index (1 <= tau <= 8) into a set of
+                                 2^tau 8-bit codes (each < 256; bit 7 - j set <=> element j, i.e. channel 8g + j,
+                                 is +1; code 0 all -1, code 255 all +1); index element e = co*(c_in/8) + g;
+                                 c_in divisible by 8, pad 0, Ho = floor((H - 1)/stride) + 1.  Only the
+                                 tensor-core path runs such a layer. */
 } snn_conv_desc_t;
 
 /*

@@ -44,7 +44,7 @@ class _Desc(ctypes.Structure):
         ("stride", ctypes.c_int32), ("pad", ctypes.c_int32), ("act_type", ctypes.c_int32),
         ("device", ctypes.c_int32),
         ("codebook", ctypes.c_void_p), ("idx_packed", ctypes.c_void_p), ("alpha", ctypes.c_void_p),
-        ("shift", ctypes.c_void_p),
+        ("shift", ctypes.c_void_p), ("ksize", ctypes.c_int32),
     ]
 
 
@@ -160,7 +160,7 @@ def forward_static(c_in, c_out, tau, codebook, idx_packed, alpha, act, out, stri
     if out.dtype != want or tuple(out.shape) != (n, ho, wo, int(c_out)):
         raise SnnError(1, f"out must be {want} of shape {(n, ho, wo, int(c_out))}")
     d = _Desc(int(c_in), int(c_out), int(tau), int(stride), int(pad), ACT_BIN, int(device),
-              cb.ctypes.data, ip.ctypes.data, al.ctypes.data, None)
+              cb.ctypes.data, ip.ctypes.data, al.ctypes.data, None, 3)
     if stream is None:
         stream = torch.cuda.current_stream(device)
     _check(load_library().snn_conv_forward_static(ctypes.byref(d), act.data_ptr(), n, h, w, out.data_ptr(),
@@ -172,34 +172,42 @@ class SnnConv:
     """One sub-bit 3x3 layer on one GPU (wraps a snn_conv_t handle)."""
 
     def __init__(self, c_in, c_out, tau, codebook, idx_packed, alpha, stride=1, pad=1, act_type=ACT_BIN, device=0,
-                 shift=None):
+                 shift=None, ksize=3):
         lib = load_library()
+        if int(ksize) not in (1, 3):
+            raise SnnError(1, f"ksize={ksize} is not 1 or 3")
+        one = int(ksize) == 1
+        if one and int(c_in) % 8:
+            raise SnnError(1, "a 1x1 layer needs c_in divisible by 8")
         cb = np.ascontiguousarray(codebook, dtype=np.uint16)
         ip = np.ascontiguousarray(idx_packed, dtype=np.uint8)
         al = np.ascontiguousarray(alpha, dtype=np.float32)
-        if not 1 <= int(tau) <= 9:
-            raise SnnError(1, f"tau={tau} outside 1..9")
+        if not 1 <= int(tau) <= (8 if one else 9):
+            raise SnnError(1, f"tau={tau} outside 1..{8 if one else 9}")
         if cb.size != (1 << int(tau)):
             raise SnnError(1, f"codebook has {cb.size} entries, expected {1 << int(tau)}")
-        if ip.size < (int(c_out) * int(c_in) * int(tau) + 7) // 8:
-            raise SnnError(1, "index stream shorter than c_out*c_in*tau bits")
+        units = int(c_out) * (int(c_in) // 8 if one else int(c_in))
+        if ip.size < (units * int(tau) + 7) // 8:
+            raise SnnError(1, "index stream shorter than one tau-bit index per kernel (or per 8-channel vector)")
         if al.size != int(c_out):
             raise SnnError(1, f"alpha has {al.size} entries, expected {c_out}")
         sh = None if shift is None else np.ascontiguousarray(shift, dtype=np.float32)
         if sh is not None and sh.size != int(c_out):
             raise SnnError(1, f"shift has {sh.size} entries, expected {c_out}")
         d = _Desc(int(c_in), int(c_out), int(tau), int(stride), int(pad), int(act_type), int(device),
-                  cb.ctypes.data, ip.ctypes.data, al.ctypes.data, None if sh is None else sh.ctypes.data)
+                  cb.ctypes.data, ip.ctypes.data, al.ctypes.data, None if sh is None else sh.ctypes.data, int(ksize))
         h = ctypes.c_void_p()
         self._h = None
         _check(lib.snn_conv_create(ctypes.byref(d), ctypes.byref(h)))
         self._h = h
         self.c_in, self.c_out, self.tau = int(c_in), int(c_out), int(tau)
         self.stride, self.pad, self.act_type, self.device = int(stride), int(pad), int(act_type), int(device)
+        self.ksize = int(ksize)
 
     # -- helpers ------------------------------------------------------------
     def out_hw(self, h, w):
-        return (h + 2 * self.pad - 3) // self.stride + 1, (w + 2 * self.pad - 3) // self.stride + 1
+        k = self.ksize
+        return (h + 2 * self.pad - k) // self.stride + 1, (w + 2 * self.pad - k) // self.stride + 1
 
     def _check_act(self, act):
         import torch

@@ -53,6 +53,7 @@ struct DeviceGuard {
 
 struct snn_conv {
   int C, K, tau, stride, pad, act_type, device;
+  int ksize = 3;
   LayerDev L;
   std::mutex mu;
   std::map<std::tuple<int, int, int>, int> tuned;        // (N,H,W) -> path measured fastest by snn_conv_tune
@@ -70,13 +71,14 @@ namespace {
 
 bool make_geom(const snn_conv* h, int N, int H, int W, Geom* g) {
   if (N < 0 || H < 1 || W < 1) return false;
-  if (H + 2 * h->pad < 3 || W + 2 * h->pad < 3) return false;
+  if (H + 2 * h->pad < h->ksize || W + 2 * h->pad < h->ksize) return false;
   g->N = N; g->H = H; g->W = W;
   g->C = h->C; g->K = h->K; g->Cw = (h->C + 31) / 32;
   g->stride = h->stride; g->pad = h->pad;
-  g->Ho = (H + 2 * h->pad - 3) / h->stride + 1;
-  g->Wo = (W + 2 * h->pad - 3) / h->stride + 1;
+  g->Ho = (H + 2 * h->pad - h->ksize) / h->stride + 1;
+  g->Wo = (W + 2 * h->pad - h->ksize) / h->stride + 1;
   g->tau = h->tau; g->T = 1 << h->tau;
+  g->ksize = h->ksize;
   // index arithmetic in the kernels is 32-bit for pixel counts
   long long in_px = (long long)N * H * W, out_px = (long long)N * g->Ho * g->Wo;
   if (in_px >= (1ll << 31) || out_px >= (1ll << 31)) return false;
@@ -85,8 +87,8 @@ bool make_geom(const snn_conv* h, int N, int H, int W, Geom* g) {
 
 bool path_ok(const snn_conv* h, int path, const Geom& g) {
   switch (path) {
-    case SNN_PATH_REUSE: return reuse_supported(g, h->act_type);
-    case SNN_PATH_DECODED: return popc_supported(g, h->act_type);
+    case SNN_PATH_REUSE: return g.ksize == 3 && reuse_supported(g, h->act_type);
+    case SNN_PATH_DECODED: return g.ksize == 3 && popc_supported(g, h->act_type);
     case SNN_PATH_DECODED_TC: return tcg_supported(g, h->act_type);
     default: return false;
   }
@@ -220,14 +222,19 @@ snn_status_t snn_conv_create(const snn_conv_desc_t* d, snn_conv_t** out) {
   if (!d->codebook || !d->idx_packed || !d->alpha) return fail(SNN_ERR_INVALID_ARG, "null codebook / index / alpha");
   if (d->c_in < 1 || d->c_out < 1) return fail(SNN_ERR_INVALID_ARG, "c_in=%d c_out=%d", d->c_in, d->c_out);
   if (d->c_in > (1 << 16) || d->c_out > (1 << 16)) return fail(SNN_ERR_INVALID_ARG, "channel count above 65536");
-  if (d->tau < 1 || d->tau > 9) return fail(SNN_ERR_INVALID_ARG, "tau=%d outside 1..9", d->tau);
+  if (d->ksize != 0 && d->ksize != 1 && d->ksize != 3) return fail(SNN_ERR_INVALID_ARG, "ksize=%d is not 1 or 3", d->ksize);
+  const bool one = d->ksize == 1;
+  if (d->tau < 1 || d->tau > (one ? 8 : 9)) return fail(SNN_ERR_INVALID_ARG, "tau=%d outside 1..%d", d->tau, one ? 8 : 9);
+  if (one && (d->c_in % 8)) return fail(SNN_ERR_INVALID_ARG, "a 1x1 layer needs c_in divisible by 8, not %d", d->c_in);
+  if (one && d->pad != 0) return fail(SNN_ERR_INVALID_ARG, "a 1x1 layer takes no padding");
   if (d->stride < 1 || d->stride > 2) return fail(SNN_ERR_INVALID_ARG, "stride=%d outside {1,2}", d->stride);
   if (d->pad < 0 || d->pad > 1) return fail(SNN_ERR_INVALID_ARG, "pad=%d outside {0,1}", d->pad);
   if (d->act_type != SNN_ACT_BIN && d->act_type != SNN_ACT_F16)
     return fail(SNN_ERR_INVALID_ARG, "act_type=%d", d->act_type);
   const int T = 1 << d->tau;
   for (int j = 0; j < T; ++j)
-    if (d->codebook[j] >= 512) return fail(SNN_ERR_INVALID_ARG, "codebook[%d]=%u is not a 9-bit code", j, d->codebook[j]);
+    if (d->codebook[j] >= (one ? 256 : 512))
+      return fail(SNN_ERR_INVALID_ARG, "codebook[%d]=%u is not a %d-bit code", j, d->codebook[j], one ? 8 : 9);
   for (int k = 0; k < d->c_out; ++k)
     if (!std::isfinite(d->alpha[k])) return fail(SNN_ERR_INVALID_ARG, "alpha[%d] is not finite", k);
   for (int k = 0; d->shift && k < d->c_out; ++k)
@@ -245,9 +252,10 @@ snn_status_t snn_conv_create(const snn_conv_desc_t* d, snn_conv_t** out) {
   if (!h) return fail(SNN_ERR_OOM, "host allocation failed");
   h->C = d->c_in; h->K = d->c_out; h->tau = d->tau; h->stride = d->stride; h->pad = d->pad;
   h->act_type = d->act_type; h->device = d->device;
+  h->ksize = one ? 1 : 3;
   Geom g;
   make_geom(h, 0, 3, 3, &g);
-  const size_t n_elem = (size_t)h->K * h->C;
+  const size_t n_elem = (size_t)h->K * (one ? h->C / 8 : h->C);
   const size_t idx_bytes = (n_elem * h->tau + 7) / 8;
   const int Tp = (T + 15) / 16 * 16;
   uint8_t* d_stream = nullptr;

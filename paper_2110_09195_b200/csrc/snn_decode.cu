@@ -46,6 +46,25 @@ __global__ void decode_planes_kernel(const uint16_t* __restrict__ idx, const uin
   for (int t = 0; t < 9; ++t) wplanes[((size_t)t * Cw + wd) * K + co] = plane[t];
 }
 
+// 1x1 extension (appendix "Extending to Bottleneck with 1x1 Kernels"): an index names an 8-input-channel vector;
+// element j of the vector (channel 8g + j) is bit 7 - j of its 8-bit code.  One plane, [word][co].
+__global__ void decode_planes1x1_kernel(const uint16_t* __restrict__ idx, const uint16_t* __restrict__ codebook,
+                                        uint32_t* __restrict__ wplanes, int C, int K, int Cw) {
+  int co = blockIdx.x * blockDim.x + threadIdx.x;
+  int wd = blockIdx.y;
+  if (co >= K) return;
+  const int G = C / 8;
+  uint32_t plane = 0;
+  for (int g4 = 0; g4 < 4; ++g4) {
+    int g = wd * 4 + g4;
+    if (g >= G) break;
+    uint32_t code = codebook[idx[(size_t)co * G + g]];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) plane |= ((code >> (7 - e)) & 1u) << (8 * g4 + e);
+  }
+  wplanes[(size_t)wd * K + co] = plane;
+}
+
 // Border corrections.  The integer kernels read a zero activation word where a
 // tap falls outside the image, which the +/-1 arithmetic takes for -1; the true
 // contribution of such a tap is 0 (zero padding).  Adding back
@@ -93,10 +112,16 @@ __global__ void match9_kernel(const uint16_t* __restrict__ codebook, uint8_t* __
 cudaError_t decode_layer(const LayerDev& L, const uint8_t* idx_packed_dev, const Geom& g, int act_type,
                          cudaStream_t s, int* launched) {
   (void)act_type;
-  long long n_elem = (long long)g.K * g.C;
+  long long n_elem = (long long)g.K * (g.ksize == 1 ? g.C / 8 : g.C);
   long long n_bytes = (n_elem * g.tau + 7) / 8;
   unpack_idx_kernel<<<(unsigned)((n_elem + 255) / 256), 256, 0, s>>>(idx_packed_dev, L.idx, n_elem, g.tau, n_bytes);
   dim3 grid((g.K + 127) / 128, g.Cw);
+  if (g.ksize == 1) {
+    // only the tensor-core path runs 1x1 layers: no border corrections (no padding), no matching-tap table
+    decode_planes1x1_kernel<<<grid, 128, 0, s>>>(L.idx, L.codebook, L.wplanes, g.C, g.K, g.Cw);
+    *launched += 2;
+    return cudaGetLastError();
+  }
   decode_planes_kernel<<<grid, 128, 0, s>>>(L.idx, L.codebook, L.wplanes, g.C, g.K, g.Cw);
   corr_kernel<<<(g.K + 127) / 128, 128, 0, s>>>(L.wplanes, L.corr, g.C, g.K, g.Cw);
   int Tp = (g.T + 15) / 16 * 16;

@@ -16,6 +16,7 @@ struct Geom {
   int stride, pad;
   int Ho, Wo;         // output map
   int tau, T;         // index width, codebook size 2^tau
+  int ksize;          // 3, or 1 for the 1x1 extension (8-input-channel vectors, pad 0)
 };
 
 // Device-resident layer data derived at create time (Sec. 4.4 storage -> compute form).

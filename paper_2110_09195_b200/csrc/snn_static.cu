@@ -55,6 +55,8 @@ extern "C" SNN_API snn_status_t snn_conv_forward_static(const snn_conv_desc_t* d
   if (!d) return api_fail(SNN_ERR_INVALID_ARG, "null descriptor");
   if (!d->codebook || !d->idx_packed || !d->alpha) return api_fail(SNN_ERR_INVALID_ARG, "null codebook / index / alpha");
   if (d->c_in < 1 || d->c_out < 1) return api_fail(SNN_ERR_INVALID_ARG, "c_in=%d c_out=%d", d->c_in, d->c_out);
+  if (d->ksize != 0 && d->ksize != 3)
+    return api_fail(SNN_ERR_UNSUPPORTED, "the no-allocation entry point runs 3x3 layers only (ksize=%d)", d->ksize);
   if (d->tau < 1 || d->tau > 9) return api_fail(SNN_ERR_INVALID_ARG, "tau=%d outside 1..9", d->tau);
   if (d->stride < 1 || d->stride > 2) return api_fail(SNN_ERR_INVALID_ARG, "stride=%d outside {1,2}", d->stride);
   if (d->pad < 0 || d->pad > 1) return api_fail(SNN_ERR_INVALID_ARG, "pad=%d outside {0,1}", d->pad);

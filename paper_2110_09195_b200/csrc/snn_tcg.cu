@@ -72,7 +72,8 @@ struct GLayer {
   int n_planes, halo, Rr; // 1 or 4 planes; largest tap shift; staged rows per plane = 128*MT + halo
   int MT;                 // M sub-tiles of 128 positions per tile
   int cb_chunks, n_cb, kpt;
-  int st_taps;            // taps per weight stage (the last stage of a channel block holds 9 % st_taps, if not 0)
+  int taps;               // 9 (3x3 layers) or 1 (the 1x1 extension)
+  int st_taps;            // taps per weight stage (the last stage of a channel block holds taps % st_taps, if not 0)
   uint32_t tap_bytes;     // weights of one tap of one channel block and channel tile = kpt * 2 * Nt * 16
   int n_ntiles, total_tiles;
   const uint16_t* rank;   // [grid] CTA b takes this problem's tiles rank[b], rank[b] + grid, ...
@@ -162,18 +163,18 @@ __device__ __forceinline__ int g_first_tile(const GLayer& L) {
 template <int MODE, int MT, int KPT>
 __device__ __forceinline__ bool g_issue_block(uint64_t a_unit, uint32_t wq, uint32_t plane_units, bool s2, uint32_t a_step,
                                               uint64_t b_desc0, uint32_t b_slot_units, uint32_t b_step, uint32_t d0,
-                                              uint32_t nt, uint32_t idesc, uint32_t& acc, int st_taps, int NS,
+                                              uint32_t nt, uint32_t idesc, uint32_t& acc, int taps, int st_taps, int NS,
                                               uint32_t bar_bfull, uint32_t bar_bempty, int& b_slot, uint32_t& b_phase,
                                               bool leader, uint32_t sf, long long& tr_b) {
   uint32_t ky = 0, kx = 0;
   int t = 0;
 #pragma unroll 1
-  while (t < 9) {
+  while (t < taps) {
     // a weight stage holds whole taps: one wait, then nothing but MMAs until its last tap
     if (!TR_WAIT(tr_b, mbar_wait(bar_bfull + 8 * b_slot, b_phase))) return false;
     tc_fence_after();
     uint64_t bd = b_desc0 + (uint64_t)((uint32_t)b_slot * b_slot_units);
-    const int t_end = t + st_taps < 9 ? t + st_taps : 9;
+    const int t_end = t + st_taps < taps ? t + st_taps : taps;
 #pragma unroll 1
     for (; t < t_end; ++t) {
       // rows (16-byte units) from a unit's origin to tap (ky, kx): a shift inside the plane, plus, for stride 2,
@@ -277,11 +278,11 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       for (int l = 0; l < p.n_layers && ok; ++l) {
         const GLayer& L = lay[l];
         const int Nt = L.Nt, NtL = L.NtL, n_cb = L.n_cb, n_ntiles = L.n_ntiles, total = L.total_tiles;
-        const int st_taps = L.st_taps, stages_per_cb = (9 + st_taps - 1) / st_taps;
+        const int taps = L.taps, st_taps = L.st_taps, stages_per_cb = (taps + st_taps - 1) / st_taps;
         const int chunks_per_tap = 2 * L.kpt;
         const uint32_t tap_bytes = L.tap_bytes;
         const uint8_t* wt = L.wt;
-        const size_t cb_bytes = (size_t)9 * L.cb_chunks * NtL * 16;   // one channel block of one layout tile
+        const size_t cb_bytes = (size_t)taps * L.cb_chunks * NtL * 16;   // one channel block of one layout tile
         const FastDiv dNt = L.dNt;
         for (int tile = g_first_tile(L); tile < total && ok; tile += G) {
           if (*abort_flag) { ok = false; break; }
@@ -293,7 +294,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           for (int cb = 0; cb < n_cb && ok; ++cb) {
             const uint8_t* src = src_tile + (size_t)cb * cb_bytes;
             for (int sg = 0; sg < stages_per_cb; ++sg) {
-              const int ntaps = 9 - sg * st_taps < st_taps ? 9 - sg * st_taps : st_taps;
+              const int ntaps = taps - sg * st_taps < st_taps ? taps - sg * st_taps : st_taps;
               const uint32_t stage_bytes = (uint32_t)ntaps * tap_bytes;
               const int chunks_per_stage = ntaps * chunks_per_tap;
               if (b_issued >= NS && !TR_WAIT(tr_w0, mbar_wait_backoff(bar_bempty + 8 * b_slot, b_phase, 32))) { ok = false; break; }
@@ -364,7 +365,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
             const uint64_t a_unit = a_desc0 + (uint64_t)((uint32_t)a_slot * a_slot_units);
 #define G_ISSUE(M, KP)                                                                                       \
   ok = g_issue_block<MODE, M, KP>(a_unit, (uint32_t)L.Wq, (uint32_t)(L.cb_chunks * Rr), L.stride != 1, a_step, b_desc0, b_slot_units, b_step, d0, (uint32_t)Nt, idesc, acc, \
-                                  st_taps, NS, bar_bfull, bar_bempty, b_slot, b_phase, leader,                   \
+                                  L.taps, st_taps, NS, bar_bfull, bar_bempty, b_slot, b_phase, leader,                   \
                                   tmem_base + G_SCALE_COL, tr_w2)
 #define G_ISSUE_K(M)                   \
   do {                                 \
@@ -811,15 +812,15 @@ namespace {
 // layout tile.  Channels that do not exist are zeros, so whatever the activation operand holds there adds 0.
 template <int MODE>
 __global__ void g_expand_weights_kernel(const uint32_t* __restrict__ wplanes, uint8_t* __restrict__ wt, int C, int K,
-                                        int Cw, long long total, int cb_chunks, int n_cb, int NtL) {
+                                        int Cw, long long total, int cb_chunks, int n_cb, int NtL, int taps) {
   long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
   if (i >= total) return;
   int row = (int)(i % NtL);
   long long r = i / NtL;
   int c = (int)(r % cb_chunks);
   r /= cb_chunks;
-  int t = (int)(r % 9);
-  r /= 9;
+  int t = (int)(r % taps);
+  r /= taps;
   int cb = (int)(r % n_cb), tile = (int)(r / n_cb);
   int co = tile * NtL + row;
   constexpr int cpc = MODE == M_F16 ? 8 : 32;
@@ -844,14 +845,14 @@ __global__ void g_expand_weights_kernel(const uint32_t* __restrict__ wplanes, ui
 }
 
 cudaError_t g_expand_weights(int mode, const uint32_t* wplanes, void* dst, int C, int K, int Cw, int Kpad, int n_chunks,
-                             int cb_chunks, int NtL, cudaStream_t s) {
-  const long long total = (long long)9 * n_chunks * Kpad;
+                             int cb_chunks, int NtL, int taps, cudaStream_t s) {
+  const long long total = (long long)taps * n_chunks * Kpad;
   const unsigned blocks = (unsigned)((total + 255) / 256);
   const int n_cb = n_chunks / cb_chunks;
   if (mode == M_F16)
-    g_expand_weights_kernel<M_F16><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL);
+    g_expand_weights_kernel<M_F16><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL, taps);
   else
-    g_expand_weights_kernel<M_FP4><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL);
+    g_expand_weights_kernel<M_FP4><<<blocks, 256, 0, s>>>(wplanes, (uint8_t*)dst, C, K, Cw, total, cb_chunks, n_cb, NtL, taps);
   return cudaGetLastError();
 }
 
@@ -868,7 +869,11 @@ bool g_plan_layer(const Geom& g, int mode, GLayer* L, int* n_chunks_out, int* Kp
   GLayer& o = *L;
   o.N = g.N; o.H = g.H; o.W = g.W; o.C = g.C; o.K = g.K; o.Cw = g.Cw;
   o.stride = g.stride; o.pad = g.pad; o.Ho = g.Ho; o.Wo = g.Wo;
-  if (g.stride == 1) {
+  o.taps = g.ksize == 1 ? 1 : 9;
+  if (g.ksize == 1) {
+    // 1x1 layer: the positions are the output pixels themselves (input pixel = stride * output pixel), no halo
+    o.Hq = g.Ho; o.Wq = g.Wo; o.n_planes = 1; o.halo = 0;
+  } else if (g.stride == 1) {
     o.Hq = g.H + g.pad; o.Wq = g.W + g.pad; o.n_planes = 1; o.halo = 2 * o.Wq + 2;
   } else {
     o.Hq = g.Ho + 1; o.Wq = g.Wo + 1; o.n_planes = 4; o.halo = o.Wq + 1;
@@ -913,7 +918,7 @@ bool g_plan_layer(const Geom& g, int mode, GLayer* L, int* n_chunks_out, int* Kp
   o.tap_bytes = (uint32_t)(o.kpt * 2 * o.Nt * 16);
   int st = (int)(kGBSlot / o.tap_bytes);
   if (st < 1) return false;
-  o.st_taps = st > 9 ? 9 : st;
+  o.st_taps = st > o.taps ? o.taps : st;
   *n_chunks_out = raw;
   *Kpad_out = Kpad;
   return true;
@@ -954,7 +959,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
     const size_t pb = (size_t)host[i].n_planes * host[i].Rr * 4;
     if (pb > pix_bytes) pix_bytes = pb;
     w_off[i] = w_total;
-    w_total += ((size_t)9 * n_chunks[i] * Kpad[i] * 16 + 255) & ~(size_t)255;
+    w_total += ((size_t)host[i].taps * n_chunks[i] * Kpad[i] * 16 + 255) & ~(size_t)255;
     tiles += host[i].total_tiles;
   }
   a_slot = (a_slot + 127) & ~(size_t)127;
@@ -1031,7 +1036,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
     std::vector<int> order(grid);
     for (int i = 0; i < count; ++i) {
       const GLayer& o = host[i];
-      const double mma = (double)o.MT * o.n_cb * 9 * o.kpt * g_mma_cycles(o.Nt);
+      const double mma = (double)o.MT * o.n_cb * o.taps * o.kpt * g_mma_cycles(o.Nt);
       const double wr = 128.0 * o.MT * (o.Nt < o.K ? o.Nt : o.K) * 4 / 13.0;
       const double cost = (mma > wr ? mma : wr) + 300.0;
       for (int b = 0; b < grid; ++b) order[b] = b;
@@ -1078,7 +1083,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
       }
     }
     e = g_expand_weights(mode, Ls[i]->wplanes, G->weights + w_off[i], gs[i].C, gs[i].K, gs[i].Cw, Kpad[i],
-                         n_chunks[i], host[i].cb_chunks, host[i].NtL, s);
+                         n_chunks[i], host[i].cb_chunks, host[i].NtL, host[i].taps, s);
     if (e == cudaSuccess) *launched += 1;
   }
   if (e == cudaSuccess) e = cudaMemcpyAsync(G->layers_dev, host, sizeof(GLayer) * count, cudaMemcpyHostToDevice, s);
