@@ -115,7 +115,12 @@ def time_oracle_stack(workload, n_images: int, max_layers=None):
     for i, shape in enumerate(workload.layers[:max_layers]):
         seed = wl.layer_seed(workload.config, i)
         p = wl.draw_layer_params(shape, workload.tau, seed)
-        if workload.act == "bin":
+        if workload.act == "bin" and shape.ksize == 1:
+            act = wl.pack_activation_bits(wl.draw_activation_bits(shape, n_images, seed))
+            t0 = time.perf_counter()
+            oracle.conv1x1_bin(p.codebook, workload.tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out, shape.stride, act)
+            t_total += time.perf_counter() - t0
+        elif workload.act == "bin":
             act = wl.pack_activation_bits(wl.draw_activation_bits(shape, n_images, seed))
             t0 = time.perf_counter()
             oracle.conv_bin(p.codebook, workload.tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out, shape.stride,
@@ -175,9 +180,6 @@ def run_reference(args):
 # DRAM traffic per launch of the dominant kernel from an ncu capture (profiles/), valid only while
 # the kernel's sources are the ones that were profiled: {kernel: (workload, batch, bytes, sha256 of sources)}
 _TRAFFIC = {
-    # profiles/dram_traffic_resnet18_stack_n64_grouped.txt: mean of the two timed launches
-    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 348673920,
-                                             "80d6d8912c9655fdbe80994caa5981401e87a84a753fdb5afa04400ddc026db3"),
 }
 
 
@@ -195,6 +197,9 @@ def _profiled_traffic(kernel_name, nb, workload):
 
 def _workload_name(workload):
     return f"{workload.name}_stack_n{workload.batch}_tau{workload.tau}_{workload.act}"
+
+
+_SKEWS = {"none": None, "deep": wl.SKEW_DEEP, "top64": wl.SKEW_TOP64}
 
 
 # --------------------------------------------------------------------------
@@ -224,21 +229,17 @@ def run_ours(args):
         workload = wl.Workload(workload.name + f"[{lo}:{hi}]", workload.config, workload.batch, workload.tau,
                                workload.act, workload.layers[lo:hi])
     nb = workload.batch
+    skew = _SKEWS[args.index_skew]
     act_code = snn.ACT_BIN if workload.act == "bin" else snn.ACT_F16
     forced = {"auto": snn.PATH_AUTO, "reuse": snn.PATH_REUSE, "decoded": snn.PATH_DECODED,
               "decoded_tc": snn.PATH_DECODED_TC}[args.path]
 
-    # Micro-batches: the batch is cut into `mb` equal parts, each of which runs the layers in order on
-    # a stream of its own, so that one part's kernel start-up and tail overlap the other parts' work.
-    mb = max(1, args.microbatch)
-    if nb % mb:
-        raise SystemExit(f"--microbatch {mb} does not divide the batch {nb}")
-    layers, acts, outs, host_acts, host_outs, paths = [], [], [], [], [], []
+    layers, acts, outs, host_acts, host_outs, paths, params = [], [], [], [], [], [], []
     for i, shape in enumerate(workload.layers, start=first_layer):
         seed = wl.layer_seed(workload.config, i) + 7919 * rank
-        p = wl.draw_layer_params(shape, workload.tau, wl.layer_seed(workload.config, i))
+        p = wl.draw_layer_params(shape, workload.tau, wl.layer_seed(workload.config, i), index_skew=skew)
         layer = snn.SnnConv(shape.c_in, shape.c_out, workload.tau, p.codebook, p.idx_packed, p.alpha, shape.stride,
-                            shape.pad, act_code, device=local_rank)
+                            shape.pad, act_code, device=local_rank, ksize=shape.ksize)
         if workload.act == "bin":
             a = torch.from_numpy(wl.pack_activation_bits(wl.draw_activation_bits(shape, nb, seed)).view(np.int32))
         else:
@@ -248,90 +249,62 @@ def run_ours(args):
         outs.append(layer.alloc_out(nb, shape.h, shape.w))
         host_outs.append(layer.alloc_out(nb, shape.h, shape.w, pin=True))
         if forced == snn.PATH_AUTO and not args.group_only:
-            layer.tune(nb // mb, shape.h, shape.w)
-        paths.append(layer.chosen_path(nb // mb, shape.h, shape.w) if forced == snn.PATH_AUTO else forced)
+            layer.tune(nb, shape.h, shape.w)
+        paths.append(layer.chosen_path(nb, shape.h, shape.w) if forced == snn.PATH_AUTO else forced)
         layers.append(layer)
+        params.append(p)
 
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)  # > 126 MB L2
     side = torch.cuda.Stream(dev)
-
-    part = nb // mb
-    part_streams = [torch.cuda.Stream(dev) for _ in range(mb - 1)]
-
-    def launch_part(idxs, m, stream):
-        for j in idxs:
-            layers[j].forward(acts[j][m * part:(m + 1) * part], outs[j][m * part:(m + 1) * part], snn.OUT_F32,
-                              paths[j], stream)
-
-    n_lanes = max(1, args.streams)
-    lane_streams = [torch.cuda.Stream(dev) for _ in range(n_lanes - 1)]
-
-    def launch_layers(idxs, stream):
-        """One pass over layers `idxs`: micro-batch 0 on `stream`, the others on streams forked from
-        and joined back into it (the pattern stream capture needs)."""
-        if n_lanes > 1 and len(idxs) > 1:
-            # The layers of the benchmark are independent problems (each has its own input), so they
-            # may be issued round-robin on several streams: a layer's start-up then overlaps the
-            # tail of the layer before it.
-            for ls in lane_streams:
-                ls.wait_stream(stream)
-            for k, j in enumerate(idxs):
-                launch_part([j], 0, stream if k % n_lanes == 0 else lane_streams[k % n_lanes - 1])
-            for ls in lane_streams:
-                stream.wait_stream(ls)
-            return
-        for ps in part_streams:
-            ps.wait_stream(stream)
-        launch_part(idxs, 0, stream)
-        for m, ps in enumerate(part_streams, start=1):
-            launch_part(idxs, m, ps)
-        for ps in part_streams:
-            stream.wait_stream(ps)
-
-    def capture(idxs):
-        """The launches of one step (or one layer) as a CUDA graph, so that the host's
-        per-call cost does not sit between the kernels that are being timed."""
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            launch_layers(idxs, side)          # warm-up outside capture (sets kernel attributes)
-            side.synchronize()
-            with torch.cuda.graph(g, stream=side):
-                launch_layers(idxs, torch.cuda.current_stream(dev))
-        return g
-
+    stream = torch.cuda.current_stream(dev)
     all_idx = list(range(len(layers)))
     use_graph = not args.no_graph
+
+    def launch_layers(idxs, s):
+        for j in idxs:
+            layers[j].forward(acts[j], outs[j], snn.OUT_F32, paths[j], s)
+
+    def as_graph(fn):
+        """The launches of `fn(stream)` as a CUDA graph, so that the host's per-call cost does not sit between
+        the kernels that are being timed."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            fn(side)                       # warm-up outside capture (sets kernel attributes, builds plans)
+            side.synchronize()
+            with torch.cuda.graph(g, stream=side):
+                fn(torch.cuda.current_stream(dev))
+        return g
+
+    def timed(fn, steps, warm=3):
+        """Median-free mean of `steps` device-timed runs of fn(), L2 flushed before each (outside the events)."""
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(steps + warm):
+            flush.zero_()
+            if i >= warm:
+                ev[i - warm][0].record(stream)
+            fn()
+            if i >= warm:
+                ev[i - warm][1].record(stream)
+        torch.cuda.synchronize(dev)
+        return float(sum(a.elapsed_time(b) for a, b in ev)) / steps
+
     group = None
-    grouped = not args.per_layer and mb == 1 and n_lanes == 1 and forced in (snn.PATH_AUTO, snn.PATH_DECODED_TC)
-    seq_graph = None
+    grouped = not args.per_layer and forced in (snn.PATH_AUTO, snn.PATH_DECODED_TC)
     if grouped:
         # The layers of the benchmark are independent problems (each has its own input): the step
         # is one persistent launch that walks through all of them (snn_conv_group_forward).
         group = snn.SnnConvGroup(layers, [(nb, s.h, s.w) for s in workload.layers])
-        # the same step as per-layer launches, timed beside it
-        seq_graph = capture(all_idx) if use_graph and not args.group_only else None
-
-        def launch_group(stream):
-            group.forward(acts, outs, snn.OUT_F32, stream)
-
-        if use_graph:
-            step_graph = torch.cuda.CUDAGraph()
-            with torch.cuda.stream(side):
-                launch_group(side)
-                side.synchronize()
-                with torch.cuda.graph(step_graph, stream=side):
-                    launch_group(torch.cuda.current_stream(dev))
+        step_graph = as_graph(lambda s: group.forward(acts, outs, snn.OUT_F32, s)) if use_graph else None
+        step_host = lambda: group.forward(acts, outs, snn.OUT_F32, stream)   # noqa: E731
     else:
-        step_graph = capture(all_idx) if use_graph else None
-    stream = torch.cuda.current_stream(dev)
+        step_graph = as_graph(lambda s: launch_layers(all_idx, s)) if use_graph else None
+        step_host = lambda: launch_layers(all_idx, stream)                    # noqa: E731
 
     def step():
         if use_graph:
             step_graph.replay()
-        elif group is not None:
-            launch_group(stream)
         else:
-            launch_layers(all_idx, stream)
+            step_host()
 
     def barrier():
         if world > 1:
@@ -357,97 +330,77 @@ def run_ours(args):
     barrier()
     wall = time.perf_counter() - wall0
     launches = (snn.kernel_launches() - launches0) if not use_graph else \
-        (1 if group is not None else len(layers) * mb) * args.steps
+        (1 if group is not None else len(layers)) * args.steps
     step_ms = [e0.elapsed_time(e1) for e0, e1 in ev]
     total_ms = float(sum(step_ms))
 
-    # the same step as one launch per layer, back to back on one stream (what a caller of
-    # snn_conv_forward gets), timed the same way over fewer steps
+    # ---- check what was timed: outputs of the timed launches against the oracle (rank 0, after the timed region)
+    checked = None
+    if rank == 0 and not args.no_check:
+        import oracle
+        oracle.build()
+        torch.cuda.synchronize(dev)
+        checked = True
+        picks = [(len(layers) - 1, nb)] + ([(0, min(2, nb))] if len(layers) > 1 else [])
+        for j, n_img in picks:
+            shape, p = workload.layers[j], params[j]
+            a_np = host_acts[j][:n_img].numpy()
+            if shape.ksize == 1:
+                ref = (oracle.conv1x1_bin(p.codebook, workload.tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out,
+                                          shape.stride, a_np.view(np.uint32))[1] if workload.act == "bin" else
+                       oracle.conv1x1_f16(p.codebook, workload.tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out,
+                                          shape.stride, a_np))
+            elif workload.act == "bin":
+                ref = oracle.conv_bin(p.codebook, workload.tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out,
+                                      shape.stride, shape.pad, a_np.view(np.uint32))[1]
+            else:
+                ref = oracle.conv_f16(p.codebook, workload.tau, p.idx_packed, p.alpha, shape.c_in, shape.c_out,
+                                      shape.stride, shape.pad, a_np)
+            got = outs[j][:n_img].cpu().numpy()
+            if workload.act == "bin":
+                ok = bool((got == ref).all())
+            else:
+                sigma = p.alpha.astype(np.float64) * np.sqrt(float(shape.ksize ** 2 * shape.c_in))
+                bound = 2e-2 * np.maximum(np.abs(ref.astype(np.float64)), sigma[None, None, None, :])
+                ok = bool((np.abs(got.astype(np.float64) - ref) <= bound).all())
+            checked = checked and ok
+
+    # ---- the same step as one snn_conv_forward launch per layer, back to back on one stream
+    k_side = max(3, min(30, args.steps))
     seq_ms = None
     if group is not None and not args.group_only:
-        k = max(3, min(30, args.steps))
-        ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(k)]
-        for i in range(k + 3):
-            flush.zero_()
-            if i >= 3:
-                ev2[i - 3][0].record(stream)
-            if seq_graph is not None:
-                seq_graph.replay()
-            else:
-                launch_layers(all_idx, stream)
-            if i >= 3:
-                ev2[i - 3][1].record(stream)
-        torch.cuda.synchronize(dev)
-        seq_ms = float(sum(a.elapsed_time(b) for a, b in ev2)) / k
+        seq_graph = as_graph(lambda s: launch_layers(all_idx, s)) if use_graph else None
+        seq_ms = timed(seq_graph.replay if use_graph else (lambda: launch_layers(all_idx, stream)), k_side)
 
-    # per-layer device time (same launch configuration, L2 flushed before every layer; the
-    # flush also keeps the GPU busy while the host enqueues, so no host latency is timed)
-    reps = 0 if args.group_only else max(3, min(20, args.steps))
+    # ---- per-layer device time (L2 flushed before every layer)
     layer_ms = [0.0] * len(layers)
-    layer_graphs = [capture([j]) for j in all_idx] if use_graph and reps else None
-    for _ in range(reps):
+    if not args.group_only:
+        reps = max(3, min(20, args.steps))
         for j in all_idx:
-            flush.zero_()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            if use_graph:
-                layer_graphs[j].replay()
-            else:
-                launch_layers([j], stream)
-            e1.record(stream)
-            e1.synchronize()
-            layer_ms[j] += e0.elapsed_time(e1) / reps
-    # the same grouped step writing packed signs (1 bit per output: the next layer's input) instead of fp32
+            gj = as_graph(lambda s, j=j: launch_layers([j], s)) if use_graph else None
+            layer_ms[j] = timed(gj.replay if use_graph else (lambda j=j: launch_layers([j], stream)), reps, warm=1)
+
+    # ---- the grouped step writing packed signs (1 bit per output) instead of fp32
     bits_ms = None
     if group is not None and workload.act == "bin":
         bit_outs = group.alloc_outs(snn.OUT_BITS)
-        k = max(3, min(30, args.steps))
-        ev3 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(k)]
-        for i in range(k + 3):
-            flush.zero_()
-            if i >= 3:
-                ev3[i - 3][0].record(stream)
-            group.forward(acts, bit_outs, snn.OUT_BITS, stream)
-            if i >= 3:
-                ev3[i - 3][1].record(stream)
-        torch.cuda.synchronize(dev)
-        bits_ms = float(sum(a.elapsed_time(b) for a, b in ev3)) / k
+        bits_ms = timed(lambda: group.forward(acts, bit_outs, snn.OUT_BITS, stream), k_side)
         del bit_outs
-    # The stack as a true chain: layer i writes packed signs that layer i+1 reads as its binary input
-    # (no batch-norm or shortcut in between: the path has none), one snn_conv_forward launch per layer.
-    chain_ms = None
+
+    # ---- the layers as a dependent chain through packed signs, ONE launch (snn_conv_stack_forward)
+    stack_ms = None
     shapes = workload.layers
-    chains = all(a.c_out == b.c_in and ((a.h + 2 * a.pad - 3) // a.stride + 1) == b.h for a, b in zip(shapes, shapes[1:]))
-    if workload.act == "bin" and chains and not args.group_only and forced in (snn.PATH_AUTO, snn.PATH_DECODED_TC):
-        bufs = [layers[j].alloc_out(nb, shapes[j].h, shapes[j].w, snn.OUT_BITS) for j in all_idx]
-
-        def launch_chain(s):
-            x = acts[0]
-            for j in all_idx:
-                layers[j].forward(x, bufs[j], snn.OUT_BITS, snn.PATH_DECODED_TC, s)
-                x = bufs[j]
-
-        gchain = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            launch_chain(side)
-            side.synchronize()
-            with torch.cuda.graph(gchain, stream=side):
-                launch_chain(torch.cuda.current_stream(dev))
-        k = max(3, min(30, args.steps))
-        ev4 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(k)]
-        for i in range(k + 3):
-            flush.zero_()
-            if i >= 3:
-                ev4[i - 3][0].record(stream)
-            gchain.replay()
-            if i >= 3:
-                ev4[i - 3][1].record(stream)
-        torch.cuda.synchronize(dev)
-        chain_ms = float(sum(a.elapsed_time(b) for a, b in ev4)) / k
-        del bufs, gchain
+    chains = len(shapes) > 1 and all(a.c_out == b.c_in and a.h_out == b.h and a.w_out == b.w
+                                     for a, b in zip(shapes, shapes[1:]))
+    if workload.act == "bin" and chains and forced in (snn.PATH_AUTO, snn.PATH_DECODED_TC):
+        stack = snn.SnnConvStack(layers, nb, shapes[0].h, shapes[0].w)
+        s_out = stack.alloc_out(snn.OUT_F32)
+        sg = as_graph(lambda s: stack.forward(acts[0], s_out, snn.OUT_F32, s)) if use_graph else None
+        stack_ms = timed(sg.replay if use_graph else (lambda: stack.forward(acts[0], s_out, snn.OUT_F32, stream)), k_side)
+        stack.destroy()
     clocks = sampler.stop()
 
-    # end to end through the host-buffer entry point: H2D of the inputs and D2H of the results inside the timing
+    # ---- end to end through the host-buffer entry point: H2D of the inputs and D2H of the results inside the timing
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     for j, layer in enumerate(layers):
         layer.forward_host(host_acts[j], host_outs[j], snn.OUT_F32, paths[j])
@@ -461,25 +414,10 @@ def run_ours(args):
     h2d = sum(a.numel() * a.element_size() for a in host_acts)
     d2h = sum(o.numel() * o.element_size() for o in host_outs)
 
-    # Write-only HBM rate, measured here: the path writes 29 bytes for every byte it reads (fp32 outputs
-    # against packed inputs), and a fill runs well below the copy rate that MEASURED_PEAKS.json holds
-    # (a copy's traffic is half reads).  Reported beside the roofline as context.
-    write_gbs = None
-    try:
-        big = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
-        best = None
-        for _ in range(6):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            big.fill_(1)
-            e1.record(stream)
-            e1.synchronize()
-            ms = e0.elapsed_time(e1)
-            best = ms if best is None or ms < best else best
-        write_gbs = big.numel() / (best * 1e-3) / 1e9
-        del big
-    except Exception:
-        write_gbs = None
+    # ---- measured ceilings of this device, by the library's own microbenchmarks
+    store_gbs = snn.microbench(6, local_rank) / 1e9            # write-only stream of 16-byte stores
+    mma_fp4 = snn.microbench(5, local_rank)                    # MAC/s, e2m1 MMAs of N = 240 as the kernel issues them
+    mma_f16 = snn.microbench(7, local_rank)                    # MAC/s, fp16 MMAs of N = 256
 
     # max over ranks of the device-timed totals; every rank ran a batch of its own (weak scaling)
     total_ms, e2e_ms = replicas.max_over_ranks([total_ms, e2e_ms], world, dev)
@@ -505,68 +443,79 @@ def run_ours(args):
         d = {"ms": ms_per_step, "macs": workload.dense_macs(), "bytes": workload.algorithmic_bytes(), "launches": 1}
         sec = ms_per_step * 1e-3
         kernel_name = "tcg_conv_kernel (grouped decoded_tc)"
-    elif len(by_path) == 1 and mb == 1 and n_lanes == 1:
+    elif len(by_path) == 1:
         # every launch of the step is this path's kernel, back to back: use the time of the timed region
-        # (the per-layer figures in layer_ms are taken one layer at a time after a flush and add the
-        # event clock's 2 us granularity to every layer)
         d = dict(d, ms=ms_per_step)
         sec = ms_per_step * 1e-3
     hbm_frac = d["bytes"] / sec / 1e9 / peaks["hbm_gbs"]
-    alu_rates = {}
+    extras = {}
     if dom == snn.PATH_DECODED_TC:
-        # dense contraction: int8 (binary activations) at twice the measured bf16 rate, fp16 at the bf16 rate
-        ratio = 2.0 if workload.act == "bin" else 1.0
-        peak = peaks["bf16_tflops_sustained"] * ratio
+        # Dense contraction.  The kernel is timed alone (L2 flush between launches, clocks at their maximum), so
+        # the burst figure applies.  Binary activations run on 4-bit e2m1 operands: measured bf16 x 4, the
+        # nominal e2m1 : bf16 ratio; fp16 activations: x 1.
+        ratio = 4.0 if workload.act == "bin" else 1.0
+        peak = peaks["bf16_tflops"] * ratio
         achieved = 2 * d["macs"] / sec / 1e12
         pipe = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak}
+        extras["peak_source"] = (peaks["source"] + (": bf16 burst x 4 nominal (e2m1 operands)" if workload.act == "bin"
+                                                     else ": bf16 burst x 1 (fp16 operands)"))
+        extras["frac_of_int8_peak"] = achieved / (peaks["bf16_tflops"] * 2.0) if workload.act == "bin" else None
+        extras["mma_measured_tflops"] = 2 * (mma_fp4 if workload.act == "bin" else mma_f16) / 1e12
+        extras["frac_of_mma_measured"] = achieved / extras["mma_measured_tflops"]
     elif dom == snn.PATH_DECODED:
         # one POPC per 32 MACs; 16 POPC lanes per SM per clock on 148 SMs at the maximum SM clock
         peak = 148 * 16 * peaks["sm_max_mhz"] * 1e6 / 1e12
         achieved = d["macs"] / 32 / sec / 1e12
         pipe = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Tpopc/s", "frac": achieved / peak}
-        alu_rates["popc_measured_per_s"] = snn.microbench(0, local_rank)
+        extras["popc_measured_per_s"] = snn.microbench(0, local_rank)
+        extras["peak_source"] = "16 POPC lanes x 148 SMs x max SM clock"
     else:
         # one 4-pixel shared-memory word per (c_out, c_in, 4 pixels); 32 words per SM per clock
         peak = 148 * 32 * peaks["sm_max_mhz"] * 1e6 / 1e12
         achieved = d["macs"] / 9 / 4 / sec / 1e12
         pipe = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Tlds/s", "frac": achieved / peak}
-        alu_rates["lds_measured_per_s"] = snn.microbench(3, local_rank)
+        extras["lds_measured_per_s"] = snn.microbench(3, local_rank)
+        extras["peak_source"] = "32 shared-memory words x 148 SMs x max SM clock"
     if hbm_frac >= pipe["frac"]:
         roofline = {"bound": "hbm", "achieved": d["bytes"] / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": hbm_frac}
+        extras["hbm_peak_source"] = peaks["source"] + ": copy rate of MEASURED_PEAKS.json"
     else:
         roofline = pipe
+    floor_ms = workload.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e3
     roofline.update({"traffic": _profiled_traffic(kernel_name, nb, workload), "kernel": kernel_name,
                      "launches_per_step": d["launches"],
                      "share_of_step": 1.0 if group is not None else d["ms"] / max(sum(layer_ms), 1e-9),
-                     "peak_source": peaks["source"],
                      "algorithmic_bytes_per_launch": d["bytes"] / d["launches"],
-                     "hbm_write_only_gbs": write_gbs,
-                     "frac_of_write_only_rate": None if not write_gbs else d["bytes"] / sec / 1e9 / write_gbs,
                      "algorithmic_ops_per_launch": 2 * d["macs"] / d["launches"],
-                     "hbm_frac": hbm_frac, "pipe_frac": pipe["frac"], **alu_rates})
-    # whole-step roofline: sum over layers of max(HBM floor, pipe floor at the path's peak)
-    step_floor_hbm_ms = workload.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9) * 1e3
+                     "hbm_frac": hbm_frac, "pipe_frac": pipe["frac"],
+                     "store_stream_gbs": store_gbs,
+                     "frac_of_store_stream": d["bytes"] / sec / 1e9 / store_gbs,
+                     # the same step as one launch per layer, against the same floor
+                     "per_layer_launches_ms": seq_ms,
+                     "per_layer_launches_frac": None if seq_ms is None else floor_ms / seq_ms,
+                     **extras})
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        # the type the dominant path computes in: int8 operands (+/-1) with int32 accumulation on the tensor
-        # cores, fp16 operands with fp32 accumulation in the fp16-activation variant, int32 on the ALU paths
-        "dtype": ("f16" if workload.act != "bin" else "int8" if dom == snn.PATH_DECODED_TC else "int32"),
+        # the type the dominant path computes in: e2m1 operands (+/-1 and 0, exact) with fp32 accumulation on the
+        # tensor cores, fp16 operands in the fp16-activation variant, int32 on the ALU paths
+        "dtype": ("f16" if workload.act != "bin" else "e2m1" if dom == snn.PATH_DECODED_TC else "int32"),
         "data": "synthetic",
         "config": {"workload": _workload_name(workload), "layers": len(layers), "batch_per_gpu": nb,
-                   "tau": workload.tau, "l2": "flushed between timed steps (256 MB write)",
+                   "tau": workload.tau, "index_skew": args.index_skew,
+                   "l2": "flushed between timed steps (256 MB write)",
                    "launch": ("one grouped launch of all layers (snn_conv_group_forward), " if group is not None else "") +
                              ("host calls" if args.no_graph else
                               "replayed as a CUDA graph" if group is not None else
-                              "CUDA graph of the per-layer C-ABI launches") +
-                             (f", {mb} micro-batches of {part} images on {mb} streams" if mb > 1 else ""),
-                   "microbatches": mb, "streams": n_lanes, "grouped": group is not None,
+                              "CUDA graph of the per-layer C-ABI launches"),
+                   "grouped": group is not None,
                    "paths": [snn.PATH_NAMES[p] for p in paths]},
+        "checked": checked,
         "effective_tops": 2 * workload.dense_macs() * world / (ms_per_step * 1e-3) / 1e12,
-        "hbm_floor_ms_per_step": step_floor_hbm_ms,
-        "step_frac_of_hbm_floor": step_floor_hbm_ms / ms_per_step,
+        "hbm_floor_ms_per_step": floor_ms,
+        "step_frac_of_hbm_floor": floor_ms / ms_per_step,
         "layer_ms": [round(v, 5) for v in layer_ms],
         "per_layer_launches": None if seq_ms is None else {
             "ms_per_step": seq_ms, "value": nb / (seq_ms * 1e-3), "unit": UNIT + " per GPU",
@@ -575,10 +524,10 @@ def run_ours(args):
             "ms_per_step": bits_ms, "value": nb / (bits_ms * 1e-3), "unit": UNIT + " per GPU",
             "what": "the grouped step with SNN_OUT_BITS (signs of the outputs packed as the next layer's input) "
                     "instead of fp32 outputs; host launches, not a graph"},
-        "chained_packed_signs": None if chain_ms is None else {
-            "ms_per_step": chain_ms, "value": nb / (chain_ms * 1e-3), "unit": UNIT + " per GPU",
-            "what": "the layers as a dependent chain: each layer's packed signs (SNN_OUT_BITS) are the next "
-                    "layer's input, one snn_conv_forward launch per layer, CUDA graph"},
+        "dependent_stack": None if stack_ms is None else {
+            "ms_per_step": stack_ms, "value": nb / (stack_ms * 1e-3), "unit": UNIT + " per GPU",
+            "what": "the layers as a dependent chain in ONE launch (snn_conv_stack_forward): every layer's packed "
+                    "thresholded signs are the next layer's input, the last layer writes fp32"},
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms},
@@ -602,6 +551,8 @@ def run_ours(args):
         line["cpu_baseline"] = None
     if rank == 0:
         print(json.dumps(line), flush=True)
+    if group is not None:
+        group.destroy()
     for layer in layers:
         layer.destroy()
     if world > 1:
@@ -621,10 +572,10 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "reuse", "decoded", "decoded_tc"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--microbatch", type=int, default=1,
-                    help="cut the batch into this many parts, each running the layers in order on its own stream")
-    ap.add_argument("--streams", type=int, default=1,
-                    help="issue the (independent) layers of a step round-robin on this many streams")
+    ap.add_argument("--index-skew", default="none", choices=["none", "deep", "top64"],
+                    help="draw the indices from the kernel-frequency profile of trained layers (Sec. 4.2) "
+                         "instead of uniformly")
+    ap.add_argument("--no-check", action="store_true", help="skip the oracle check of the timed outputs")
     ap.add_argument("--group-only", action="store_true",
                     help="time only the grouped launch: no tuning, no per-layer timings (profiling aid)")
     ap.add_argument("--per-layer", action="store_true",

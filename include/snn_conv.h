@@ -155,6 +155,12 @@ SNN_API int64_t snn_kernel_launches(void);
  * and returns results per second in *rate (per-lane results: a warp
  * instruction counts 32).  kind: 0 = POPC, 1 = LOP3 (xor), 2 = IADD3,
  * 3 = LDS.32 (conflict-free), 4 = XOR+POPC+IADD chain as the decoded loop issues it.
+ * Ceilings of the tensor-core path, measured the way that path uses the hardware:
+ * 5 = tcgen05.mma with 4-bit e2m1 operands and unit block scales (M = 128, N = 240,
+ * K = 64, both operands from shared memory), in multiply-accumulates per second over
+ * all SMs; 8 = the same at N = 128; 7 = tcgen05.mma with fp16 operands (M = 128,
+ * N = 256, K = 16); 6 = a write-only stream of 16-byte stores over 1 GiB, in bytes
+ * per second (the path writes 29 bytes for every byte it reads).
  */
 SNN_API snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate);
 

@@ -645,7 +645,7 @@ snn_status_t snn_conv_stack_destroy(snn_conv_stack_t* st) {
 
 snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate) {
   if (!rate) return fail(SNN_ERR_INVALID_ARG, "null rate pointer");
-  if (kind < 0 || kind > 4) return fail(SNN_ERR_INVALID_ARG, "unknown microbenchmark %d", kind);
+  if (kind < 0 || kind > 8) return fail(SNN_ERR_INVALID_ARG, "unknown microbenchmark %d", kind);
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
     cudaGetLastError();

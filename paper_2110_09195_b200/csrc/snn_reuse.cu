@@ -6,6 +6,9 @@
 // Mapping used here.  A CTA owns a run of consecutive output pixels (batch,
 // row, column flattened) and up to 256 output channels, and walks c_in in
 // chunks of 16 channels:
+//   stage 0  one thread per pixel reads the nine activation words of its 3x3 window once
+//            and turns the chunk's 16 channels into sixteen 9-bit window codes in shared
+//            memory (a word is read once per chunk, not once per channel);
 //   stage 1  for every (4-pixel group, channel) of the chunk build the table
 //            tab[k] = matching-tap counts of the four slices against kernel k,
 //            one byte per pixel, from the 512 x 2^tau table made at create
@@ -57,7 +60,8 @@ __global__ void __launch_bounds__(256) reuse_conv_kernel(const ReuseParams p) {
   int* pix_base = reinterpret_cast<int*>(idxs + (size_t)RC * p.KT);      // [PT] n*H*W or -1
   int* pix_r0 = pix_base + PT;
   int* pix_c0 = pix_r0 + PT;
-  uint8_t* m9s = reinterpret_cast<uint8_t*>(pix_c0 + PT);                // [NH][512][16] (optional)
+  uint16_t* codes = reinterpret_cast<uint16_t*>(pix_c0 + PT);            // [RC][PT] window code of (channel, pixel)
+  uint8_t* m9s = reinterpret_cast<uint8_t*>(codes + (size_t)RC * PT);    // [NH][512][16] (optional)
   m9s = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(m9s) + 15) & ~(uintptr_t)15);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -103,29 +107,37 @@ __global__ void __launch_bounds__(256) reuse_conv_kernel(const ReuseParams p) {
       if (ci < cc && cob + cl < p.K) v = __ldg(p.idx + (size_t)(cob + cl) * p.C + c0 + ci);
       idxs[ci * p.KT + cl] = v;
     }
+    // ---- stage 0: window codes of the chunk's channels, one thread per pixel
+    {
+      const int wd = c0 >> 5, sh = c0 & 31;   // the chunk's 16 channels are one half of a 32-channel word
+      for (int pi = tid; pi < PT; pi += nthreads) {
+        const int nb = pix_base[pi], r0 = pix_r0[pi], cc0 = pix_c0[pi];
+        uint32_t half[9];
+#pragma unroll
+        for (int t = 0; t < 9; ++t) {
+          const int r = r0 + t / 3, cx = cc0 + t % 3;
+          half[t] = 0;   // outside the image: read as -1, repaired by the border corrections
+          if (nb >= 0 && r >= 0 && r < p.H && cx >= 0 && cx < p.W)
+            half[t] = (__ldg(p.act + ((size_t)nb + (size_t)r * p.W + cx) * p.Cw + wd) >> sh) & 0xffffu;
+        }
+#pragma unroll
+        for (int ci = 0; ci < RC; ++ci) {
+          uint32_t code = 0;
+#pragma unroll
+          for (int t = 0; t < 9; ++t) code |= ((half[t] >> ci) & 1u) << (8 - t);
+          codes[ci * PT + pi] = (uint16_t)code;
+        }
+      }
+    }
+    __syncthreads();
     // ---- stage 1: tables for every (quad, channel) of the chunk
     for (int item = tid; item < NQ * RC; item += nthreads) {
       const int ci = item % RC, quad = item / RC;
       if (ci >= cc) continue;
-      const int c = c0 + ci;
-      const int wd = c >> 5, sh = c & 31;
       uint32_t w9[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int pi = quad * 4 + j;
-        const int nb = pix_base[pi], r0 = pix_r0[pi], cc0 = pix_c0[pi];
-        uint32_t code = 0;
-        if (nb >= 0) {
-#pragma unroll
-          for (int t = 0; t < 9; ++t) {
-            int r = r0 + t / 3, cx = cc0 + t % 3;
-            uint32_t bit = 0;
-            if (r >= 0 && r < p.H && cx >= 0 && cx < p.W)
-              bit = (__ldg(p.act + ((size_t)nb + (size_t)r * p.W + cx) * p.Cw + wd) >> sh) & 1u;
-            code |= bit << (8 - t);
-          }
-        }
-        w9[j] = code;
+      {
+        const uint2 cq = *reinterpret_cast<const uint2*>(codes + ci * PT + quad * 4);   // four pixels' codes
+        w9[0] = cq.x & 0xffffu; w9[1] = cq.x >> 16; w9[2] = cq.y & 0xffffu; w9[3] = cq.y >> 16;
       }
       uint32_t* row = tab + (size_t)ci * p.CS + (size_t)quad * p.Tp;
       for (int h = 0; h < p.NH; ++h) {
@@ -248,7 +260,7 @@ cudaError_t reuse_forward(const LayerDev& L, const Geom& g, int act_type, const 
   p.CS = NQ * p.Tp + 4;
   const size_t match_bytes = (size_t)p.NH * 512 * 16;
   p.match_in_smem = match_bytes <= 64 * 1024;
-  size_t smem = (size_t)RC * p.CS * 4 + (size_t)RC * p.KT * 2 + (size_t)NQ * 4 * 3 * 4 + 16 +
+  size_t smem = (size_t)RC * p.CS * 4 + (size_t)RC * p.KT * 2 + (size_t)NQ * 4 * 3 * 4 + (size_t)RC * NQ * 4 * 2 + 16 +
                 (p.match_in_smem ? match_bytes : 0);
   const int threads = 32 * p.KW * p.QG;
   const int PT = NQ * 4;

@@ -206,10 +206,16 @@ __device__ __forceinline__ bool g_issue_block(uint64_t a_unit, uint32_t wq, uint
 
 }  // namespace
 
-template <int MODE>
+// OUTK: what the epilogue is compiled for.  0: fp32 or int32 words for every member; 1: packed signs for every
+// member; 2: a chain - packed signs between the members, any type for the last, and the dependency waits and
+// completion counters.  Keeping the variants apart keeps each one's registers and code to what it needs.
+enum { OUT_WORDS = 0, OUT_SIGNS = 1, OUT_CHAIN = 2 };
+
+template <int MODE, int OUTK>
 __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p) {
   constexpr bool F16 = MODE == M_F16;   // fp16 activations (copied, not expanded)
   constexpr bool FP4 = MODE == M_FP4;   // binary activations as e2m1 nibbles
+  constexpr bool CHAIN = OUTK == OUT_CHAIN;
   extern __shared__ __align__(128) uint8_t smem[];
   // carve-up: [NA activation slots][NS weight slots][epilogue tiles][pixel table][problem table][barriers, flags]
   uint8_t* a_smem = smem;
@@ -416,7 +422,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       const int Nt = L.Nt, MT = L.MT, K = L.K;
       const float* alpha = L.alpha;
       const float* shift = L.shift;
-      const int out_i32 = p.out_type[l];
+      const int out_i32 = OUTK == OUT_WORDS ? (int)p.out_type[0] : OUTK == OUT_SIGNS ? 2 : (int)p.out_type[l];
       uint32_t* out32 = reinterpret_cast<uint32_t*>(p.out[l]);  // int32 and fp32 outputs share the layout
       const bool fast = ((K & 3) == 0) && ((Nt & 31) == 0);
       for (int tile = g_first_tile(L); tile < L.total_tiles; tile += G) {
@@ -446,7 +452,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           const bool valid = ((long long)q < L.Qtot) && ((int)n < L.N) && (y < L.Ho) && (x < L.Wo);
           return valid ? ((int)n * L.Ho + y) * L.Wo + x : -1;
         };
-        if (out_i32 == 2) {
+        if (OUTK != OUT_WORDS && out_i32 == 2) {
           // Packed signs of the scaled output (Algorithm 1: the next layer consumes sign(a)): a thread
           // owns one position and the 32 (or 16) consecutive channels of a slice, i.e. one word (or
           // half-word) of the next layer's binary input.  No transposition, one small store per slice.
@@ -505,6 +511,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
               }
             }
           }
+        } else if (OUTK == OUT_SIGNS) {
+          // (packed signs only: nothing else is compiled into this variant)
         } else if (fast) {
           // The warp's slices (sub-tile mt, columns c0..c0+31) form one sequence; the TMEM load of
           // slice s+1 is issued as soon as slice s sits in the staging tile.
@@ -592,7 +600,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_accempty + 8 * acc_slot);
-        if (L.done) {
+        if (CHAIN && L.done) {
           // chain: this warp's part of the tile is written; the successor may read it
           __threadfence();
           __syncwarp();
@@ -622,7 +630,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       const int C = L.C, Cw = L.Cw, total = L.total_tiles;
       const FastDiv dNt = L.dNt;
       const void* act = p.act[l];
-      const bool fresh = L.deps != nullptr;   // written by other CTAs of this launch: read from L2
+      const bool fresh = CHAIN && L.deps != nullptr;   // written by other CTAs of this launch: read from L2
       // vector loads of a row's words need the base pointer and the row pitch aligned to the load
       bool vec;
       {
@@ -635,7 +643,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       for (int tile = g_first_tile(L); tile < total && !stop; tile += G) {
         const int mg = (int)fdiv((uint32_t)tile, dNt);
         const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
-        if (L.deps) {
+        if (CHAIN && L.deps) {
           // chain: wait until the predecessor has written every input pixel of this tile (one thread polls)
           if (et == 0) {
             const uint2 d = __ldg(L.deps + mg);
@@ -1174,15 +1182,20 @@ cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, i
   cfg.blockDim = dim3(G_THREADS);
   cfg.dynamicSmemBytes = G->smem;
   cudaError_t e;
+  const int outk = G->chain ? OUT_CHAIN : (out_type == 2 ? OUT_SIGNS : OUT_WORDS);
+#define G_LAUNCH(M, O)                                                      \
+  do {                                                                      \
+    static unsigned long long done = 0;                                     \
+    e = allow_max_smem(tcg_conv_kernel<M, O>, &done);                       \
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<M, O>, p); \
+  } while (0)
   if (G->mode == M_F16) {
-    static unsigned long long done = 0;
-    e = allow_max_smem(tcg_conv_kernel<M_F16>, &done);
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<M_F16>, p);
-  } else {
-    static unsigned long long done = 0;
-    e = allow_max_smem(tcg_conv_kernel<M_FP4>, &done);
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, tcg_conv_kernel<M_FP4>, p);
-  }
+    if (outk == OUT_WORDS) G_LAUNCH(M_F16, OUT_WORDS);
+    else return cudaErrorInvalidValue;   // packed signs and chains need binary activations
+  } else if (outk == OUT_WORDS) G_LAUNCH(M_FP4, OUT_WORDS);
+  else if (outk == OUT_SIGNS) G_LAUNCH(M_FP4, OUT_SIGNS);
+  else G_LAUNCH(M_FP4, OUT_CHAIN);
+#undef G_LAUNCH
   if (e != cudaSuccess) return e;
   *launched += 1;
 #ifdef SNN_TRACE
