@@ -201,6 +201,10 @@ __device__ __forceinline__ uint32_t spread_pairs16(uint32_t x) {
   x = (x | (x << 2)) & 0x33333333u;
   return x;
 }
+// 16 bytes to shared memory at a 32-bit shared-space address
+__device__ __forceinline__ void sts16(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
 __device__ __forceinline__ uint4 expand_word_fp4(uint32_t bits, bool present) {
   if (!present) return make_uint4(0, 0, 0, 0);
   const uint32_t lut = 0x222aa2aau;  // byte i = nibble pair of the 2-bit value i

@@ -44,6 +44,7 @@ namespace {
 // operands.  Both accumulate in fp32.
 enum { M_F16 = 1, M_FP4 = 2 };
 constexpr int G_EW = 8;                       // epilogue warps = expander warps
+
 // Warps 13 and 17 stay idle: a warp's scheduler is warp % 4, and the MMA-issuing warp (1) then
 // shares its scheduler with two epilogue warps only instead of two epilogue and two expander warps.
 constexpr int G_THREADS = 64 + 64 * G_EW + 64;
@@ -216,6 +217,12 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
   constexpr bool F16 = MODE == M_F16;   // fp16 activations (copied, not expanded)
   constexpr bool FP4 = MODE == M_FP4;   // binary activations as e2m1 nibbles
   constexpr bool CHAIN = OUTK == OUT_CHAIN;
+  // Word outputs (fp32 / int32) are bound by the stores: there the epilogue warps form two groups of four (one
+  // warp per quarter of the accumulator's lanes) that take the tiles in turn, group g draining accumulator
+  // buffer g, so that one group's stores drain while the other reads tensor memory and transposes.  Packed
+  // signs are bound by the epilogue's instructions: all eight warps drain every tile together.
+  constexpr bool G_EPI_SPLIT = OUTK == OUT_WORDS;
+  constexpr int G_EPI_ARRIVALS = G_EPI_SPLIT ? G_EW / 2 : G_EW;   // epilogue warps that drain one tile
   extern __shared__ __align__(128) uint8_t smem[];
   // carve-up: [NA activation slots][NS weight slots][epilogue tiles][pixel table][problem table][barriers, flags]
   uint8_t* a_smem = smem;
@@ -240,7 +247,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 
   if (tid < 28) {
     uint32_t count = 1;
-    if (tid >= 26) count = G_EW;                       // acc_empty: one arrival per epilogue warp
+    if (tid >= 26) count = G_EPI_ARRIVALS;             // acc_empty: one arrival per epilogue warp of the tile
     if (tid >= 16 && tid < 20) count = G_EXP_THREADS;  // a_full: every expander thread arrives
     mbar_init(smem_u32(bars + tid), count);
   }
@@ -410,9 +417,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     // each store instruction writes whole 128-byte rows.
     const int ew = warp - 2;
     const int rq = warp & 3, half = ew >> 2;
+    const int cfirst = G_EPI_SPLIT ? 0 : 32 * half, cstep = G_EPI_SPLIT ? 32 : 64;   // this warp's 32-column slices
+    long long seq = 0;   // tiles of this CTA so far, over all problems (the MMA issuer alternates the buffers the same way)
     uint8_t* stage = epi_smem + (size_t)ew * (32 * G_EPI_PITCH);
     const int srow = lane >> 3, scol = lane & 7;  // this lane's (row mod 4, 16-byte column) when storing
-    int acc_slot = 0;
+    // Staging tile: row r, 16-byte chunk c sits at r*128 + ((c ^ (r & 7)) << 4).  A lane writes its own row
+    // (chunk e at st_lane ^ (e << 4)) and reads chunk scol of rows srow + 4i.
+    const uint32_t st_lane = smem_u32(stage) + (uint32_t)(lane * G_EPI_PITCH + ((lane & 7) << 4));
+    const uint32_t ld_even = smem_u32(stage) + (uint32_t)(srow * G_EPI_PITCH + ((scol ^ srow) << 4));
+    const uint32_t ld_odd = smem_u32(stage) + (uint32_t)((srow + 4) * G_EPI_PITCH + ((scol ^ (srow + 4)) << 4));
+    (void)st_lane; (void)ld_even; (void)ld_odd;
+    int acc_slot = G_EPI_SPLIT ? half : 0;
     uint32_t acc_phase = 0;
     bool live = true;
     long long tr_w0 = 0, tr_w1 = 0, tr_w2 = 0, tr_t0 = clock64();
@@ -425,7 +440,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       const int out_i32 = OUTK == OUT_WORDS ? (int)p.out_type[0] : OUTK == OUT_SIGNS ? 2 : (int)p.out_type[l];
       uint32_t* out32 = reinterpret_cast<uint32_t*>(p.out[l]);  // int32 and fp32 outputs share the layout
       const bool fast = ((K & 3) == 0) && ((Nt & 31) == 0);
-      for (int tile = g_first_tile(L); tile < L.total_tiles; tile += G) {
+      for (int tile = g_first_tile(L); tile < L.total_tiles; tile += G, ++seq) {
+        if (G_EPI_SPLIT && (int)(seq & 1) != half) continue;   // the other group's tile
         const int mg = (int)fdiv((uint32_t)tile, L.dNt), nti = tile - mg * L.n_ntiles;
         const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
         const int n0 = nti * Nt;
@@ -458,13 +474,13 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           // half-word) of the next layer's binary input.  No transposition, one small store per slice.
           const int Kw = (K + 31) >> 5;
           if ((Nt & 31) == 0) {
-            const int per_mt = (Nt - 32 * half + 63) / 64;
+            const int per_mt = (Nt - cfirst + cstep - 1) / cstep;
 #pragma unroll 1
             for (int mt = 0; mt < MT; ++mt) {
               const int pix = row_pixel(mt);
 #pragma unroll 1
               for (int ci = 0; ci < per_mt; ++ci) {
-                const int c0 = 32 * half + 64 * ci, co0 = n0 + c0;
+                const int c0 = cfirst + cstep * ci, co0 = n0 + c0;
                 uint32_t v[32];
                 __syncwarp();  // the load is a warp-wide instruction: no lane may still be in the store below
                 tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * Nt + c0), v);
@@ -489,7 +505,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 #pragma unroll 1
             for (int mt = 0; mt < MT; ++mt) {
               const int pix = row_pixel(mt);
-              for (int c0 = 16 * half; c0 < Nt; c0 += 32) {
+              for (int c0 = G_EPI_SPLIT ? 0 : 16 * half; c0 < Nt; c0 += G_EPI_SPLIT ? 16 : 32) {
                 uint32_t v[16];
                 __syncwarp();
                 tmem_ld16(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * Nt + c0), v);
@@ -514,61 +530,83 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         } else if (OUTK == OUT_SIGNS) {
           // (packed signs only: nothing else is compiled into this variant)
         } else if (fast) {
-          // The warp's slices (sub-tile mt, columns c0..c0+31) form one sequence; the TMEM load of
-          // slice s+1 is issued as soon as slice s sits in the staging tile.
-          const int per_mt = (Nt - 32 * half + 63) / 64;
+          // The warp's slices (sub-tile mt, columns c0..c0+31) form one sequence; the TMEM load of slice s+1 is
+          // issued as soon as slice s sits in the staging tile.  The loop is written for few instructions (this
+          // role is bound by how many it issues): shared-memory addresses are fixed per lane, values travel as
+          // 64-bit pairs from the staging tile through the packed fp32 multiply to the 16-byte store, and a row's
+          // place in the output is one 32-bit element offset per sub-tile.
+          const int per_mt = (Nt - cfirst + cstep - 1) / cstep;
           const int total_sl = MT * per_mt;
           uint32_t v[32];
-          int ro[8];
-          if (total_sl > 0) tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(32 * half), v);
+          uint32_t roff[8];   // element offset of (row srow + 4i, this lane's four channels of a slice's first column), or none
+          if (total_sl > 0) tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)cfirst, v);
           int mt = 0, ci = 0;
 #pragma unroll 1
           for (int sl = 0; sl < total_sl; ++sl) {
-            const int c0 = 32 * half + 64 * ci;
+            const int c0 = cfirst + cstep * ci;
             if (ci == 0) {
               const int mine = row_pixel(mt);
 #pragma unroll
-              for (int i = 0; i < 8; ++i) ro[i] = __shfl_sync(0xffffffffu, mine, srow + 4 * i);
+              for (int i = 0; i < 8; ++i) {
+                const int r = __shfl_sync(0xffffffffu, mine, srow + 4 * i);
+                roff[i] = r >= 0 ? (uint32_t)r * (uint32_t)K + (uint32_t)(n0 + scol * 4) : 0xffffffffu;
+              }
             }
             const int co = n0 + c0 + scol * 4;
-            float4 al = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (!out_i32 && co < K) al = __ldg(reinterpret_cast<const float4*>(alpha + co));
+            unsigned long long alA = 0, alB = 0;   // (alpha[co], alpha[co+1]) and (alpha[co+2], alpha[co+3])
+            if (!out_i32 && co < K) {
+              const float4 al = __ldg(reinterpret_cast<const float4*>(alpha + co));
+              asm("mov.b64 %0, {%1, %2};" : "=l"(alA) : "f"(al.x), "f"(al.y));
+              asm("mov.b64 %0, {%1, %2};" : "=l"(alB) : "f"(al.z), "f"(al.w));
+            }
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 8; ++e)
-              *reinterpret_cast<uint4*>(stage + lane * G_EPI_PITCH + ((e ^ (lane & 7)) << 4)) =
-                  make_uint4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+              asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(st_lane ^ (uint32_t)(e << 4)), "r"(v[4 * e]),
+                           "r"(v[4 * e + 1]), "r"(v[4 * e + 2]), "r"(v[4 * e + 3])
+                           : "memory");
             __syncwarp();
             if (++ci == per_mt) { ci = 0; ++mt; }
             if (sl + 1 < total_sl)
-              tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * Nt + 32 * half + 64 * ci), v);
+              tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * Nt + cfirst + cstep * ci), v);
             if (co < K) {  // K is a multiple of 4 here, so the four channels exist together
-              uint4 u[8];
+              const uint32_t* obase = out32 + c0;
 #pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const int row = srow + 4 * i;
-                u[i] = *reinterpret_cast<const uint4*>(stage + row * G_EPI_PITCH + ((scol ^ (row & 7)) << 4));
-              }
-              if (!out_i32) {
+              for (int hh = 0; hh < 2; ++hh) {   // four rows at a time: 16 registers of values in flight
+                unsigned long long ua[4], ub[4];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                  scale_pair(u[i].x, u[i].y, al.x, al.y);
-                  scale_pair(u[i].z, u[i].w, al.z, al.w);
+                for (int j = 0; j < 4; ++j) {    // row srow + 4i, i = 4hh + j: even i from ld_even, odd i from ld_odd
+                  const int i = 4 * hh + j;
+                  asm volatile("ld.shared.v2.b64 {%0,%1}, [%2];"
+                               : "=l"(ua[j]), "=l"(ub[j])
+                               : "r"(((i & 1) ? ld_odd : ld_even) + (uint32_t)((i >> 1) * 1024))
+                               : "memory");
                 }
-              } else {
-                // int32 sums asked of fp32 accumulators: the sums are integers, the conversion is exact
+                if (!out_i32) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                  u[i].x = (uint32_t)__float2int_rn(__uint_as_float(u[i].x));
-                  u[i].y = (uint32_t)__float2int_rn(__uint_as_float(u[i].y));
-                  u[i].z = (uint32_t)__float2int_rn(__uint_as_float(u[i].z));
-                  u[i].w = (uint32_t)__float2int_rn(__uint_as_float(u[i].w));
+                  for (int j = 0; j < 4; ++j) {
+                    asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(ua[j]) : "l"(alA));
+                    asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(ub[j]) : "l"(alB));
+                  }
+                } else {
+                  // int32 sums asked of fp32 accumulators: the sums are integers, the conversion is exact
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    uint32_t x, y, z, w;
+                    asm("mov.b64 {%0, %1}, %2;" : "=r"(x), "=r"(y) : "l"(ua[j]));
+                    asm("mov.b64 {%0, %1}, %2;" : "=r"(z), "=r"(w) : "l"(ub[j]));
+                    x = (uint32_t)__float2int_rn(__uint_as_float(x)); y = (uint32_t)__float2int_rn(__uint_as_float(y));
+                    z = (uint32_t)__float2int_rn(__uint_as_float(z)); w = (uint32_t)__float2int_rn(__uint_as_float(w));
+                    asm("mov.b64 %0, {%1, %2};" : "=l"(ua[j]) : "r"(x), "r"(y));
+                    asm("mov.b64 %0, {%1, %2};" : "=l"(ub[j]) : "r"(z), "r"(w));
+                  }
                 }
-              }
-              uint32_t* obase32 = out32 + co;
 #pragma unroll
-              for (int i = 0; i < 8; ++i)
-                if (ro[i] >= 0) *reinterpret_cast<uint4*>(obase32 + wide_mul((uint32_t)ro[i], (uint32_t)K)) = u[i];
+                for (int j = 0; j < 4; ++j)
+                  if (roff[4 * hh + j] != 0xffffffffu)
+                    asm volatile("st.global.v2.b64 [%0], {%1,%2};" ::"l"(obase + roff[4 * hh + j]), "l"(ua[j]), "l"(ub[j])
+                                 : "memory");
+              }
             }
             __syncwarp();
           }
@@ -579,7 +617,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           for (int mt = 0; mt < MT; ++mt) {
             const int pix = row_pixel(mt);
             const uint32_t trow = d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * Nt);
-            for (int c0 = 16 * half; c0 < Nt; c0 += 32) {
+            for (int c0 = G_EPI_SPLIT ? 0 : 16 * half; c0 < Nt; c0 += G_EPI_SPLIT ? 16 : 32) {
               uint32_t v[16];
               tmem_ld16(trow + (uint32_t)c0, v);
               tmem_ld_wait();
@@ -606,7 +644,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           __syncwarp();
           if (lane == 0) atomicAdd(L.done + mg, 1u);
         }
-        if (++acc_slot == 2) { acc_slot = 0; acc_phase ^= 1u; }
+        if (G_EPI_SPLIT) acc_phase ^= 1u;
+        else if (++acc_slot == 2) { acc_slot = 0; acc_phase ^= 1u; }
       }
     }
     if (warp == 2 && lane == 0) TR_REPORT(2, clock64() - tr_t0, tr_w0, tr_w1, tr_w2);
@@ -735,42 +774,68 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
                   }
                 }
               } else if (FP4) {
-                // a 32-channel word is one chunk of nibbles; four (or two) words per row as one vector load
+                // A 32-channel word becomes one 16-byte chunk of nibbles.  The common case (an even number of
+                // words per pixel, so that a block's words are read two or four at a time) is kept free of
+                // per-word conditions: this role, too, is bound by the instructions it issues.
                 const int wb = cb * cb_chunks;
-                for (int k0 = 0; k0 < cb_chunks; k0 += 4) {
-                  const int nw = cb_chunks - k0 < 4 ? cb_chunks - k0 : 4;  // 4 or 2
-                  uint32_t bits[G_EXP_ROWS][4];
+                const uint32_t cstride = (uint32_t)Rr * 16u;   // bytes from one chunk of a plane to the next
+                uint32_t da[G_EXP_ROWS];
 #pragma unroll
-                  for (int j = 0; j < G_EXP_ROWS; ++j) {
-                    bits[j][0] = bits[j][1] = bits[j][2] = bits[j][3] = 0;
-                    const int w0 = wb + k0;
-                    if (pix[j] >= 0 && w0 < Cw) {
-                      const uint32_t* src = (const uint32_t*)act + wide_mul((uint32_t)pix[j], (uint32_t)Cw) + w0;
-                      if (vec4) {
-                        const uint4 t = g_ld4(src, fresh);
-                        bits[j][0] = t.x; bits[j][1] = t.y; bits[j][2] = t.z; bits[j][3] = t.w;
-                      } else if (vec) {
-                        const uint2 t = g_ld2(src, fresh);
-                        bits[j][0] = t.x; bits[j][1] = t.y;
-                        if (nw == 4) {
-                          const uint2 t2 = g_ld2(src + 2, fresh);
-                          bits[j][2] = t2.x; bits[j][3] = t2.y;
+                for (int j = 0; j < G_EXP_ROWS; ++j) da[j] = smem_u32(dst[j]);
+                if (vec) {
+                  const uint32_t* src[G_EXP_ROWS];
+#pragma unroll
+                  for (int j = 0; j < G_EXP_ROWS; ++j)
+                    src[j] = (const uint32_t*)act + wide_mul((uint32_t)(pix[j] < 0 ? 0 : pix[j]), (uint32_t)Cw) + wb;
+                  if (vec4) {
+                    for (int k0 = 0; k0 < cb_chunks; k0 += 4) {
+                      uint4 t[G_EXP_ROWS];
+#pragma unroll
+                      for (int j = 0; j < G_EXP_ROWS; ++j) {
+                        t[j] = make_uint4(0, 0, 0, 0);
+                        if (pix[j] >= 0) t[j] = g_ld4(src[j] + k0, fresh);
+                      }
+#pragma unroll
+                      for (int j = 0; j < G_EXP_ROWS; ++j) {
+                        if (pix[j] != -2) {
+                          const bool on = pix[j] >= 0;
+                          const uint32_t d = da[j] + (uint32_t)k0 * cstride;
+                          sts16(d, expand_word_fp4(t[j].x, on));
+                          sts16(d + cstride, expand_word_fp4(t[j].y, on));
+                          sts16(d + 2 * cstride, expand_word_fp4(t[j].z, on));
+                          sts16(d + 3 * cstride, expand_word_fp4(t[j].w, on));
                         }
-                      } else {
+                      }
+                    }
+                  } else {
+                    for (int k0 = 0; k0 < cb_chunks; k0 += 2) {
+                      uint2 t[G_EXP_ROWS];
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                          if (k < nw && w0 + k < Cw) bits[j][k] = g_ld1(src + k, fresh);
+                      for (int j = 0; j < G_EXP_ROWS; ++j) {
+                        t[j] = make_uint2(0, 0);
+                        if (pix[j] >= 0) t[j] = g_ld2(src[j] + k0, fresh);
+                      }
+#pragma unroll
+                      for (int j = 0; j < G_EXP_ROWS; ++j) {
+                        if (pix[j] != -2) {
+                          const bool on = pix[j] >= 0;
+                          const uint32_t d = da[j] + (uint32_t)k0 * cstride;
+                          sts16(d, expand_word_fp4(t[j].x, on));
+                          sts16(d + cstride, expand_word_fp4(t[j].y, on));
+                        }
                       }
                     }
                   }
+                } else {
+                  // an odd number of words per pixel, or a pointer that is not 8-byte aligned: word by word
+                  for (int k = 0; k < cb_chunks; ++k) {
 #pragma unroll
-                  for (int j = 0; j < G_EXP_ROWS; ++j) {
-                    if (pix[j] != -2) {
-#pragma unroll
-                      for (int k = 0; k < 4; ++k)
-                        if (k < nw)
-                          *reinterpret_cast<uint4*>(dst[j] + (size_t)(k0 + k) * Rr * 16) =
-                              expand_word_fp4(bits[j][k], pix[j] >= 0 && wb + k0 + k < Cw);
+                    for (int j = 0; j < G_EXP_ROWS; ++j) {
+                      if (pix[j] == -2) continue;
+                      const bool on = pix[j] >= 0 && wb + k < Cw;
+                      uint32_t w = 0;
+                      if (on) w = g_ld1((const uint32_t*)act + wide_mul((uint32_t)pix[j], (uint32_t)Cw) + wb + k, fresh);
+                      sts16(da[j] + (uint32_t)k * cstride, expand_word_fp4(w, on));
                     }
                   }
                 }
@@ -893,6 +958,7 @@ bool g_plan_layer(const Geom& g, int mode, GLayer* L, int* n_chunks_out, int* Kp
   if (o.Qtot + 1024 + o.halo >= (1ll << 31)) return false;  // positions are 32-bit in the kernel
   if (g.C > (1 << 20)) return false;                        // 9 * c_in stays far below 2^24: exact fp32 sums
   if ((long long)g.N * g.H * g.W >= (1ll << 31) || (long long)g.N * g.Ho * g.Wo >= (1ll << 31)) return false;
+  if ((long long)g.N * g.Ho * g.Wo * g.K >= 0xffffffffLL) return false;   // output element offsets are 32-bit
   // layout tile of the weight operand = channels per tile: all of them up to 256; beyond that 256
   // when that pads little (fewer channel tiles re-expand the same activations), else 128
   if (mode == M_FP4) o.NtL = g.K <= acc_cols ? round_up(g.K, 16) : 128;   // (columns 480..511 hold the scales)
@@ -1087,7 +1153,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
       if (i > 0) {
         host[i].deps = G->deps + deps_off[i];
         host[i].prev_done = G->done + done_off[i - 1];
-        host[i].prev_target = (uint32_t)(G_EW * host[i - 1].n_ntiles);
+        host[i].prev_target = (uint32_t)(G_EW * host[i - 1].n_ntiles);   // (all eight warps drain a chain's tiles)
       }
     }
     e = g_expand_weights(mode, Ls[i]->wplanes, G->weights + w_off[i], gs[i].C, gs[i].K, gs[i].Cw, Kpad[i],
