@@ -180,6 +180,9 @@ def run_reference(args):
 # DRAM traffic per launch of the dominant kernel from an ncu capture (profiles/), valid only while
 # the kernel's sources are the ones that were profiled: {kernel: (workload, batch, bytes, sha256 of sources)}
 _TRAFFIC = {
+    # profiles/dram_traffic_resnet18_stack_n64_grouped.txt: mean of the two captured launches
+    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 343414912,
+                                             "e180723259a6740d323d753ce7d17fb6745c6489d23781077c8629a40400f262"),
 }
 
 
