@@ -161,6 +161,12 @@ SNN_API int64_t snn_kernel_launches(void);
  * all SMs; 8 = the same at N = 128; 7 = tcgen05.mma with fp16 operands (M = 128,
  * N = 256, K = 16); 6 = a write-only stream of 16-byte stores over 1 GiB, in bytes
  * per second (the path writes 29 bytes for every byte it reads).
+ * 9 = self-test of the bounded device-side waits, not a rate: one thread waits, with the
+ * helper every kernel of the library waits with, on a barrier nothing ever arrives on.  The
+ * wait must give up at its attempt limit and raise the status word the host reads, after
+ * which the kernel ends normally: the call returns SNN_ERR_TIMEOUT (the expected outcome)
+ * with *rate = the seconds the kernel took (about a second), and the device stays usable.
+ * Any other return value means the mechanism is broken.
  */
 SNN_API snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate);
 

@@ -645,7 +645,7 @@ snn_status_t snn_conv_stack_destroy(snn_conv_stack_t* st) {
 
 snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate) {
   if (!rate) return fail(SNN_ERR_INVALID_ARG, "null rate pointer");
-  if (kind < 0 || kind > 8) return fail(SNN_ERR_INVALID_ARG, "unknown microbenchmark %d", kind);
+  if (kind < 0 || kind > 9) return fail(SNN_ERR_INVALID_ARG, "unknown microbenchmark %d", kind);
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
     cudaGetLastError();
@@ -655,6 +655,11 @@ snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate) {
   if (!guard.ok) return fail(SNN_ERR_CUDA, "cannot select device %d", device);
   cudaError_t e = microbench(kind, rate);
   g_launches += 2;
+  if (kind == 9) {
+    // self-test of the bounded waits: giving up is the expected outcome
+    if (e == cudaErrorTimeout) return fail(SNN_ERR_TIMEOUT, "self-test: the wait gave up after %.3f s and reported it", *rate);
+    if (e == cudaSuccess) return fail(SNN_ERR_CUDA, "self-test: a wait on a barrier nothing arrives on came back without a report");
+  }
   if (e != cudaSuccess) return cuda_fail(e, "snn_microbench");
   return SNN_OK;
 }

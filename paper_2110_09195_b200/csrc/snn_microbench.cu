@@ -223,8 +223,59 @@ static cudaError_t run_store_stream(double* rate) {
   return cudaGetLastError();
 }
 
+// Self-test of the bounded waits: one thread waits, with the helper every kernel of the library uses, on a
+// barrier nothing ever arrives on.  The wait must give up after its attempt limit and raise the status word
+// in mapped host memory, exactly as a convolution kernel would; the kernel then ends normally and the
+// context stays usable.
+__global__ void wait_selftest_kernel(int* status, long long* cycles) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const long long t0 = clock64();
+    if (!mbar_wait(smem_u32(&bar), 0)) raise_status(status, 7);
+    *cycles = clock64() - t0;
+  }
+}
+
+// cudaErrorTimeout = the wait gave up and said so (the expected outcome); *rate = seconds the kernel took
+cudaError_t run_wait_selftest(double* rate) {
+  int* status_host = nullptr;
+  int* status_dev = nullptr;
+  long long* cycles = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaError_t e = cudaHostAlloc((void**)&status_host, sizeof(int), cudaHostAllocMapped);
+  if (e == cudaSuccess) {
+    *status_host = 0;
+    e = cudaHostGetDevicePointer((void**)&status_dev, status_host, 0);
+  }
+  if (e == cudaSuccess) e = cudaMalloc((void**)&cycles, sizeof(long long));
+  if (e == cudaSuccess) e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  float ms = 0.f;
+  if (e == cudaSuccess) {
+    cudaEventRecord(e0);
+    wait_selftest_kernel<<<1, 32>>>(status_dev, cycles);
+    cudaEventRecord(e1);
+    e = cudaEventSynchronize(e1);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+  }
+  const int code = status_host ? *status_host : 0;
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (cycles) cudaFree(cycles);
+  if (status_host) cudaFreeHost(status_host);
+  if (e != cudaSuccess) return e;
+  *rate = (double)ms * 1e-3;
+  return code == 7 ? cudaErrorTimeout : cudaSuccess;
+}
+
 cudaError_t microbench(int kind, double* rate) {
   switch (kind) {
+    case 9: return run_wait_selftest(rate);
     case 5: return run_mma_rate<true>(240, rate);
     case 6: return run_store_stream(rate);
     case 7: return run_mma_rate<false>(256, rate);

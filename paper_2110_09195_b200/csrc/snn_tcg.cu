@@ -1,31 +1,38 @@
-// Several independent sub-bit convolutions in ONE persistent tensor-core launch.
+// The tensor-core kernel: one or several sub-bit convolutions in ONE persistent launch.
 //
-// Each problem of a group is the forward pass of Sec. 3 / Algorithm 1 for one layer
-// on its own input (decoded +/-1 weights as int8 or fp16 operands, implicit GEMM
-// over a padded, flattened position space, exactly as in the position-major kernel
-// of snn_tc.cu).  The problems do not depend on each other, so one CTA per SM walks
-// through all of them without any grid-wide step in between: while the MMAs of one
-// problem's last tile run, the expander warps already stage the next problem's first
-// activations, the weight producer streams its first stages, and the epilogue warps
-// still drain the tile before.  Start-up, first loads and last drain, which cost a
-// single-layer launch about as much as its MMAs at batch 64, are paid once per group.
+// Each problem of a launch is the forward pass of Sec. 3 / Algorithm 1 for one layer (3x3, or the 1x1
+// extension of the appendix) on its own input: decoded +1/-1 weights as 4-bit e2m1 operands (binary
+// activations) or fp16 operands (fp16 activations), implicit GEMM over a padded, flattened position space
+// in which the nine taps are the same staged activations read from shifted start addresses.  One CTA per
+// SM walks through all problems without any grid-wide step in between: while the MMAs of one problem's
+// last tile run, the expander warps already stage the next problem's first activations, the weight
+// producer streams its first stages, and the epilogue warps still drain the tile before.  Start-up, first
+// loads and last drain, which cost a single-layer launch about as much as its MMAs at batch 64, are paid
+// once per launch.  A single layer is a launch of one problem.
+//
+// Independent problems (a group) need nothing else.  A chain (a stack: problem i + 1 reads the packed signs
+// problem i writes) runs in the same launch on per-tile completion counters: the epilogue bumps the counter
+// of a tile's row block when its part is written, and the expanders of the successor wait (bounded) until the
+// row blocks under a tile's input window are complete.  The launch is cooperative then, so that all CTAs are
+// resident while some of them wait.
 //
 // What makes this possible is a ring geometry that is the same for every problem:
 //   activation units  NA slots of a_slot_bytes   (a problem's unit uses a prefix)
-//   weight stages     NS slots of b_slot_bytes   (a stage = a run of K steps of one
-//                                                 channel block, taps outermost)
-//   accumulators      two buffers of 256 tensor-memory columns
+//   weight stages     NS slots of b_slot_bytes   (a stage = whole taps of one channel block)
+//   accumulators      two buffers of 240 (e2m1) or 256 (fp16) tensor-memory columns
 // so slots, barriers and phases simply carry on from one problem to the next.
 // Tiles of a problem are dealt to the CTAs round-robin; which CTAs get a problem's odd
 // tiles is decided on the host from the time the CTAs have been given so far, so that the
 // CTAs end close together.
 //
 //      warp 0        one thread streams weight stages (cp.async.bulk onto mbarriers)
-//      warp 1        one thread issues tcgen05.mma and commits barriers
-//      warps 2-9     epilogue: TMEM -> registers -> shared-memory transposition ->
-//                    alpha -> 128-byte row stores
-//      warps 10-17   expanders: packed bits -> +1/-1 bytes (or fp16 copied) into the
-//                    activation ring
+//      warp 1        issues tcgen05.mma and commits barriers (warp-uniform, one elected lane)
+//      warps 2-9     epilogue: TMEM -> registers -> shared-memory transposition -> alpha ->
+//                    128-byte row stores; or TMEM -> registers -> threshold -> packed sign words
+//      warps 10-19   expanders (13 and 17 idle): packed bits -> e2m1 nibbles (or fp16 copied)
+//                    into the activation ring
+// The kernel is compiled per operand mode and per output kind (words, packed signs, chain), so that
+// no variant carries another one's code in its loops.
 // Every wait is bounded; one that runs out raises a status word the host reads, and
 // the CTA still frees its tensor memory and returns.
 #include <algorithm>
