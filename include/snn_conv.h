@@ -184,7 +184,8 @@ SNN_API snn_status_t snn_microbench(int32_t kind, int32_t device, double* rate);
  * activation type on one device; N[i], H[i], W[i] fix the input shape of member i.
  * The group keeps the handles' device data by reference: the handles must outlive
  * the group.  It builds its own tiled weight operands (device memory owned by the
- * group).  Errors: INVALID_ARG (null, count out of range, mixed activation types
+ * group), one set per output kind (words, packed signs): the tile shapes the kernel
+ * is planned with differ between the two.  Errors: INVALID_ARG (null, count out of range, mixed activation types
  * or devices, a shape giving no output), UNSUPPORTED (a member the tensor-core
  * path cannot run; nothing is kept), CUDA, OOM.
  *

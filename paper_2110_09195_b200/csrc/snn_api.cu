@@ -57,7 +57,8 @@ struct snn_conv {
   LayerDev L;
   std::mutex mu;
   std::map<std::tuple<int, int, int>, int> tuned;        // (N,H,W) -> path measured fastest by snn_conv_tune
-  std::map<std::tuple<int, int, int>, GroupDev*> solo;   // (N,H,W) -> tensor-core plan and weight operand (a group of one)
+  // (N,H,W, packed-sign output?) -> tensor-core plan and weight operand (a group of one)
+  std::map<std::tuple<int, int, int, int>, GroupDev*> solo;
   // staging for snn_conv_forward_host
   void* stage_in = nullptr;
   void* stage_out = nullptr;
@@ -122,14 +123,15 @@ int auto_path(snn_conv* h, const Geom& g) {
 
 // The tensor-core kernel's plan and weight operand for this input shape: built (and allocated) at the first
 // call for the shape, reused afterwards.
-cudaError_t solo_group(snn_conv* h, const Geom& g, GroupDev** out, int* launched) {
+cudaError_t solo_group(snn_conv* h, const Geom& g, int out_type, GroupDev** out, int* launched) {
   std::lock_guard<std::mutex> lk(h->mu);
-  const auto key = std::make_tuple(g.N, g.H, g.W);
+  const int kind = out_type == SNN_OUT_BITS ? TCG_SIGNS : TCG_WORDS;
+  const auto key = std::make_tuple(g.N, g.H, g.W, kind);
   auto it = h->solo.find(key);
   if (it != h->solo.end()) { *out = it->second; return cudaSuccess; }
   const LayerDev* Lp = &h->L;
   GroupDev* G = nullptr;
-  cudaError_t e = tcg_create(&Lp, &g, 1, h->act_type, 0, h->host_stream, &G, launched);
+  cudaError_t e = tcg_create(&Lp, &g, 1, h->act_type, kind, h->host_stream, &G, launched);
   if (e != cudaSuccess) return e;
   h->solo[key] = G;
   *out = G;
@@ -144,7 +146,7 @@ snn_status_t run_path(snn_conv* h, int path, const Geom& g, const Launch& l) {
     case SNN_PATH_DECODED: e = popc_forward(h->L, g, l, &launched); break;
     case SNN_PATH_DECODED_TC: {
       GroupDev* G = nullptr;
-      e = solo_group(h, g, &G, &launched);
+      e = solo_group(h, g, l.out_i32, &G, &launched);
       if (e == cudaSuccess) e = tcg_forward(G, &l.act, &l.out, l.out_i32, l.stream, h->tc_status_dev, &launched);
       break;
     }
@@ -466,7 +468,8 @@ snn_status_t snn_conv_tune(snn_conv_t* h, int32_t N, int32_t H, int32_t W, int32
 
 struct snn_conv_group {
   int device = 0, count = 0, act_type = 0;
-  GroupDev* G = nullptr;
+  GroupDev* G = nullptr;        // planned for fp32 / int32 outputs
+  GroupDev* G_signs = nullptr;  // planned for packed-sign outputs (binary activations only)
   int* status_host = nullptr;  // pinned, written by the kernel on a bounded-wait timeout
   int* status_dev = nullptr;
 };
@@ -501,9 +504,13 @@ snn_status_t snn_conv_group_create(snn_conv_t* const* layers, int32_t count, con
     e = cudaHostGetDevicePointer((void**)&g->status_dev, g->status_host, 0);
   }
   int launched = 0;
-  if (e == cudaSuccess) e = tcg_create(Ls, gs, count, g->act_type, 0, layers[0]->host_stream, &g->G, &launched);
+  if (e == cudaSuccess) e = tcg_create(Ls, gs, count, g->act_type, TCG_WORDS, layers[0]->host_stream, &g->G, &launched);
+  if (e == cudaSuccess && g->act_type == SNN_ACT_BIN)
+    e = tcg_create(Ls, gs, count, g->act_type, TCG_SIGNS, layers[0]->host_stream, &g->G_signs, &launched);
   g_launches += launched;
   if (e != cudaSuccess) {
+    tcg_destroy(g->G);
+    tcg_destroy(g->G_signs);
     if (g->status_host) cudaFreeHost(g->status_host);
     delete g;
     if (e == cudaErrorInvalidConfiguration) {
@@ -537,8 +544,8 @@ snn_status_t snn_conv_group_forward(snn_conv_group_t* g, const void* const* act_
     return fail(SNN_ERR_TIMEOUT, "an earlier launch of the group gave up a bounded wait (code %d)", code);
   }
   int launched = 0;
-  cudaError_t e = tcg_forward(g->G, act_dev, out_dev, out_type, (cudaStream_t)cuda_stream, g->status_dev,
-                              &launched);
+  cudaError_t e = tcg_forward(out_type == SNN_OUT_BITS ? g->G_signs : g->G, act_dev, out_dev, out_type,
+                              (cudaStream_t)cuda_stream, g->status_dev, &launched);
   g_launches += launched;
   if (e != cudaSuccess) return cuda_fail(e, "snn_conv_group_forward");
   return SNN_OK;
@@ -548,6 +555,7 @@ snn_status_t snn_conv_group_destroy(snn_conv_group_t* g) {
   if (!g) return SNN_OK;
   DeviceGuard guard(g->device);
   tcg_destroy(g->G);
+  tcg_destroy(g->G_signs);
   if (g->status_host) cudaFreeHost(g->status_host);
   delete g;
   return SNN_OK;
@@ -598,7 +606,7 @@ snn_status_t snn_conv_stack_create(snn_conv_t* const* layers, int32_t count, int
     e = cudaHostGetDevicePointer((void**)&st->status_dev, st->status_host, 0);
   }
   int launched = 0;
-  if (e == cudaSuccess) e = tcg_create(Ls, gs, count, SNN_ACT_BIN, 1, layers[0]->host_stream, &st->G, &launched);
+  if (e == cudaSuccess) e = tcg_create(Ls, gs, count, SNN_ACT_BIN, TCG_CHAIN, layers[0]->host_stream, &st->G, &launched);
   g_launches += launched;
   if (e != cudaSuccess) {
     if (st->status_host) cudaFreeHost(st->status_host);

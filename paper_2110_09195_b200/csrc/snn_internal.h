@@ -52,10 +52,15 @@ cudaError_t reuse_forward(const LayerDev& L, const Geom& g, int act_type, const 
 // layers as ONE persistent launch; a single layer is a group of one.
 // Several independent problems in one persistent tensor-core launch (snn_tcg.cu).
 struct GroupDev;
-// chain = 1: member i + 1 reads the packed signs member i writes (binary activations; the members' shapes must
-// follow from one another); tcg_forward then takes the first member's input in act[0] and the last member's
-// output in out[0], and out_type is the last member's.
-cudaError_t tcg_create(const LayerDev* const* layers, const Geom* geoms, int count, int act_type, int chain,
+// What a launch is planned for: the tile shapes and the number of accumulator buffers differ between the kinds.
+//   TCG_WORDS  independent problems, fp32 / int32 outputs
+//   TCG_CHAIN  member i + 1 reads the packed signs member i writes (binary activations; the members' shapes must
+//              follow from one another); tcg_forward then takes the first member's input in act[0] and the last
+//              member's output in out[0], and out_type is the last member's
+//   TCG_SIGNS  independent problems, packed-sign outputs (binary activations)
+// tcg_forward refuses an output type the plan was not made for.
+enum { TCG_WORDS = 0, TCG_CHAIN = 1, TCG_SIGNS = 2 };
+cudaError_t tcg_create(const LayerDev* const* layers, const Geom* geoms, int count, int act_type, int kind,
                        cudaStream_t s, GroupDev** out, int* launched);
 cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, int out_type, cudaStream_t s,
                         int* status_dev, int* launched);

@@ -19,7 +19,7 @@
 // What makes this possible is a ring geometry that is the same for every problem:
 //   activation units  NA slots of a_slot_bytes   (a problem's unit uses a prefix)
 //   weight stages     NS slots of b_slot_bytes   (a stage = whole taps of one channel block)
-//   accumulators      two buffers of 240 (e2m1) or 256 (fp16) tensor-memory columns
+//   accumulators      three buffers of 160 (e2m1) or two of 256 (fp16) tensor-memory columns
 // so slots, barriers and phases simply carry on from one problem to the next.
 // Tiles of a problem are dealt to the CTAs round-robin; which CTAs get a problem's odd
 // tiles is decided on the host from the time the CTAs have been given so far, so that the
@@ -61,7 +61,12 @@ constexpr int G_EPI_PITCH = 128;
 constexpr int G_EPI_BYTES = G_EW * 32 * G_EPI_PITCH;
 constexpr int G_NS_MAX = 8;
 constexpr uint32_t G_ACC_COLS = 256;          // tensor-memory columns of one accumulator buffer
-constexpr uint32_t G_ACC_COLS_FP4 = 240;      // 4-bit mode: columns 480..511 hold the (unit) block scales
+constexpr uint32_t G_ACC_COLS_FP4 = 240;      // 4-bit mode, two buffers: columns 480..511 hold the (unit) block scales
+constexpr uint32_t G_ACC_COLS_FP4_3 = 160;    // 4-bit mode, three buffers
+// Accumulator buffers.  Word outputs on 4-bit operands use three: the MMAs of the tile after next run while both
+// epilogue groups still drain, so a group never waits for them (the epilogue is what bounds that variant).  The
+// other variants are bound elsewhere and do better with two larger buffers (larger tiles).
+constexpr int G_NACC = 2, G_NACC_WORDS = 3;
 constexpr uint32_t G_SCALE_COL = 480;
 constexpr size_t kGTail = 512;
 constexpr size_t kGSmemBudget = 226 * 1024;
@@ -102,6 +107,7 @@ struct GParams {
   int* status;
   uint8_t out_type[SNN_GROUP_MAX];   // per member: 0 fp32 alpha*S, 1 int32 S, 2 packed signs of alpha*S + shift
   uint32_t acc_cols;      // tensor-memory columns of one accumulator buffer
+  int n_acc;              // accumulator buffers (tile seq of a CTA uses buffer seq % n_acc)
   int NA, NS;
   uint32_t a_slot_bytes, b_slot_bytes;
   uint32_t off_b, off_epi, off_pix, off_lay, off_tail;
@@ -217,18 +223,22 @@ __device__ __forceinline__ bool g_issue_block(uint64_t a_unit, uint32_t wq, uint
 // OUTK: what the epilogue is compiled for.  0: fp32 or int32 words for every member; 1: packed signs for every
 // member; 2: a chain - packed signs between the members, any type for the last, and the dependency waits and
 // completion counters.  Keeping the variants apart keeps each one's registers and code to what it needs.
-enum { OUT_WORDS = 0, OUT_SIGNS = 1, OUT_CHAIN = 2 };
+// 3: words again, with the expanders' two-stage load pipeline instead of their plain loop (4-bit operands whose rows
+// can be read two words at a time); a separate instantiation so that neither carries the other's code.
+enum { OUT_WORDS = 0, OUT_SIGNS = 1, OUT_CHAIN = 2, OUT_WORDS_PIPED = 3 };
 
 template <int MODE, int OUTK>
 __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p) {
   constexpr bool F16 = MODE == M_F16;   // fp16 activations (copied, not expanded)
   constexpr bool FP4 = MODE == M_FP4;   // binary activations as e2m1 nibbles
   constexpr bool CHAIN = OUTK == OUT_CHAIN;
+  constexpr bool WORDS = OUTK == OUT_WORDS || OUTK == OUT_WORDS_PIPED;
+  constexpr bool PIPED = OUTK == OUT_WORDS_PIPED;
   // Word outputs (fp32 / int32) are bound by the stores: there the epilogue warps form two groups of four (one
   // warp per quarter of the accumulator's lanes) that take the tiles in turn, group g draining accumulator
   // buffer g, so that one group's stores drain while the other reads tensor memory and transposes.  Packed
   // signs are bound by the epilogue's instructions: all eight warps drain every tile together.
-  constexpr bool G_EPI_SPLIT = OUTK == OUT_WORDS;
+  constexpr bool G_EPI_SPLIT = WORDS;
   constexpr int G_EPI_ARRIVALS = G_EPI_SPLIT ? G_EW / 2 : G_EW;   // epilogue warps that drain one tile
   extern __shared__ __align__(128) uint8_t smem[];
   // carve-up: [NA activation slots][NS weight slots][epilogue tiles][pixel table][problem table][barriers, flags]
@@ -241,21 +251,26 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
   // epilogue's registers are all taken by the slices it transposes.
   const GLayer* lay = reinterpret_cast<const GLayer*>(smem + p.off_lay);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + p.off_tail);
-  // barriers: b_full[8] b_empty[8] a_full[4] a_empty[4] acc_full[2] acc_empty[2]
+  // barriers: b_full[8] b_empty[8] a_full[4] a_empty[4] acc_full[4] acc_empty[3]
+  // acc_full is indexed by the tile's sequence number in the CTA (seq % 4), not by the buffer: an epilogue group
+  // that takes every other tile then sees every phase of the barriers it waits on (seq % 4 = g and g + 2), and a
+  // barrier's next phase cannot complete before its last one was consumed (tile seq + 3 needs the buffer tile seq
+  // releases).  acc_empty is per buffer.
   const uint32_t bar_bfull = smem_u32(bars), bar_bempty = smem_u32(bars + 8);
   const uint32_t bar_afull = smem_u32(bars + 16), bar_aempty = smem_u32(bars + 20);
-  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 26);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 28);
+  const uint32_t bar_accfull = smem_u32(bars + 24), bar_accempty = smem_u32(bars + 28);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 31);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int NS = p.NS, NA = p.NA;
   const int G = (int)gridDim.x;
 
-  if (tid < 28) {
+  if (tid < 31) {
     uint32_t count = 1;
-    if (tid >= 26) count = G_EPI_ARRIVALS;             // acc_empty: one arrival per epilogue warp of the tile
-    if (tid >= 16 && tid < 20) count = G_EXP_THREADS;  // a_full: every expander thread arrives
+    if (tid >= 28) count = G_EPI_ARRIVALS;             // acc_empty: one arrival per epilogue warp of the tile
+    if (tid >= 16 && tid < 20)   // a_full: every expander thread arrives, or one lane per expander warp (pipelined form)
+      count = PIPED ? G_EXP_THREADS / 32 : G_EXP_THREADS;
     mbar_init(smem_u32(bars + tid), count);
   }
   if (tid == 32) *abort_flag = 0;
@@ -354,8 +369,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     {
       const bool leader = elect_one();
       bool ok = true;
-      int a_slot = 0, b_slot = 0, acc_slot = 0;
+      int a_slot = 0, b_slot = 0, acc_slot = 0, full_slot = 0;
       uint32_t a_phase = 0, b_phase = 0, acc_phase = 1;
+      const int n_acc = p.n_acc;
       long long tiles_done = 0;
       long long tr_w0 = 0, tr_w1 = 0, tr_w2 = 0, tr_t0 = clock64();
       (void)tr_w0; (void)tr_w1; (void)tr_w2; (void)tr_t0;
@@ -373,7 +389,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         const uint64_t b_desc0 = make_desc(smem_u32(b_smem), (uint32_t)Nt * 16, 128);
         const uint32_t a_step = 2u * (uint32_t)Rr, b_step = 2u * (uint32_t)Nt;  // two chunks per MMA
         for (int tile = g_first_tile(L); tile < total && ok; tile += G, ++tiles_done) {
-          if (tiles_done >= 2) {
+          if (tiles_done >= n_acc) {
             if (!TR_WAIT(tr_w0, mbar_wait(bar_accempty + 8 * acc_slot, acc_phase))) { ok = false; break; }
             tc_fence_after();
           }
@@ -405,8 +421,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
             if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
           }
           if (!ok) break;
-          if (leader) tc_commit(bar_accfull + 8 * acc_slot);  // fires when this tile's MMAs are complete
-          if (++acc_slot == 2) { acc_slot = 0; acc_phase ^= 1u; }
+          if (leader) tc_commit(bar_accfull + 8 * full_slot);  // fires when this tile's MMAs are complete
+          full_slot = (full_slot + 1) & 3;
+          if (++acc_slot == n_acc) { acc_slot = 0; acc_phase ^= 1u; }
         }
       }
       if (!ok && leader && !*abort_flag) {
@@ -434,8 +451,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     const uint32_t ld_even = smem_u32(stage) + (uint32_t)(srow * G_EPI_PITCH + ((scol ^ srow) << 4));
     const uint32_t ld_odd = smem_u32(stage) + (uint32_t)((srow + 4) * G_EPI_PITCH + ((scol ^ (srow + 4)) << 4));
     (void)st_lane; (void)ld_even; (void)ld_odd;
-    int acc_slot = G_EPI_SPLIT ? half : 0;
-    uint32_t acc_phase = 0;
+    int acc_slot = 0;   // buffer of tile seq: seq % n_acc, kept in step with seq
+    const int n_acc = p.n_acc;
     bool live = true;
     long long tr_w0 = 0, tr_w1 = 0, tr_w2 = 0, tr_t0 = clock64();
     (void)tr_w0; (void)tr_w1; (void)tr_w2; (void)tr_t0;
@@ -444,16 +461,17 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       const int Nt = L.Nt, MT = L.MT, K = L.K;
       const float* alpha = L.alpha;
       const float* shift = L.shift;
-      const int out_i32 = OUTK == OUT_WORDS ? (int)p.out_type[0] : OUTK == OUT_SIGNS ? 2 : (int)p.out_type[l];
+      const int out_i32 = WORDS ? (int)p.out_type[0] : OUTK == OUT_SIGNS ? 2 : (int)p.out_type[l];
       uint32_t* out32 = reinterpret_cast<uint32_t*>(p.out[l]);  // int32 and fp32 outputs share the layout
       const bool fast = ((K & 3) == 0) && ((Nt & 31) == 0);
-      for (int tile = g_first_tile(L); tile < L.total_tiles; tile += G, ++seq) {
+      for (int tile = g_first_tile(L); tile < L.total_tiles; tile += G, ++seq, acc_slot = acc_slot + 1 == n_acc ? 0 : acc_slot + 1) {
         if (G_EPI_SPLIT && (int)(seq & 1) != half) continue;   // the other group's tile
+        const uint32_t full_bar = bar_accfull + 8u * (uint32_t)(seq & 3), full_phase = (uint32_t)((seq >> 2) & 1);
         const int mg = (int)fdiv((uint32_t)tile, L.dNt), nti = tile - mg * L.n_ntiles;
         const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * MT);
         const int n0 = nti * Nt;
         int okw = 1;
-        if (lane == 0) okw = (!*abort_flag && TR_WAIT(tr_w0, mbar_wait_backoff(bar_accfull + 8 * acc_slot, acc_phase, 100))) ? 1 : 0;
+        if (lane == 0) okw = (!*abort_flag && TR_WAIT(tr_w0, mbar_wait_backoff(full_bar, full_phase, 100))) ? 1 : 0;
         okw = __shfl_sync(0xffffffffu, okw, 0);
         if (!okw) {
           if (lane == 0 && !*abort_flag) {
@@ -475,7 +493,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           const bool valid = ((long long)q < L.Qtot) && ((int)n < L.N) && (y < L.Ho) && (x < L.Wo);
           return valid ? ((int)n * L.Ho + y) * L.Wo + x : -1;
         };
-        if (OUTK != OUT_WORDS && out_i32 == 2) {
+        if (!WORDS && out_i32 == 2) {
           // Packed signs of the scaled output (Algorithm 1: the next layer consumes sign(a)): a thread
           // owns one position and the 32 (or 16) consecutive channels of a slice, i.e. one word (or
           // half-word) of the next layer's binary input.  No transposition, one small store per slice.
@@ -651,8 +669,6 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           __syncwarp();
           if (lane == 0) atomicAdd(L.done + mg, 1u);
         }
-        if (G_EPI_SPLIT) acc_phase ^= 1u;
-        else if (++acc_slot == 2) { acc_slot = 0; acc_phase ^= 1u; }
       }
     }
     if (warp == 2 && lane == 0) TR_REPORT(2, clock64() - tr_t0, tr_w0, tr_w1, tr_w2);
@@ -669,8 +685,153 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     volatile int* dep_flag = abort_flag + 2;
     bool stop = false;
     long long tr_w0 = 0, tr_t0 = clock64();
-    (void)tr_w0; (void)tr_t0;
-    for (int l = 0; l < p.n_layers && !stop; ++l) {
+    (void)tr_w0; (void)tr_t0; (void)exp_flag; (void)dep_flag;
+    if (!CHAIN) {
+      // Independent problems: all inputs exist when the launch starts and are small beside the L2 (1/29 of the
+      // outputs).  The CTAs pull them into L2 together, once, so that the staging loads below see L2 latency
+      // instead of DRAM latency: a unit is one round trip, and the round trip is what the expanders' rate is.
+      for (int l = 0; l < p.n_layers; ++l) {
+        const GLayer& L = lay[l];
+        const size_t bytes = (size_t)L.N * L.H * L.W * (F16 ? (size_t)L.C * 2 : (size_t)L.Cw * 4);
+        const char* base = reinterpret_cast<const char*>(p.act[l]);
+        for (size_t off = ((size_t)blockIdx.x * G_EXP_THREADS + et) * 128; off < bytes; off += (size_t)G * G_EXP_THREADS * 128)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
+      }
+    }
+    // Independent problems on 4-bit operands whose rows can be read two words at a time run a two-stage software
+    // pipeline per thread: a "group" is up to three rows of one unit with one vector load each; the loads of
+    // group g + 1 are issued (into registers) before group g is expanded into shared memory, so that a unit no
+    // longer costs a full round trip to memory - with few words per row the round trip is nearly all of it.
+    constexpr bool piped = PIPED;   // (the host has checked the alignment of all inputs)
+    if constexpr (PIPED) {
+      struct XGroup {
+        uint4 t[G_EXP_ROWS];        // the rows' words (two or four of them)
+        uint32_t da[G_EXP_ROWS];    // where a row's first chunk goes
+        uint32_t cstride;           // bytes from one chunk of a plane to the next
+        uint32_t flags;             // bit j: row j exists; bit 4 + j: its pixel is inside the image; 8: four words per
+                                    // row; 9: first group of its unit; 10: last group of its unit
+      };
+      // issue side: the next group to load
+      int il = 0, itile = 0, itotal = 0, icb = 0, irb = 0, ik0 = 0, i_slot = 0;
+      int Rr = 0, n_planes = 0, n_cb = 0, cbc = 0, Cw = 0, all_rows = 0, kstep = 2;
+      const uint32_t* act = nullptr;
+      bool ivalid = false;
+      auto enter_layer = [&]() {   // first layer from il on in which this CTA has a tile
+        for (; il < p.n_layers; ++il) {
+          const GLayer& L = lay[il];
+          itile = g_first_tile(L);
+          itotal = L.total_tiles;
+          if (itile >= itotal) continue;
+          Rr = L.Rr; n_planes = L.n_planes; n_cb = L.n_cb; cbc = L.cb_chunks; Cw = L.Cw;
+          all_rows = n_planes * Rr;
+          act = reinterpret_cast<const uint32_t*>(p.act[il]);
+          kstep = ((reinterpret_cast<uintptr_t>(act) & 15) == 0 && (Cw & 3) == 0 && (cbc & 3) == 0) ? 4 : 2;
+          icb = irb = ik0 = 0;
+          ivalid = true;
+          return;
+        }
+        ivalid = false;
+      };
+      auto enter_tile = [&]() {    // input pixel of each of this thread's rows of the tile
+        const GLayer& L = lay[il];
+        const int mg = (int)fdiv((uint32_t)itile, L.dNt);
+        const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * L.MT);
+        for (int f = et; f < all_rows; f += G_EXP_THREADS) {
+          const int pl = (f >= Rr) + (f >= 2 * Rr) + (f >= 3 * Rr);
+          pix_tab[f] = g_position_to_pixel(L, Q0 + (uint32_t)(f - pl * Rr), pl >> 1, pl & 1);
+        }
+      };
+      auto issue = [&](XGroup& g) {   // loads of the group at the issue position; moves the position on
+        const uint32_t cs = (uint32_t)Rr * 16u;
+        uint32_t flags = (kstep == 4 ? 0x100u : 0u) | ((irb == 0 && ik0 == 0) ? 0x200u : 0u);
+        const uint32_t unit = smem_u32(a_smem) + (uint32_t)i_slot * p.a_slot_bytes;
+#pragma unroll
+        for (int j = 0; j < G_EXP_ROWS; ++j) {
+          const int f = irb + et + j * G_EXP_THREADS;
+          const int pix = f < all_rows ? pix_tab[f] : -2;
+          const int pl = (f >= Rr) + (f >= 2 * Rr) + (f >= 3 * Rr);
+          g.da[j] = unit + (uint32_t)(pl * cbc * Rr + (f - pl * Rr)) * 16u + (uint32_t)ik0 * cs;
+          if (pix != -2) flags |= 1u << j;
+          g.t[j] = make_uint4(0, 0, 0, 0);
+          if (pix >= 0) {
+            flags |= 0x10u << j;
+            const uint32_t* src = act + wide_mul((uint32_t)pix, (uint32_t)Cw) + icb * cbc + ik0;
+            if (kstep == 4) {
+              g.t[j] = __ldg(reinterpret_cast<const uint4*>(src));
+            } else {
+              const uint2 v = __ldg(reinterpret_cast<const uint2*>(src));
+              g.t[j].x = v.x;
+              g.t[j].y = v.y;
+            }
+          }
+        }
+        g.cstride = cs;
+        ik0 += kstep;
+        if (ik0 >= cbc) {
+          ik0 = 0;
+          irb += G_EXP_ROWS * G_EXP_THREADS;
+          if (irb >= all_rows) {   // the unit ends with this group
+            irb = 0;
+            flags |= 0x400u;
+            i_slot = i_slot + 1 == NA ? 0 : i_slot + 1;
+            if (++icb >= n_cb) {
+              icb = 0;
+              itile += G;
+              if (itile >= itotal) {
+                ++il;
+                enter_layer();
+              }
+              if (ivalid) enter_tile();
+            }
+          }
+        }
+        g.flags = flags;
+      };
+      enter_layer();
+      if (ivalid) enter_tile();
+      XGroup cur, nxt;
+      bool nvalid = ivalid;
+      if (nvalid) issue(nxt);
+      while (nvalid && !stop) {
+        cur = nxt;
+        nvalid = ivalid;
+        if (nvalid) issue(nxt);
+        if ((cur.flags & 0x200u) && a_done >= NA) {
+          int okf = 1;
+          if (lane == 0) okf = (!*abort_flag && TR_WAIT(tr_w0, mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 64))) ? 1 : 0;
+          okf = __shfl_sync(0xffffffffu, okf, 0);
+          if (!okf) {
+            if (lane == 0 && !*abort_flag) {
+              *abort_flag = 1;
+              raise_status(p.status, 1);
+            }
+            stop = true;
+            break;
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < G_EXP_ROWS; ++j) {
+          if (cur.flags & (1u << j)) {
+            const bool on = (cur.flags & (0x10u << j)) != 0;
+            const uint32_t d = cur.da[j], cs = cur.cstride;
+            sts16(d, expand_word_fp4(cur.t[j].x, on));
+            sts16(d + cs, expand_word_fp4(cur.t[j].y, on));
+            if (cur.flags & 0x100u) {
+              sts16(d + 2 * cs, expand_word_fp4(cur.t[j].z, on));
+              sts16(d + 3 * cs, expand_word_fp4(cur.t[j].w, on));
+            }
+          }
+        }
+        if (cur.flags & 0x400u) {
+          fence_proxy_async();  // generic-proxy writes -> visible to the tensor core's reads
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_afull + 8 * a_slot);
+          ++a_done;
+          if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
+        }
+      }
+    }
+    for (int l = 0; l < (piped ? 0 : p.n_layers) && !stop; ++l) {
       const GLayer& L = lay[l];
       const int Rr = L.Rr, n_planes = L.n_planes, n_cb = L.n_cb, cb_chunks = L.cb_chunks, MT = L.MT;
       const int C = L.C, Cw = L.Cw, total = L.total_tiles;
@@ -870,6 +1031,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 // ------------------------------------------------------------------ host side
 struct GroupDev {
   int count = 0, act_type = 0, mode = M_FP4;
+  int kind = TCG_WORDS;           // what the tiles were planned for (word outputs, packed signs, chain)
+  bool words_even = false;        // every member has an even number of activation words per pixel
   int chain = 0;                  // 1: member i + 1 reads the packed signs member i writes (one launch, dependency counters)
   uint8_t* chain_buf = nullptr;   // the packed signs between the members, one buffer per boundary
   size_t chain_off[SNN_GROUP_MAX] = {};
@@ -942,9 +1105,14 @@ inline int g_mode_for(int act_type) { return act_type == SNN_ACT_F16 ? M_F16 : M
 // channel plus a constant that does not overlap the previous MMA.
 inline double g_mma_cycles(int nt) { return 0.5 * nt + 33.0; }
 
-bool g_plan_layer(const Geom& g, int mode, GLayer* L, int* n_chunks_out, int* Kpad_out) {
+inline int g_n_acc(int mode, int kind) { return (mode == M_FP4 && kind == TCG_WORDS) ? G_NACC_WORDS : G_NACC; }
+inline int g_acc_cols(int mode, int kind) {
+  return mode != M_FP4 ? (int)G_ACC_COLS : kind == TCG_WORDS ? (int)G_ACC_COLS_FP4_3 : (int)G_ACC_COLS_FP4;
+}
+
+bool g_plan_layer(const Geom& g, int mode, int kind, GLayer* L, int* n_chunks_out, int* Kpad_out) {
   const int cpc = mode == M_F16 ? 8 : 32;
-  const int acc_cols = mode == M_FP4 ? (int)G_ACC_COLS_FP4 : (int)G_ACC_COLS;
+  const int acc_cols = g_acc_cols(mode, kind);
   const int raw = round_up(g.C, 2 * cpc) / cpc;  // 16-byte chunks along the channels, even
   GLayer& o = *L;
   o.N = g.N; o.H = g.H; o.W = g.W; o.C = g.C; o.K = g.K; o.Cw = g.Cw;
@@ -1022,11 +1190,12 @@ int h_position_to_pixel(const GLayer& L, long long q, int pa, int pb) {
 }
 }  // namespace
 
-cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int act_type, int chain, cudaStream_t s,
+cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int act_type, int kind, cudaStream_t s,
                        GroupDev** out, int* launched) {
   *out = nullptr;
   if (count < 1 || count > SNN_GROUP_MAX) return cudaErrorInvalidConfiguration;
-  if (chain && act_type != SNN_ACT_BIN) return cudaErrorInvalidConfiguration;
+  if (kind != TCG_WORDS && act_type != SNN_ACT_BIN) return cudaErrorInvalidConfiguration;
+  const int chain = kind == TCG_CHAIN;
   const int mode = g_mode_for(act_type);
   GLayer host[SNN_GROUP_MAX];
   int n_chunks[SNN_GROUP_MAX], Kpad[SNN_GROUP_MAX];
@@ -1034,7 +1203,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   size_t a_slot = 0, pix_bytes = 0;
   long long tiles = 0;
   for (int i = 0; i < count; ++i) {
-    if (!g_plan_layer(gs[i], mode, &host[i], &n_chunks[i], &Kpad[i])) return cudaErrorInvalidConfiguration;
+    if (!g_plan_layer(gs[i], mode, kind, &host[i], &n_chunks[i], &Kpad[i])) return cudaErrorInvalidConfiguration;
     const size_t unit = (size_t)host[i].n_planes * host[i].cb_chunks * host[i].Rr * 16;
     if (unit > a_slot) a_slot = unit;
     const size_t pb = (size_t)host[i].n_planes * host[i].Rr * 4;
@@ -1135,6 +1304,10 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   G->mode = mode;
   G->grid = grid;
   G->chain = chain;
+  G->kind = kind;
+  G->words_even = true;
+  for (int i = 0; i < count; ++i)
+    if (gs[i].Cw & 1) G->words_even = false;
   cudaError_t e = cudaMalloc(&G->weights, w_total);
   if (chain) {
     G->done_words = done_words;
@@ -1178,7 +1351,8 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   p.n_layers = count;
   p.NA = na;
   p.NS = ns;
-  p.acc_cols = mode == M_FP4 ? G_ACC_COLS_FP4 : G_ACC_COLS;
+  p.acc_cols = (uint32_t)g_acc_cols(mode, kind);
+  p.n_acc = g_n_acc(mode, kind);
   p.a_slot_bytes = (uint32_t)a_slot;
   p.b_slot_bytes = kGBSlot;
   p.off_b = (uint32_t)((size_t)na * a_slot);
@@ -1209,14 +1383,19 @@ void tcg_destroy(GroupDev* G) {
 int tcg_count(const GroupDev* G) { return G->count; }
 
 bool tcg_supported(const Geom& g, int act_type) {
-  GLayer L;
-  int n_chunks = 0, Kpad = 0;
-  if (!g_plan_layer(g, g_mode_for(act_type), &L, &n_chunks, &Kpad)) return false;
-  // one problem alone: three activation slots, the fixed parts and three weight slots must fit
-  const size_t unit = (((size_t)L.n_planes * L.cb_chunks * L.Rr * 16) + 127) & ~(size_t)127;
-  const size_t pix = (((size_t)L.n_planes * L.Rr * 4) + 127) & ~(size_t)127;
-  const size_t fixed = (size_t)G_EPI_BYTES + pix + 256 + kGTail;
-  return 2 * unit + fixed + 3 * (size_t)kGBSlot <= kGSmemBudget;
+  // one problem alone, under every plan a launch may use: two activation slots, the fixed parts and three
+  // weight slots must fit
+  for (int kind = TCG_WORDS; kind <= TCG_SIGNS; ++kind) {
+    if (kind != TCG_WORDS && act_type != SNN_ACT_BIN) continue;
+    GLayer L;
+    int n_chunks = 0, Kpad = 0;
+    if (!g_plan_layer(g, g_mode_for(act_type), kind, &L, &n_chunks, &Kpad)) return false;
+    const size_t unit = (((size_t)L.n_planes * L.cb_chunks * L.Rr * 16) + 127) & ~(size_t)127;
+    const size_t pix = (((size_t)L.n_planes * L.Rr * 4) + 127) & ~(size_t)127;
+    const size_t fixed = (size_t)G_EPI_BYTES + pix + 256 + kGTail;
+    if (2 * unit + fixed + 3 * (size_t)kGBSlot > kGSmemBudget) return false;
+  }
+  return true;
 }
 
 cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, int out_type, cudaStream_t s,
@@ -1256,6 +1435,11 @@ cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, i
   cfg.dynamicSmemBytes = G->smem;
   cudaError_t e;
   const int outk = G->chain ? OUT_CHAIN : (out_type == 2 ? OUT_SIGNS : OUT_WORDS);
+  if (!G->chain && (outk == OUT_SIGNS) != (G->kind == TCG_SIGNS)) return cudaErrorInvalidValue;  // planned for the other kind
+  bool piped = G->mode == M_FP4 && outk == OUT_WORDS && G->words_even;
+  // rows are read two or four words at a time by the pipelined expanders: every input 8-byte aligned
+  for (int i = 0; piped && i < G->count; ++i)
+    if (reinterpret_cast<uintptr_t>(act[i]) & 7) piped = false;
 #define G_LAUNCH(M, O)                                                      \
   do {                                                                      \
     static unsigned long long done = 0;                                     \
@@ -1265,7 +1449,8 @@ cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, i
   if (G->mode == M_F16) {
     if (outk == OUT_WORDS) G_LAUNCH(M_F16, OUT_WORDS);
     else return cudaErrorInvalidValue;   // packed signs and chains need binary activations
-  } else if (outk == OUT_WORDS) G_LAUNCH(M_FP4, OUT_WORDS);
+  } else if (outk == OUT_WORDS && piped) G_LAUNCH(M_FP4, OUT_WORDS_PIPED);
+  else if (outk == OUT_WORDS) G_LAUNCH(M_FP4, OUT_WORDS);
   else if (outk == OUT_SIGNS) G_LAUNCH(M_FP4, OUT_SIGNS);
   else G_LAUNCH(M_FP4, OUT_CHAIN);
 #undef G_LAUNCH

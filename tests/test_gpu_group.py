@@ -219,6 +219,8 @@ def test_group_packed_sign_outputs(snn, oracle_mod):
         (wl.LayerShape(128, 256, 12, 12, 2, 1), 3),
         (wl.LayerShape(64, 512, 7, 7, 1, 1), 3),
         (wl.LayerShape(2, 40, 6, 6, 1, 1), 2),     # tiny c_in: many sums are exactly 0
+        (wl.LayerShape(96, 240, 6, 6, 1, 1), 2),   # the widest single channel tile of the packed-sign plan
+        (wl.LayerShape(64, 176, 6, 6, 1, 1), 2),   # one tile here, two under the word-output plan
     ]
     layers, acts, refs = [], [], []
     for i, (shape, n) in enumerate(members):

@@ -217,8 +217,11 @@ TC_SHAPES = [
     (200, 130, 7, 5, 1, 2),      # ragged channels in and out
     (1056, 48, 9, 8, 2, 1),      # several channel blocks, padded
     (512, 512, 7, 7, 1, 4),      # deep layer: two channel blocks, four channel tiles
-    (96, 240, 6, 6, 1, 2),       # the widest single channel tile of the 4-bit mode
-    (64, 248, 6, 6, 1, 2),       # just beyond it: two tiles, the second mostly padding
+    (96, 160, 6, 6, 1, 2),       # the widest single channel tile with three accumulator buffers (word outputs)
+    (64, 176, 6, 6, 1, 2),       # just beyond it: two tiles, the second mostly padding
+    (96, 240, 6, 6, 1, 2),       # the widest single channel tile with two accumulator buffers (packed signs)
+    (64, 248, 6, 6, 1, 2),       # just beyond that
+    (66, 64, 11, 9, 1, 3),       # an odd number of activation words per pixel: the expanders' plain loop
 ]
 
 
@@ -232,7 +235,7 @@ def test_tensor_core_shapes(snn, oracle_mod, c_in, c_out, h, w, stride, n):
 
 
 def test_tensor_core_many_tiles(snn, oracle_mod):
-    """More tiles than CTAs: both accumulator buffers, ring wrap-around, weight stages streamed over
+    """More tiles than CTAs: all accumulator buffers, ring wrap-around, weight stages streamed over
     several tiles of one CTA, and a tile assignment with a ragged last round."""
     for shape, n in [(wl.LayerShape(128, 128, 28, 28, 1, 1), 40), (wl.LayerShape(64, 64, 56, 56, 1, 1), 8),
                      (wl.LayerShape(256, 256, 14, 14, 1, 1), 48), (wl.LayerShape(512, 512, 7, 7, 1, 1), 64),
