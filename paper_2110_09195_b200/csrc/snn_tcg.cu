@@ -223,8 +223,10 @@ __device__ __forceinline__ bool g_issue_block(uint64_t a_unit, uint32_t wq, uint
 // OUTK: what the epilogue is compiled for.  0: fp32 or int32 words for every member; 1: packed signs for every
 // member; 2: a chain - packed signs between the members, any type for the last, and the dependency waits and
 // completion counters.  Keeping the variants apart keeps each one's registers and code to what it needs.
-// 3: words again, with the expanders' two-stage load pipeline instead of their plain loop (4-bit operands whose rows
-// can be read two words at a time); a separate instantiation so that neither carries the other's code.
+// 3: the common case of 0 compiled alone - fp32 outputs, 4-bit operands, every member's channel count a multiple
+// of 4 and its channel tile a multiple of 32, rows readable two words at a time: the expanders run their
+// two-stage load pipeline instead of the plain loop, and the epilogue has its one fast path and no other.  The
+// roles share instruction caches; what a variant does not carry makes the rest faster.
 enum { OUT_WORDS = 0, OUT_SIGNS = 1, OUT_CHAIN = 2, OUT_WORDS_PIPED = 3 };
 
 template <int MODE, int OUTK>
@@ -461,9 +463,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
       const int Nt = L.Nt, MT = L.MT, K = L.K;
       const float* alpha = L.alpha;
       const float* shift = L.shift;
-      const int out_i32 = WORDS ? (int)p.out_type[0] : OUTK == OUT_SIGNS ? 2 : (int)p.out_type[l];
+      const int out_i32 = PIPED ? 0 : WORDS ? (int)p.out_type[0] : OUTK == OUT_SIGNS ? 2 : (int)p.out_type[l];
       uint32_t* out32 = reinterpret_cast<uint32_t*>(p.out[l]);  // int32 and fp32 outputs share the layout
-      const bool fast = ((K & 3) == 0) && ((Nt & 31) == 0);
+      const bool fast = PIPED || (((K & 3) == 0) && ((Nt & 31) == 0));   // (checked on the host for variant 3)
       for (int tile = g_first_tile(L); tile < L.total_tiles; tile += G, ++seq, acc_slot = acc_slot + 1 == n_acc ? 0 : acc_slot + 1) {
         if (G_EPI_SPLIT && (int)(seq & 1) != half) continue;   // the other group's tile
         const uint32_t full_bar = bar_accfull + 8u * (uint32_t)(seq & 3), full_phase = (uint32_t)((seq >> 2) & 1);
@@ -1033,6 +1035,7 @@ struct GroupDev {
   int count = 0, act_type = 0, mode = M_FP4;
   int kind = TCG_WORDS;           // what the tiles were planned for (word outputs, packed signs, chain)
   bool words_even = false;        // every member has an even number of activation words per pixel
+  bool all_fast = false;          // every member: c_out a multiple of 4, channel tile a multiple of 32
   int chain = 0;                  // 1: member i + 1 reads the packed signs member i writes (one launch, dependency counters)
   uint8_t* chain_buf = nullptr;   // the packed signs between the members, one buffer per boundary
   size_t chain_off[SNN_GROUP_MAX] = {};
@@ -1305,9 +1308,11 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   G->grid = grid;
   G->chain = chain;
   G->kind = kind;
-  G->words_even = true;
-  for (int i = 0; i < count; ++i)
+  G->words_even = G->all_fast = true;
+  for (int i = 0; i < count; ++i) {
     if (gs[i].Cw & 1) G->words_even = false;
+    if ((gs[i].K & 3) || (host[i].Nt & 31)) G->all_fast = false;
+  }
   cudaError_t e = cudaMalloc(&G->weights, w_total);
   if (chain) {
     G->done_words = done_words;
@@ -1436,7 +1441,7 @@ cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, i
   cudaError_t e;
   const int outk = G->chain ? OUT_CHAIN : (out_type == 2 ? OUT_SIGNS : OUT_WORDS);
   if (!G->chain && (outk == OUT_SIGNS) != (G->kind == TCG_SIGNS)) return cudaErrorInvalidValue;  // planned for the other kind
-  bool piped = G->mode == M_FP4 && outk == OUT_WORDS && G->words_even;
+  bool piped = G->mode == M_FP4 && outk == OUT_WORDS && out_type == 0 && G->words_even && G->all_fast;
   // rows are read two or four words at a time by the pipelined expanders: every input 8-byte aligned
   for (int i = 0; piped && i < G->count; ++i)
     if (reinterpret_cast<uintptr_t>(act[i]) & 7) piped = false;
