@@ -58,7 +58,9 @@ constexpr int G_THREADS = 64 + 64 * G_EW + 64;
 constexpr int G_EXP_THREADS = 32 * G_EW;
 constexpr int G_EXP_ROWS = 3;                 // rows of a unit one expander thread loads together
 constexpr int G_EPI_PITCH = 128;
-constexpr int G_EPI_BYTES = G_EW * 32 * G_EPI_PITCH;
+constexpr int G_EPI_ALPHA = 1024;              // per epilogue warp: the scales of a tile's channels (at most 256)
+constexpr int G_EPI_WARP = 32 * G_EPI_PITCH + G_EPI_ALPHA;
+constexpr int G_EPI_BYTES = G_EW * G_EPI_WARP;
 constexpr int G_NS_MAX = 8;
 constexpr uint32_t G_ACC_COLS = 256;          // tensor-memory columns of one accumulator buffer
 constexpr uint32_t G_ACC_COLS_FP4 = 240;      // 4-bit mode, two buffers: columns 480..511 hold the (unit) block scales
@@ -445,7 +447,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     const int rq = warp & 3, half = ew >> 2;
     const int cfirst = G_EPI_SPLIT ? 0 : 32 * half, cstep = G_EPI_SPLIT ? 32 : 64;   // this warp's 32-column slices
     long long seq = 0;   // tiles of this CTA so far, over all problems (the MMA issuer alternates the buffers the same way)
-    uint8_t* stage = epi_smem + (size_t)ew * (32 * G_EPI_PITCH);
+    uint8_t* stage = epi_smem + (size_t)ew * G_EPI_WARP;
+    const uint32_t a_stage = smem_u32(stage) + 32 * G_EPI_PITCH;   // this warp's copy of the tile's scales
     const int srow = lane >> 3, scol = lane & 7;  // this lane's (row mod 4, 16-byte column) when storing
     // Staging tile: row r, 16-byte chunk c sits at r*128 + ((c ^ (r & 7)) << 4).  A lane writes its own row
     // (chunk e at st_lane ^ (e << 4)) and reads chunk scol of rows srow + 4i.
@@ -567,6 +570,19 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           uint32_t v[32];
           uint32_t roff[8];   // element offset of (row srow + 4i, this lane's four channels of a slice's first column), or none
           if (total_sl > 0) tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)cfirst, v);
+          if (PIPED) {
+            // The tile's scales go to shared memory once: a global load issued between the slices' stores waits
+            // behind them in the load/store unit's queue, one per slice was a stall of hundreds of cycles each.
+            __syncwarp();   // the previous tile's last slice has read its scales
+            for (int c = lane * 4; c < Nt; c += 128) {
+              float4 al = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (n0 + c < K) al = __ldg(reinterpret_cast<const float4*>(alpha + n0 + c));
+              asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a_stage + (uint32_t)c * 4u), "f"(al.x), "f"(al.y),
+                           "f"(al.z), "f"(al.w)
+                           : "memory");
+            }
+            __syncwarp();
+          }
           int mt = 0, ci = 0;
 #pragma unroll 1
           for (int sl = 0; sl < total_sl; ++sl) {
@@ -581,7 +597,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
             }
             const int co = n0 + c0 + scol * 4;
             unsigned long long alA = 0, alB = 0;   // (alpha[co], alpha[co+1]) and (alpha[co+2], alpha[co+3])
-            if (!out_i32 && co < K) {
+            if (PIPED) {
+              asm volatile("ld.shared.v2.b64 {%0,%1}, [%2];" : "=l"(alA), "=l"(alB) : "r"(a_stage + (uint32_t)(c0 + scol * 4) * 4u) : "memory");
+            } else if (!out_i32 && co < K) {
               const float4 al = __ldg(reinterpret_cast<const float4*>(alpha + co));
               asm("mov.b64 %0, {%1, %2};" : "=l"(alA) : "f"(al.x), "f"(al.y));
               asm("mov.b64 %0, {%1, %2};" : "=l"(alB) : "f"(al.z), "f"(al.w));
