@@ -56,6 +56,10 @@ constexpr int G_EW = 8;                       // epilogue warps = expander warps
 // shares its scheduler with two epilogue warps only instead of two epilogue and two expander warps.
 constexpr int G_THREADS = 64 + 64 * G_EW + 64;
 constexpr int G_EXP_THREADS = 32 * G_EW;
+#ifndef SNN_XG
+#define SNN_XG 2
+#endif
+constexpr int G_XTEAMS = SNN_XG;               // teams of expander warps in the pipelined form
 constexpr int G_EXP_ROWS = 3;                 // rows of a unit one expander thread loads together
 constexpr int G_EPI_PITCH = 128;
 constexpr int G_EPI_ALPHA = 1024;              // per epilogue warp: the scales of a tile's channels (at most 256)
@@ -113,6 +117,7 @@ struct GParams {
   int NA, NS;
   uint32_t a_slot_bytes, b_slot_bytes;
   uint32_t off_b, off_epi, off_pix, off_lay, off_tail;
+  uint32_t pix_words;     // entries of one pixel table (the pipelined expanders keep one per team)
 };
 
 // Profiling aid (build with -DSNN_TRACE): every role's reporting lane adds up the cycles it spends in its
@@ -274,7 +279,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     uint32_t count = 1;
     if (tid >= 28) count = G_EPI_ARRIVALS;             // acc_empty: one arrival per epilogue warp of the tile
     if (tid >= 16 && tid < 20)   // a_full: every expander thread arrives, or one lane per expander warp (pipelined form)
-      count = PIPED ? G_EXP_THREADS / 32 : G_EXP_THREADS;
+      count = PIPED ? G_EXP_THREADS / 32 / G_XTEAMS : G_EXP_THREADS;
     mbar_init(smem_u32(bars + tid), count);
   }
   if (tid == 32) *abort_flag = 0;
@@ -731,9 +736,16 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         uint32_t flags;             // bit j: row j exists; bit 4 + j: its pixel is inside the image; 8: four words per
                                     // row; 9: first group of its unit; 10: last group of its unit
       };
-      // issue side: the next group to load
-      int il = 0, itile = 0, itotal = 0, icb = 0, irb = 0, ik0 = 0, i_slot = 0;
+      // The expander warps form XG teams that take the units in turn (the ring has a multiple of XG slots, so a
+      // slot always belongs to the same team): with few rows per unit a unit is a chain of latencies, and two
+      // chains in flight are what doubles the rate.
+      constexpr int XG = G_XTEAMS, XT = G_EXP_THREADS / XG;
+      const int gx = et / XT, etg = et % XT;
+      int* const pix = pix_tab + gx * (int)p.pix_words;
+      // issue side: the unit (il, itile, icb) with sequence number iu, and the next group to load in it
+      int il = 0, itile = 0, itotal = 0, icb = 0, irb = 0, ik0 = 0, i_slot = 0, iu = 0;
       int Rr = 0, n_planes = 0, n_cb = 0, cbc = 0, Cw = 0, all_rows = 0, kstep = 2;
+      int pix_l = -1, pix_t = -1;   // the tile the pixel table holds
       const uint32_t* act = nullptr;
       bool ivalid = false;
       auto enter_layer = [&]() {   // first layer from il on in which this CTA has a tile
@@ -746,19 +758,36 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           all_rows = n_planes * Rr;
           act = reinterpret_cast<const uint32_t*>(p.act[il]);
           kstep = ((reinterpret_cast<uintptr_t>(act) & 15) == 0 && (Cw & 3) == 0 && (cbc & 3) == 0) ? 4 : 2;
-          icb = irb = ik0 = 0;
+          icb = 0;
           ivalid = true;
           return;
         }
         ivalid = false;
       };
-      auto enter_tile = [&]() {    // input pixel of each of this thread's rows of the tile
-        const GLayer& L = lay[il];
-        const int mg = (int)fdiv((uint32_t)itile, L.dNt);
-        const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * L.MT);
-        for (int f = et; f < all_rows; f += G_EXP_THREADS) {
-          const int pl = (f >= Rr) + (f >= 2 * Rr) + (f >= 3 * Rr);
-          pix_tab[f] = g_position_to_pixel(L, Q0 + (uint32_t)(f - pl * Rr), pl >> 1, pl & 1);
+      auto next_unit = [&]() {     // the unit after (il, itile, icb) in the CTA's sequence
+        ++iu;
+        i_slot = i_slot + 1 == NA ? 0 : i_slot + 1;
+        if (++icb >= n_cb) {
+          icb = 0;
+          itile += G;
+          if (itile >= itotal) {
+            ++il;
+            enter_layer();
+          }
+        }
+      };
+      auto seek_own = [&]() {      // on to this team's next unit; input pixel of each of this thread's rows of its tile
+        while (ivalid && (iu % XG) != gx) next_unit();
+        if (ivalid && (pix_l != il || pix_t != itile)) {
+          const GLayer& L = lay[il];
+          const int mg = (int)fdiv((uint32_t)itile, L.dNt);
+          const uint32_t Q0 = (uint32_t)mg * (uint32_t)(128 * L.MT);
+          for (int f = etg; f < all_rows; f += XT) {
+            const int pl = (f >= Rr) + (f >= 2 * Rr) + (f >= 3 * Rr);
+            pix[f] = g_position_to_pixel(L, Q0 + (uint32_t)(f - pl * Rr), pl >> 1, pl & 1);
+          }
+          pix_l = il;
+          pix_t = itile;
         }
       };
       auto issue = [&](XGroup& g) {   // loads of the group at the issue position; moves the position on
@@ -767,15 +796,15 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         const uint32_t unit = smem_u32(a_smem) + (uint32_t)i_slot * p.a_slot_bytes;
 #pragma unroll
         for (int j = 0; j < G_EXP_ROWS; ++j) {
-          const int f = irb + et + j * G_EXP_THREADS;
-          const int pix = f < all_rows ? pix_tab[f] : -2;
+          const int f = irb + etg + j * XT;
+          const int px = f < all_rows ? pix[f] : -2;
           const int pl = (f >= Rr) + (f >= 2 * Rr) + (f >= 3 * Rr);
           g.da[j] = unit + (uint32_t)(pl * cbc * Rr + (f - pl * Rr)) * 16u + (uint32_t)ik0 * cs;
-          if (pix != -2) flags |= 1u << j;
+          if (px != -2) flags |= 1u << j;
           g.t[j] = make_uint4(0, 0, 0, 0);
-          if (pix >= 0) {
+          if (px >= 0) {
             flags |= 0x10u << j;
-            const uint32_t* src = act + wide_mul((uint32_t)pix, (uint32_t)Cw) + icb * cbc + ik0;
+            const uint32_t* src = act + wide_mul((uint32_t)px, (uint32_t)Cw) + icb * cbc + ik0;
             if (kstep == 4) {
               g.t[j] = __ldg(reinterpret_cast<const uint4*>(src));
             } else {
@@ -789,26 +818,20 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         ik0 += kstep;
         if (ik0 >= cbc) {
           ik0 = 0;
-          irb += G_EXP_ROWS * G_EXP_THREADS;
+          irb += G_EXP_ROWS * XT;
           if (irb >= all_rows) {   // the unit ends with this group
             irb = 0;
             flags |= 0x400u;
-            i_slot = i_slot + 1 == NA ? 0 : i_slot + 1;
-            if (++icb >= n_cb) {
-              icb = 0;
-              itile += G;
-              if (itile >= itotal) {
-                ++il;
-                enter_layer();
-              }
-              if (ivalid) enter_tile();
-            }
+            next_unit();
+            seek_own();
           }
         }
         g.flags = flags;
       };
       enter_layer();
-      if (ivalid) enter_tile();
+      seek_own();
+      // completion side: this team's slots gx, gx + XG, ... of the ring
+      a_slot = gx;
       XGroup cur, nxt;
       bool nvalid = ivalid;
       if (nvalid) issue(nxt);
@@ -816,7 +839,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
         cur = nxt;
         nvalid = ivalid;
         if (nvalid) issue(nxt);
-        if ((cur.flags & 0x200u) && a_done >= NA) {
+        if ((cur.flags & 0x200u) && a_done >= NA / XG) {
           int okf = 1;
           if (lane == 0) okf = (!*abort_flag && TR_WAIT(tr_w0, mbar_wait_backoff(bar_aempty + 8 * a_slot, a_phase, 64))) ? 1 : 0;
           okf = __shfl_sync(0xffffffffu, okf, 0);
@@ -847,7 +870,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_afull + 8 * a_slot);
           ++a_done;
-          if (++a_slot == NA) { a_slot = 0; a_phase ^= 1u; }
+          a_slot += XG;
+          if (a_slot >= NA) { a_slot -= NA; a_phase ^= 1u; }
         }
       }
     }
@@ -1235,9 +1259,14 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   }
   a_slot = (a_slot + 127) & ~(size_t)127;
   pix_bytes = (pix_bytes + 127) & ~(size_t)127;
+  const size_t pix_one = pix_bytes;
+  if (mode == M_FP4 && kind == TCG_WORDS) pix_bytes *= G_XTEAMS;   // one table per expander team
   const size_t lay_bytes = ((size_t)count * sizeof(GLayer) + 127) & ~(size_t)127;
   const size_t fixed = (size_t)G_EPI_BYTES + pix_bytes + lay_bytes + kGTail;
-  int na = 3, ns = 0;
+  // ring depth: three slots if they fit, else two; the plan for word outputs on 4-bit operands takes two, a
+  // multiple of the number of expander teams (four slots never fit beside three weight slots of these sizes)
+  int na = (mode == M_FP4 && kind == TCG_WORDS) ? 2 : 3, ns = 0;
+  static_assert(G_XTEAMS == 1 || G_XTEAMS == 2, "the ring depth below is a multiple of the team count");
   for (; na >= 2; --na) {
     if ((size_t)na * a_slot + fixed + 3 * (size_t)kGBSlot > kGSmemBudget) continue;
     ns = (int)((kGSmemBudget - fixed - (size_t)na * a_slot) / kGBSlot);
@@ -1382,6 +1411,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   p.off_epi = p.off_b + (uint32_t)ns * kGBSlot;
   p.off_pix = p.off_epi + G_EPI_BYTES;
   p.off_lay = p.off_pix + (uint32_t)pix_bytes;
+  p.pix_words = (uint32_t)(pix_one / 4);
   p.off_tail = p.off_lay + (uint32_t)lay_bytes;
   G->smem = (size_t)p.off_tail + kGTail;
   if (G->smem > (size_t)kMaxDynSmem || G->smem >= (1u << 18)) {
