@@ -508,6 +508,8 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
           // owns one position and the 32 (or 16) consecutive channels of a slice, i.e. one word (or
           // half-word) of the next layer's binary input.  No transposition, one small store per slice.
           const int Kw = (K + 31) >> 5;
+          // the scale and threshold arrays can be read four at a time (their allocations are; a tile starts at a multiple of 16)
+          const bool sign_vec = ((reinterpret_cast<uintptr_t>(alpha) | reinterpret_cast<uintptr_t>(shift)) & 15) == 0;
           if ((Nt & 31) == 0) {
             const int per_mt = (Nt - cfirst + cstep - 1) / cstep;
 #pragma unroll 1
@@ -520,7 +522,35 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
                 __syncwarp();  // the load is a warp-wide instruction: no lane may still be in the store below
                 tmem_ld32(d0 + ((uint32_t)(rq * 32) << 16) + (uint32_t)(mt * Nt + c0), v);
                 tmem_ld_wait();
-                if (pix >= 0 && co0 < K) {
+                if (pix >= 0 && co0 + 32 <= K && sign_vec) {
+                  // all 32 channels exist: scales and thresholds four at a time (the same addresses in every
+                  // lane), multiply and add as packed fp32 pairs - each half rounds as the scalar instruction does
+                  uint32_t word = 0;
+#pragma unroll
+                  for (int e = 0; e < 32; e += 4) {
+                    const float4 a = __ldg(reinterpret_cast<const float4*>(alpha + co0 + e));
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(shift + co0 + e));
+                    unsigned long long x0, x1, m0, m1, t0, t1;
+                    asm("mov.b64 %0, {%1, %2};" : "=l"(x0) : "r"(v[e]), "r"(v[e + 1]));
+                    asm("mov.b64 %0, {%1, %2};" : "=l"(x1) : "r"(v[e + 2]), "r"(v[e + 3]));
+                    asm("mov.b64 %0, {%1, %2};" : "=l"(m0) : "f"(a.x), "f"(a.y));
+                    asm("mov.b64 %0, {%1, %2};" : "=l"(m1) : "f"(a.z), "f"(a.w));
+                    asm("mov.b64 %0, {%1, %2};" : "=l"(t0) : "f"(t.x), "f"(t.y));
+                    asm("mov.b64 %0, {%1, %2};" : "=l"(t1) : "f"(t.z), "f"(t.w));
+                    asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(x0) : "l"(m0));
+                    asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(x1) : "l"(m1));
+                    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(x0) : "l"(t0));
+                    asm("add.rn.f32x2 %0, %0, %1;" : "+l"(x1) : "l"(t1));
+                    float y0, y1, y2, y3;
+                    asm("mov.b64 {%0, %1}, %2;" : "=f"(y0), "=f"(y1) : "l"(x0));
+                    asm("mov.b64 {%0, %1}, %2;" : "=f"(y2), "=f"(y3) : "l"(x1));
+                    word |= (y0 >= 0.f ? 1u : 0u) << e;
+                    word |= (y1 >= 0.f ? 1u : 0u) << (e + 1);
+                    word |= (y2 >= 0.f ? 1u : 0u) << (e + 2);
+                    word |= (y3 >= 0.f ? 1u : 0u) << (e + 3);
+                  }
+                  out32[wide_mul((uint32_t)pix, (uint32_t)Kw) + (uint32_t)(co0 >> 5)] = word;
+                } else if (pix >= 0 && co0 < K) {
                   uint32_t word = 0;
 #pragma unroll
                   for (int e = 0; e < 32; ++e) {
