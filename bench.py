@@ -181,8 +181,8 @@ def run_reference(args):
 # the kernel's sources are the ones that were profiled: {kernel: (workload, batch, bytes, sha256 of sources)}
 _TRAFFIC = {
     # profiles/dram_traffic_resnet18_stack_n64_grouped.txt: mean of the two captured launches
-    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 343414912,
-                                             "e8cf4af385d6489a4c71d3c02ce714c3f8cb710259305b9a14950a4340c6ed72"),
+    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 351543424,
+                                             "b02e7e908933656337ca771c5bbd9aac961ddfc545de6ada92ffc9d84185d3c9"),
 }
 
 
