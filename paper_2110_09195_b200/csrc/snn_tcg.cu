@@ -704,6 +704,27 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
               const int co0 = n0 + c0;
               if (pix < 0 || co0 >= K) continue;
               uint32_t* o = out32 + wide_mul((uint32_t)pix, (uint32_t)K) + co0;
+              if ((K & 3) == 0 && co0 + 16 <= K) {
+                // all 16 channels exist and rows are 16-byte aligned: four channels per load, multiply and store
+#pragma unroll
+                for (int e = 0; e < 16; e += 4) {
+                  uint4 r;
+                  if (out_i32) {
+                    r.x = (uint32_t)__float2int_rn(__uint_as_float(v[e]));
+                    r.y = (uint32_t)__float2int_rn(__uint_as_float(v[e + 1]));
+                    r.z = (uint32_t)__float2int_rn(__uint_as_float(v[e + 2]));
+                    r.w = (uint32_t)__float2int_rn(__uint_as_float(v[e + 3]));
+                  } else {
+                    const float4 al = __ldg(reinterpret_cast<const float4*>(alpha + co0 + e));
+                    r.x = __float_as_uint(__fmul_rn(__uint_as_float(v[e]), al.x));
+                    r.y = __float_as_uint(__fmul_rn(__uint_as_float(v[e + 1]), al.y));
+                    r.z = __float_as_uint(__fmul_rn(__uint_as_float(v[e + 2]), al.z));
+                    r.w = __float_as_uint(__fmul_rn(__uint_as_float(v[e + 3]), al.w));
+                  }
+                  *reinterpret_cast<uint4*>(o + e) = r;
+                }
+                continue;
+              }
 #pragma unroll
               for (int e = 0; e < 16; ++e) {
                 if (co0 + e < K) {
