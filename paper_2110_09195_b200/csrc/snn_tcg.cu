@@ -762,9 +762,9 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
     bool stop = false;
     long long tr_w0 = 0, tr_t0 = clock64();
     (void)tr_w0; (void)tr_t0; (void)exp_flag; (void)dep_flag;
-    if (!CHAIN) {
+    if (!CHAIN && FP4) {
       // Independent problems: all inputs exist when the launch starts and are small beside the L2 (1/29 of the
-      // outputs).  The CTAs pull them into L2 together, once, so that the staging loads below see L2 latency
+      // outputs; fp16 inputs are not: half of the outputs).  The CTAs pull them into L2 together, once, so that the staging loads below see L2 latency
       // instead of DRAM latency: a unit is one round trip, and the round trip is what the expanders' rate is.
       for (int l = 0; l < p.n_layers; ++l) {
         const GLayer& L = lay[l];
@@ -1005,7 +1005,24 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
                 const int pl = (f >= Rr) + (f >= 2 * Rr) + (f >= 3 * Rr);
                 dst[j] = unit + ((size_t)pl * cb_chunks * Rr + (size_t)(f - pl * Rr)) * 16;
               }
-              if (F16) {
+              if (F16 && vec) {
+                // fp16 activations are copied: asynchronous 16-byte copies straight into the unit (zero-filled where
+                // the row is padding or the channels end), all of a thread's chunks in flight together; the thread
+                // waits for its own copies before it makes them visible to the tensor core and arrives.
+#pragma unroll
+                for (int j = 0; j < G_EXP_ROWS; ++j) {
+                  if (pix[j] == -2) continue;
+                  const __half* row = (const __half*)act + wide_mul((uint32_t)(pix[j] < 0 ? 0 : pix[j]), (uint32_t)C);
+                  const uint32_t d = smem_u32(dst[j]);
+                  for (int c0 = 0; c0 < cb_chunks; ++c0) {
+                    const int ch = (cb * cb_chunks + c0) * 8;  // first channel of the chunk
+                    const bool on = pix[j] >= 0 && ch < C;
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d + (uint32_t)c0 * (uint32_t)Rr * 16u),
+                                 "l"(on ? (const void*)(row + ch) : act), "r"(on ? 16 : 0)
+                                 : "memory");
+                  }
+                }
+              } else if (F16) {
                 for (int c0 = 0; c0 < cb_chunks; c0 += 2) {
                   uint4 v[G_EXP_ROWS][2];
 #pragma unroll
@@ -1105,6 +1122,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
               }
             }
           }
+          if (F16) asm volatile("cp.async.wait_all;" ::: "memory");
           fence_proxy_async();  // generic-proxy writes -> visible to the tensor core's reads
           mbar_arrive(bar_afull + 8 * a_slot);
           ++a_done;
