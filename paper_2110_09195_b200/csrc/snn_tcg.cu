@@ -19,7 +19,8 @@
 // What makes this possible is a ring geometry that is the same for every problem:
 //   activation units  NA slots of a_slot_bytes   (a problem's unit uses a prefix)
 //   weight stages     NS slots of b_slot_bytes   (a stage = whole taps of one channel block)
-//   accumulators      three buffers of 160 (e2m1) or two of 256 (fp16) tensor-memory columns
+//   accumulators      two or three buffers of tensor-memory columns (by operand mode and output kind:
+//                     3 x 160 for word outputs on e2m1 operands, else 2 x 240; 2 x 256 with fp16 operands)
 // so slots, barriers and phases simply carry on from one problem to the next.
 // Tiles of a problem are dealt to the CTAs round-robin; which CTAs get a problem's odd
 // tiles is decided on the host from the time the CTAs have been given so far, so that the
@@ -31,8 +32,9 @@
 //                    128-byte row stores; or TMEM -> registers -> threshold -> packed sign words
 //      warps 10-19   expanders (13 and 17 idle): packed bits -> e2m1 nibbles (or fp16 copied)
 //                    into the activation ring
-// The kernel is compiled per operand mode and per output kind (words, packed signs, chain), so that
-// no variant carries another one's code in its loops.
+// The kernel is compiled per operand mode and per output kind (words, the common case of words alone, packed
+// signs, chain), so that no variant carries another one's code in its loops; the plan (tile shapes, accumulator
+// buffers) is made per output kind as well.
 // Every wait is bounded; one that runs out raises a status word the host reads, and
 // the CTA still frees its tensor memory and returns.
 #include <algorithm>
