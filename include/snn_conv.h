@@ -66,8 +66,9 @@ enum {
 };
 enum {
   SNN_PATH_AUTO = 0,       /* tuned choice if snn_conv_tune ran for the shape, else a heuristic */
-  SNN_PATH_REUSE = 1,      /* codebook-reuse: per-channel partial maps + index-driven accumulate (Sec. 4.5) */
-  SNN_PATH_DECODED = 2,    /* decoded weights, XOR + popcount implicit GEMM (Sec. 3) */
+  SNN_PATH_REUSE = 1,      /* codebook-reuse: per-channel partial maps + index-driven accumulate (Sec. 4.5);
+                              binary activations, or fp16 activations with at most 1024 output channels */
+  SNN_PATH_DECODED = 2,    /* decoded weights, XOR + popcount implicit GEMM (Sec. 3); binary activations */
   SNN_PATH_DECODED_TC = 3  /* decoded weights on the tcgen05 tensor cores */
 };
 

@@ -11,7 +11,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 INCLUDE = PKG.parent / "include"
 LIB = PKG / "libsnnconv.so"
-SOURCES = ["snn_api.cu", "snn_decode.cu", "snn_popc.cu", "snn_reuse.cu", "snn_tcg.cu", "snn_microbench.cu", "snn_static.cu"]
+SOURCES = ["snn_api.cu", "snn_decode.cu", "snn_popc.cu", "snn_reuse.cu", "snn_reuse_f16.cu", "snn_tcg.cu", "snn_microbench.cu", "snn_static.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", f"-I{INCLUDE}", f"-I{CSRC}",

@@ -47,6 +47,9 @@ cudaError_t popc_forward(const LayerDev& L, const Geom& g, const Launch& l, int*
 
 bool reuse_supported(const Geom& g, int act_type);
 cudaError_t reuse_forward(const LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched);
+// the same sharing with fp16 activations (snn_reuse_f16.cu); reuse_supported / reuse_forward dispatch to these
+bool reuse_f16_supported(const Geom& g);
+cudaError_t reuse_f16_forward(const LayerDev& L, const Geom& g, const Launch& l, int* launched);
 
 // The tensor-core kernel (snn_tcg.cu) runs one layer, several independent layers, or a chain of dependent
 // layers as ONE persistent launch; a single layer is a group of one.

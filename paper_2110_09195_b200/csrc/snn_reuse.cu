@@ -208,6 +208,7 @@ __global__ void __launch_bounds__(256) reuse_conv_kernel(const ReuseParams p) {
 }
 
 bool reuse_supported(const Geom& g, int act_type) {
+  if (act_type == SNN_ACT_F16) return reuse_f16_supported(g);
   if (act_type != SNN_ACT_BIN) return false;
   // 16-bit lanes hold the matching-tap total 9*C
   return (long long)9 * g.C <= 65535;
@@ -229,7 +230,7 @@ static cudaError_t launch_reuse(const ReuseParams& p, size_t smem, dim3 grid, in
 }
 
 cudaError_t reuse_forward(const LayerDev& L, const Geom& g, int act_type, const Launch& l, int* launched) {
-  (void)act_type;
+  if (act_type == SNN_ACT_F16) return reuse_f16_forward(L, g, l, launched);
   ReuseParams p;
   p.act = (const uint32_t*)l.act;
   p.idx = L.idx;

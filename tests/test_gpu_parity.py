@@ -199,6 +199,20 @@ def test_f16_activation_variant(snn, oracle_mod, c_in, c_out, h, w, stride, pad,
     assert len(ran) >= 2  # at least one named path plus AUTO
 
 
+@pytest.mark.parametrize("c_in,c_out,h,w,stride,pad,tau,n", [
+    (64, 300, 6, 6, 1, 1, 5, 2),     # two output channels per thread
+    (8, 520, 5, 5, 2, 1, 9, 2),      # the full codebook: one input channel per table; four channels per thread
+    (24, 16, 7, 9, 1, 0, 1, 3),      # two codebook kernels
+    (35, 9, 6, 5, 2, 1, 3, 2),       # c_in not a multiple of 8: scalar staging, ragged last chunk
+])
+def test_f16_codebook_reuse_form(snn, oracle_mod, c_in, c_out, h, w, stride, pad, tau, n):
+    """The fp16-activation variant through the codebook-reuse path (the paper's deployment form: signed
+    additions once per codebook kernel, then the index-driven accumulation), at the fp16 tolerance."""
+    shape = wl.LayerShape(c_in, c_out, h, w, stride, pad)
+    ran = check_f16_layer(snn, oracle_mod, shape, tau, n, 97)
+    assert snn.PATH_REUSE in ran
+
+
 def test_tensor_core_path_runs_the_stack_shapes(snn):
     """The tcgen05 path must cover every ResNet-18/34 layer shape at the benchmark batch."""
     wk = wl.get_workload("resnet18")
@@ -251,12 +265,14 @@ def test_tensor_core_fp16(snn, oracle_mod):
 
 
 def test_auto_refuses_a_layer_no_path_can_run(snn):
-    """fp16 activations run on the tensor-core path only; a map so wide that one activation unit no longer
-    fits shared memory must be refused (status UNSUPPORTED), by name and by AUTO, with nothing launched."""
-    shape = wl.LayerShape(16, 16, 3, 700, 1, 1)
+    """fp16 activations run on the tensor-core path or, up to 1024 output channels, on the reuse path; a layer
+    with more channels on a map so wide that one activation unit no longer fits shared memory must be refused
+    (status UNSUPPORTED), by name and by AUTO, with nothing launched."""
+    shape = wl.LayerShape(16, 1040, 3, 700, 1, 1)
     p = wl.draw_layer_params(shape, 5, 7)
-    layer = snn.SnnConv(16, 16, 5, p.codebook, p.idx_packed, p.alpha, act_type=snn.ACT_F16)
+    layer = snn.SnnConv(16, 1040, 5, p.codebook, p.idx_packed, p.alpha, act_type=snn.ACT_F16)
     assert not layer.path_supported(snn.PATH_DECODED_TC, 1, 3, 700)
+    assert not layer.path_supported(snn.PATH_REUSE, 1, 3, 700)
     act = torch.zeros((1, 3, 700, 16), dtype=torch.float16, device="cuda")
     before = snn.kernel_launches()
     for path in (snn.PATH_AUTO, snn.PATH_DECODED_TC, snn.PATH_DECODED, snn.PATH_REUSE):
