@@ -3,7 +3,7 @@
 //   stage 1   P[ci][k][pixel] = sum over the nine taps of  K_k[tap] * a[pixel + tap][ci]      (+/- additions)
 //             for every kernel k of the layer's codebook, once per input channel and pixel,
 //   stage 2   S[co][pixel] = sum over ci of P[ci][idx[co][ci]][pixel]                           (index-driven)
-// and Y = alpha[co] * S.  Sums are fp32 (the oracle's are fp64; the tolerance of the fp16 variant covers it).
+// and Y = alpha[co] * S.  Sums are fp32, in the order of the two stages.
 //
 // One CTA owns 16 consecutive output pixels and all output channels.  Input channels go through in chunks
 // of CC = min(8, 512 / 2^tau): the chunk's 3x3 windows are converted to fp32 in shared memory, stage 1 fills
