@@ -181,8 +181,8 @@ def run_reference(args):
 # the kernel's sources are the ones that were profiled: {kernel: (workload, batch, bytes, sha256 of sources)}
 _TRAFFIC = {
     # profiles/dram_traffic_resnet18_stack_n64_grouped.txt: mean of the two captured launches
-    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 351543424,
-                                             "b02e7e908933656337ca771c5bbd9aac961ddfc545de6ada92ffc9d84185d3c9"),
+    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 351878912,
+                                             "6d33739769ec708af9774c7eff8d9df457ac5f0f946bce7aa3284b08c7b43a78"),
 }
 
 
