@@ -182,7 +182,7 @@ def run_reference(args):
 _TRAFFIC = {
     # profiles/dram_traffic_resnet18_stack_n64_grouped.txt: mean of the two captured launches
     "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 351878912,
-                                             "6d33739769ec708af9774c7eff8d9df457ac5f0f946bce7aa3284b08c7b43a78"),
+                                             "314c22579083c5d34dbd81d82e9ccc88b2956fe90749d4096e4318c48d135b0b"),
 }
 
 

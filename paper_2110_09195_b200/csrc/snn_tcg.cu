@@ -58,10 +58,7 @@ constexpr int G_EW = 8;                       // epilogue warps = expander warps
 // shares its scheduler with two epilogue warps only instead of two epilogue and two expander warps.
 constexpr int G_THREADS = 64 + 64 * G_EW + 64;
 constexpr int G_EXP_THREADS = 32 * G_EW;
-#ifndef SNN_XG
-#define SNN_XG 2
-#endif
-constexpr int G_XTEAMS = SNN_XG;               // teams of expander warps in the pipelined form
+constexpr int G_XTEAMS = 2;                    // teams of expander warps in the pipelined form
 constexpr int G_EXP_ROWS = 3;                 // rows of a unit one expander thread loads together
 constexpr int G_EPI_PITCH = 128;
 constexpr int G_EPI_ALPHA = 1024;              // per epilogue warp: the scales of a tile's channels (at most 256)
