@@ -1144,8 +1144,7 @@ __global__ void __launch_bounds__(G_THREADS, 1) tcg_conv_kernel(const GParams p)
 struct GroupDev {
   int count = 0, act_type = 0, mode = M_FP4;
   int kind = TCG_WORDS;           // what the tiles were planned for (word outputs, packed signs, chain)
-  bool words_even = false;        // every member has an even number of activation words per pixel
-  bool all_fast = false;          // every member: c_out a multiple of 4, channel tile a multiple of 32
+  bool hot = false;               // planned for the hot variant of the word-output kernel (see tcg_create)
   int chain = 0;                  // 1: member i + 1 reads the packed signs member i writes (one launch, dependency counters)
   uint8_t* chain_buf = nullptr;   // the packed signs between the members, one buffer per boundary
   size_t chain_off[SNN_GROUP_MAX] = {};
@@ -1218,14 +1217,14 @@ inline int g_mode_for(int act_type) { return act_type == SNN_ACT_F16 ? M_F16 : M
 // channel plus a constant that does not overlap the previous MMA.
 inline double g_mma_cycles(int nt) { return 0.5 * nt + 33.0; }
 
-inline int g_n_acc(int mode, int kind) { return (mode == M_FP4 && kind == TCG_WORDS) ? G_NACC_WORDS : G_NACC; }
-inline int g_acc_cols(int mode, int kind) {
-  return mode != M_FP4 ? (int)G_ACC_COLS : kind == TCG_WORDS ? (int)G_ACC_COLS_FP4_3 : (int)G_ACC_COLS_FP4;
+// tensor-memory columns of one accumulator buffer when there are n_acc of them
+inline int g_acc_cols(int mode, int n_acc) {
+  return mode != M_FP4 ? (int)G_ACC_COLS : n_acc == G_NACC_WORDS ? (int)G_ACC_COLS_FP4_3 : (int)G_ACC_COLS_FP4;
 }
 
-bool g_plan_layer(const Geom& g, int mode, int kind, GLayer* L, int* n_chunks_out, int* Kpad_out) {
+bool g_plan_layer(const Geom& g, int mode, int n_acc, GLayer* L, int* n_chunks_out, int* Kpad_out) {
   const int cpc = mode == M_F16 ? 8 : 32;
-  const int acc_cols = g_acc_cols(mode, kind);
+  const int acc_cols = g_acc_cols(mode, n_acc);
   const int raw = round_up(g.C, 2 * cpc) / cpc;  // 16-byte chunks along the channels, even
   GLayer& o = *L;
   o.N = g.N; o.H = g.H; o.W = g.W; o.C = g.C; o.K = g.K; o.Cw = g.Cw;
@@ -1315,8 +1314,20 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   size_t w_off[SNN_GROUP_MAX], w_total = 0;
   size_t a_slot = 0, pix_bytes = 0;
   long long tiles = 0;
+  // Word outputs on 4-bit operands get three accumulator buffers where the launch can run its hot variant (every
+  // member: c_out a multiple of 4, channel tile a multiple of 32, an even number of activation words per pixel);
+  // with the plain expanders two larger buffers measure faster, so everything else is planned with two.
+  int n_acc = (mode == M_FP4 && kind == TCG_WORDS) ? G_NACC_WORDS : G_NACC;
+  bool hot = n_acc == G_NACC_WORDS;
+  if (hot) {
+    for (int i = 0; i < count && hot; ++i) {
+      if (!g_plan_layer(gs[i], mode, n_acc, &host[i], &n_chunks[i], &Kpad[i])) return cudaErrorInvalidConfiguration;
+      if ((gs[i].Cw & 1) || (gs[i].K & 3) || (host[i].Nt & 31)) hot = false;
+    }
+    if (!hot) n_acc = G_NACC;
+  }
   for (int i = 0; i < count; ++i) {
-    if (!g_plan_layer(gs[i], mode, kind, &host[i], &n_chunks[i], &Kpad[i])) return cudaErrorInvalidConfiguration;
+    if (!g_plan_layer(gs[i], mode, n_acc, &host[i], &n_chunks[i], &Kpad[i])) return cudaErrorInvalidConfiguration;
     const size_t unit = (size_t)host[i].n_planes * host[i].cb_chunks * host[i].Rr * 16;
     if (unit > a_slot) a_slot = unit;
     const size_t pb = (size_t)host[i].n_planes * host[i].Rr * 4;
@@ -1328,12 +1339,12 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   a_slot = (a_slot + 127) & ~(size_t)127;
   pix_bytes = (pix_bytes + 127) & ~(size_t)127;
   const size_t pix_one = pix_bytes;
-  if (mode == M_FP4 && kind == TCG_WORDS) pix_bytes *= G_XTEAMS;   // one table per expander team
+  if (hot) pix_bytes *= G_XTEAMS;   // one table per expander team
   const size_t lay_bytes = ((size_t)count * sizeof(GLayer) + 127) & ~(size_t)127;
   const size_t fixed = (size_t)G_EPI_BYTES + pix_bytes + lay_bytes + kGTail;
   // ring depth: three slots if they fit, else two; the plan for word outputs on 4-bit operands takes two, a
   // multiple of the number of expander teams (four slots never fit beside three weight slots of these sizes)
-  int na = (mode == M_FP4 && kind == TCG_WORDS) ? 2 : 3, ns = 0;
+  int na = hot ? 2 : 3, ns = 0;
   static_assert(G_XTEAMS == 1 || G_XTEAMS == 2, "the ring depth below is a multiple of the team count");
   for (; na >= 2; --na) {
     if ((size_t)na * a_slot + fixed + 3 * (size_t)kGBSlot > kGSmemBudget) continue;
@@ -1423,11 +1434,7 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   G->grid = grid;
   G->chain = chain;
   G->kind = kind;
-  G->words_even = G->all_fast = true;
-  for (int i = 0; i < count; ++i) {
-    if (gs[i].Cw & 1) G->words_even = false;
-    if ((gs[i].K & 3) || (host[i].Nt & 31)) G->all_fast = false;
-  }
+  G->hot = hot;
   cudaError_t e = cudaMalloc(&G->weights, w_total);
   if (chain) {
     G->done_words = done_words;
@@ -1471,8 +1478,8 @@ cudaError_t tcg_create(const LayerDev* const* Ls, const Geom* gs, int count, int
   p.n_layers = count;
   p.NA = na;
   p.NS = ns;
-  p.acc_cols = (uint32_t)g_acc_cols(mode, kind);
-  p.n_acc = g_n_acc(mode, kind);
+  p.acc_cols = (uint32_t)g_acc_cols(mode, n_acc);
+  p.n_acc = n_acc;
   p.a_slot_bytes = (uint32_t)a_slot;
   p.b_slot_bytes = kGBSlot;
   p.off_b = (uint32_t)((size_t)na * a_slot);
@@ -1506,14 +1513,14 @@ int tcg_count(const GroupDev* G) { return G->count; }
 bool tcg_supported(const Geom& g, int act_type) {
   // one problem alone, under every plan a launch may use: two activation slots, the fixed parts and three
   // weight slots must fit
-  for (int kind = TCG_WORDS; kind <= TCG_SIGNS; ++kind) {
-    if (kind != TCG_WORDS && act_type != SNN_ACT_BIN) continue;
+  const int mode = g_mode_for(act_type);
+  for (int n_acc = G_NACC; n_acc <= (mode == M_FP4 ? G_NACC_WORDS : G_NACC); ++n_acc) {
     GLayer L;
     int n_chunks = 0, Kpad = 0;
-    if (!g_plan_layer(g, g_mode_for(act_type), kind, &L, &n_chunks, &Kpad)) return false;
+    if (!g_plan_layer(g, mode, n_acc, &L, &n_chunks, &Kpad)) return false;
     const size_t unit = (((size_t)L.n_planes * L.cb_chunks * L.Rr * 16) + 127) & ~(size_t)127;
     const size_t pix = (((size_t)L.n_planes * L.Rr * 4) + 127) & ~(size_t)127;
-    const size_t fixed = (size_t)G_EPI_BYTES + pix + 256 + kGTail;
+    const size_t fixed = (size_t)G_EPI_BYTES + G_XTEAMS * pix + 256 + kGTail;
     if (2 * unit + fixed + 3 * (size_t)kGBSlot > kGSmemBudget) return false;
   }
   return true;
@@ -1557,7 +1564,7 @@ cudaError_t tcg_forward(GroupDev* G, const void* const* act, void* const* out, i
   cudaError_t e;
   const int outk = G->chain ? OUT_CHAIN : (out_type == 2 ? OUT_SIGNS : OUT_WORDS);
   if (!G->chain && (outk == OUT_SIGNS) != (G->kind == TCG_SIGNS)) return cudaErrorInvalidValue;  // planned for the other kind
-  bool piped = G->mode == M_FP4 && outk == OUT_WORDS && out_type == 0 && G->words_even && G->all_fast;
+  bool piped = G->hot && outk == OUT_WORDS && out_type == 0;
   // rows are read two or four words at a time by the pipelined expanders: every input 8-byte aligned
   for (int i = 0; piped && i < G->count; ++i)
     if (reinterpret_cast<uintptr_t>(act[i]) & 7) piped = false;
