@@ -181,8 +181,8 @@ def run_reference(args):
 # the kernel's sources are the ones that were profiled: {kernel: (workload, batch, bytes, sha256 of sources)}
 _TRAFFIC = {
     # profiles/dram_traffic_resnet18_stack_n64_grouped.txt: mean of the two captured launches
-    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 351878912,
-                                             "314c22579083c5d34dbd81d82e9ccc88b2956fe90749d4096e4318c48d135b0b"),
+    "tcg_conv_kernel (grouped decoded_tc)": ("resnet18", 64, 351645312,
+                                             "80cb07752f0febac30141a098d3da70cbee8f49414eaad1867e0df037338bf63"),
 }
 
 
