@@ -106,7 +106,11 @@ SNN_API snn_status_t snn_conv_create(const snn_conv_desc_t* desc, snn_conv_t** o
  * DEVICE pointers owned by the caller (layouts above), act_dev 16-byte aligned,
  * out_dev 16-byte aligned; they are neither kept nor freed.  The call is
  * asynchronous on cuda_stream (a cudaStream_t, NULL = default stream) and does
- * not allocate.  N may be 0 (nothing is launched).
+ * not allocate, with one exception: the tensor-core path builds its plan and its
+ * tiled weight operand (device memory owned by the handle) at the first call for
+ * an input shape and output kind, so make that first call outside stream capture
+ * (snn_conv_tune for the shape does it for fp32 and int32 outputs).  N may be 0
+ * (nothing is launched).
  * Errors: INVALID_ARG (null, H/W giving no output, I32 or BITS output with fp16
  * activations, unknown path), UNSUPPORTED (the named path cannot run this
  * layer; AUTO never returns it, except for SNN_OUT_BITS on a layer the
